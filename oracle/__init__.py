@@ -1,0 +1,14 @@
+"""CPU oracle (test infrastructure only).
+
+Only tests, the smoke check and the benchmark's cpu_baseline / reference legs may
+import this package.  The CUDA library never does.
+"""
+from .ps_oracle import (  # noqa: F401
+    Oracle,
+    OracleConfig,
+    build_oracle,
+    philox4x32,
+    row_stats,
+    uniforms,
+    verify,
+)
