@@ -1,0 +1,207 @@
+/* ps.h -- C ABI of the ParallelSpec draft+verify library for NVIDIA B200 (sm_100a).
+ *
+ * One context = one drafter (weights + per-sequence KV caches) on one GPU.
+ * The drafter is the EAGLE-style parallel drafter of the paper: a fully connected
+ * layer over [token embedding ; target feature] followed by ONE Llama-style
+ * Transformer layer with the target layer's hyper-parameters, decoded by the target's
+ * LM head (Sec. 4.3, Sec. 5.1 "Models").  One call of ps_draft_step evaluates the last
+ * real position plus k appended [MASK] positions in a single pass and so yields k+1
+ * next-token distributions (Sec. 4.1 "Inference"); ps_verify applies speculative-sampling
+ * acceptance (Eq. 1; Algorithm 1 with one child per node) against target logits.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA global memory of the context's GPU, "host" pointers are
+ *     ordinary process memory.  Every tensor is dense, row-major, innermost index last.
+ *   - The library allocates no device memory.  Weights, inputs, outputs and the workspace
+ *     are owned by the caller and must stay valid while the context uses them.
+ *   - dtype 0: weights, hidden states and the KV cache are float; dtype 1: bf16
+ *     (accumulation is fp32 in both).  Logits and statistics are always float.
+ *   - Calls validate on the host, enqueue work on the given CUDA stream (a cudaStream_t
+ *     passed as void*, NULL = default stream) and return without waiting.  Conditions found
+ *     on the device (non-finite logits) set a device status word that ps_poll reads.
+ *   - Every function returns a negative ps_status on error and never aborts; after an error
+ *     outputs are unspecified but nothing outside the declared extents is written.
+ */
+#ifndef PS_H_
+#define PS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ps_ctx ps_ctx; /* opaque, host memory owned by the library */
+
+typedef enum {
+  PS_OK = 0,
+  PS_ERR_INVALID_ARG = -1, /* null pointer, size out of range, slot used twice in a batch */
+  PS_ERR_UNSUPPORTED = -2, /* a shape the kernels do not cover (see ps_init) */
+  PS_ERR_CAPACITY = -3,    /* a KV slab or the workspace is too small */
+  PS_ERR_CUDA = -4,        /* a CUDA runtime call failed; ps_last_error has its text */
+  PS_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired */
+  PS_ERR_NONFINITE = -6    /* NaN or +inf met in logits given to ps_verify */
+} ps_status;
+
+enum { PS_DTYPE_F32 = 0, PS_DTYPE_BF16 = 1 };
+enum {
+  PS_FLAG_FC_BIAS = 1,          /* ps_weights.b_fc is used */
+  PS_FLAG_UNFUSED_KERNELS = 2   /* force the unfused fp32-activation kernels (debugging aid) */
+};
+enum { PS_MAX_BATCH = 128, PS_MAX_MASKS = 15, PS_MAX_TOP_N = 8 };
+
+typedef struct ps_config {
+  int dtype;      /* PS_DTYPE_* */
+  int hidden;     /* H, multiple of 8 */
+  int n_heads;    /* query heads; n_heads * head_dim is the attention width */
+  int n_kv_heads; /* divides n_heads */
+  int head_dim;   /* 64 or 128 */
+  int ffn;        /* SwiGLU inner width F, multiple of 8 */
+  int vocab;      /* V */
+  int k_masks;    /* number of [MASK] positions k (Sec. 4.1), 0..PS_MAX_MASKS */
+  int max_batch;  /* number of sequence slots, 1..PS_MAX_BATCH */
+  int max_ctx;    /* KV rows per slot, INCLUDING the k+1 uncommitted rows of a draft step */
+  float rope_base;
+  float rms_eps;
+  int flags;      /* PS_FLAG_* */
+} ps_config;
+
+/* Device pointers, storage type given by ps_config.dtype, matrices row-major [out][in].
+ * Sec. 4.3: embed and w_lm are the target's (frozen) embedding and LM head; mask_embed and
+ * mask_feat are the k learned [MASK] inputs of the fc layer (embedding half, feature half). */
+typedef struct ps_weights {
+  const void* embed;      /* [V][H] */
+  const void* mask_embed; /* [k][H] */
+  const void* mask_feat;  /* [k][H] */
+  const void* w_fc;       /* [H][2H], input order [embedding ; feature] */
+  const void* b_fc;       /* [H] or NULL */
+  const void* g_in;       /* [H] RMSNorm gain before attention */
+  const void* w_q;        /* [n_heads*head_dim][H] */
+  const void* w_k;        /* [n_kv_heads*head_dim][H] */
+  const void* w_v;        /* [n_kv_heads*head_dim][H] */
+  const void* w_o;        /* [H][n_heads*head_dim] */
+  const void* g_post;     /* [H] RMSNorm gain before the FFN */
+  const void* w_gate;     /* [F][H] */
+  const void* w_up;       /* [F][H] */
+  const void* w_down;     /* [H][F] */
+  const void* g_final;    /* [H] RMSNorm gain before the LM head */
+  const void* w_lm;       /* [V][H] */
+} ps_weights;
+
+/* Bytes of device workspace ps_init needs for this configuration (KV slabs for max_batch
+ * slots, activation buffers, verify scratch).  Returns 0 if the configuration is invalid. */
+size_t ps_workspace_bytes(const ps_config* cfg);
+
+/* Creates a context.  `workspace` is device memory of at least ps_workspace_bytes(cfg) bytes,
+ * 256-byte aligned; the library zero-initialises what it needs on `stream`.  All KV caches
+ * start empty.  PS_ERR_UNSUPPORTED: head_dim not 64/128, hidden or ffn not a multiple of 8,
+ * n_heads not a multiple of n_kv_heads.  The CUDA device current at this call is the
+ * context's device. */
+ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* weights, void* workspace,
+                  size_t workspace_bytes, void* stream);
+
+/* Appends real positions to the drafter's KV caches (Sec. 4.1: only real tokens persist; the
+ * [MASK] rows of a draft step are never cached).  For sequence i of the call, rows
+ * row_offset[i] .. row_offset[i]+n_new[i]-1 of `hidden` / `tokens` are its new (target
+ * feature, token) pairs in order; they pass through the fc layer, the pre-attention norm and
+ * the K/V projections (+RoPE at their absolute positions) and land at cache rows
+ * [len, len+n_new), then len += n_new.
+ *   B            number of sequences in this call (1..max_batch)
+ *   seq_slot     host [B], distinct slots in [0, max_batch)
+ *   n_new        host [B], >= 0
+ *   row_offset   host [B+1], row_offset[0] = 0, row_offset[i+1] = row_offset[i] + n_new[i]
+ *   hidden       device [total][H], config dtype
+ *   tokens       device [total] int32 in [0, V)
+ * PS_ERR_CAPACITY if len + n_new > max_ctx for a sequence (nothing is appended). */
+ps_status ps_kv_append(ps_ctx* ctx, int B, const int* seq_slot, const int* n_new,
+                       const int* row_offset, const void* hidden, const int* tokens, void* stream);
+
+/* One parallel draft step (Sec. 4.1 "Inference"; the k+1 distributions of Algorithm 1).
+ * For each sequence: row 0 is the last real position (token_last, hidden_last), rows 1..k are
+ * [MASK]_1..[MASK]_k; row j sits at position len+j, attends to the cached real positions and
+ * to rows 0..j, and its logits are the drafter's distribution for the token j places after
+ * the next one.  The committed cache length does not change; rows [len, len+k] of the slab
+ * are overwritten as scratch.  Calling it twice gives identical outputs.
+ *   B            sequences (1..max_batch);  seq_slot host [B], distinct
+ *   hidden_last  device [B][H], config dtype;  token_last device [B] int32
+ *   top_n        0..PS_MAX_TOP_N entries per row (0: top_ids/top_logit unused)
+ *   top_ids      device [B][k+1][top_n] int32, descending logit, ties to the lower id
+ *   top_logit    device [B][k+1][top_n] float
+ *   row_max      device [B][k+1] float, max logit of the row (or NULL)
+ *   row_lse      device [B][k+1] float, log-sum-exp of the row (or NULL)
+ *   logits_out   device [B][k+1][V] float, or NULL to keep logits out of memory
+ *   feat_out     device [B][k+1][H] float, or NULL: the layer output before the final norm
+ *                (the drafted feature of Sec. 4.3)
+ * PS_ERR_CAPACITY if len + k + 1 > max_ctx. */
+ps_status ps_draft_step(ps_ctx* ctx, int B, const int* seq_slot, const void* hidden_last,
+                        const int* token_last, int top_n, int* top_ids, float* top_logit,
+                        float* row_max, float* row_lse, float* logits_out, float* feat_out,
+                        void* stream);
+
+/* Lossless verification of a drafted chain (Eq. 1; Algorithm 1 with one child per node).
+ * For position i = 0..n_draft-1 of sequence b, with p = softmax(target_logits[b][i]/T),
+ * q = softmax(draft_logits[b][i]/T) and x = draft_tokens[b][i]: accept iff
+ * r < min(1, p(x)/q(x)); at the first rejection emit one token drawn from
+ * max(0, p-q) normalised and stop; if every draft is accepted and n_target = n_draft+1, emit
+ * one token drawn from p of the extra row.  r and the sampling uniform are words 0 and 1 of
+ * Philox-4x32-10 with key = seed and counter = (i, b, offset), mapped to [0,1) by their top
+ * 24 bits.  temperature 0 is greedy: accept iff x is the arg-max of the target row (ties to
+ * the lower id), emit the arg-max otherwise.
+ *   draft_tokens  device [B][n_draft] int32
+ *   draft_logits  device [B][n_draft][V] float, or NULL: q is the point mass on x
+ *   target_logits device [B][n_target][V] float, n_target = n_draft or n_draft+1
+ *   accept_len    device [B] int32: number of accepted drafts
+ *   out_tokens    device [B][n_draft+1] int32: accepted drafts, then the emitted token, then -1
+ *   n_out         device [B] int32: tokens written to out_tokens
+ * 1 <= n_draft <= PS_MAX_MASKS+1.  NaN or +inf in a row that is examined: that position is
+ * rejected, the arg-max over its non-NaN target logits is emitted and ps_poll reports
+ * PS_ERR_NONFINITE. */
+ps_status ps_verify(ps_ctx* ctx, int B, int n_draft, int n_target, const int* draft_tokens,
+                    const float* draft_logits, const float* target_logits, float temperature,
+                    uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
+                    void* stream);
+
+/* Host-buffer convenience for one draft+verify round: copies hidden_last / token_last /
+ * target_logits from host memory, runs ps_draft_step (arg-max drafts of all k+1 rows) and
+ * ps_verify (n_draft = n_target = k+1) on `stream`, copies accept_len / out_tokens / n_out
+ * back and waits for the stream.  All pointers except ctx are host memory; pinned memory
+ * makes the copies asynchronous.
+ *   hidden_last [B][H] config dtype, token_last [B], target_logits [B][k+1][V] float,
+ *   accept_len [B], out_tokens [B][k+2], n_out [B]. */
+ps_status ps_round_host(ps_ctx* ctx, int B, const int* seq_slot, const void* hidden_last,
+                        const int* token_last, const float* target_logits, float temperature,
+                        uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,
+                        int* n_out, void* stream);
+
+/* Committed cache length of a slot (host bookkeeping, no device access). */
+ps_status ps_kv_len(ps_ctx* ctx, int slot, int* len);
+/* Empties a slot's cache (host bookkeeping only; nothing is enqueued). */
+ps_status ps_kv_reset(ps_ctx* ctx, int slot);
+
+/* Test helpers: copy a slot's committed cache rows out of / into the slab.
+ * K, V: device [len][n_kv_heads*head_dim] in config dtype (K as cached, i.e. after RoPE). */
+ps_status ps_kv_export(ps_ctx* ctx, int slot, void* K, void* V, void* stream);
+ps_status ps_kv_import(ps_ctx* ctx, int slot, int len, const void* K, const void* V, void* stream);
+
+/* Waits for `stream`, then returns and clears the device status word: PS_OK,
+ * PS_ERR_NONFINITE or PS_ERR_TIMEOUT. */
+ps_status ps_poll(ps_ctx* ctx, void* stream);
+
+/* Number of kernel launches the context has enqueued so far (host counter). */
+long long ps_launch_count(ps_ctx* ctx);
+
+/* Text of the last error of this context (host string owned by the context). */
+const char* ps_last_error(ps_ctx* ctx);
+void ps_destroy(ps_ctx* ctx);
+
+/* Philox-4x32-10 (Salmon et al., SC'11) evaluated on the device for n counters:
+ * out[i] = philox(key, ctr[i]).  key: host [2]; ctr, out: device [n][4] uint32.  Lets a caller
+ * check that the device stream equals the published generator word for word. */
+ps_status ps_philox_fill(const uint32_t key[2], const uint32_t* ctr, uint32_t* out, int n,
+                         void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PS_H_ */

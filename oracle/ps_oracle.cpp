@@ -200,10 +200,14 @@ inline double prob(const float* row, int v, double T, const RowStat& s) {
   return std::exp((double)row[v] / T - s.zmax) / s.S;
 }
 
+// Arg-max with ties to the lower id; a NaN entry counts as -inf.
 int argmax_row(const float* row, int V) {
   int best = 0;
-  for (int v = 1; v < V; ++v)
-    if (row[v] > row[best]) best = v;  // ties keep the lower id
+  double bv = std::isnan(row[0]) ? -std::numeric_limits<double>::infinity() : (double)row[0];
+  for (int v = 1; v < V; ++v) {
+    double x = std::isnan(row[v]) ? -std::numeric_limits<double>::infinity() : (double)row[v];
+    if (x > bv) { best = v; bv = x; }
+  }
   return best;
 }
 

@@ -1,0 +1,315 @@
+// C ABI entry points: argument validation, workspace carve-up, host bookkeeping of the
+// cache lengths and the choice of kernels.  See include/ps.h for the contract of each call.
+#include <algorithm>
+#include <cstring>
+
+#include "ps_internal.cuh"
+
+namespace ps {
+
+ps_status fail(ps_ctx* c, ps_status s, const std::string& what) {
+  if (c) c->err = what;
+  return s;
+}
+
+ps_status cuda_check(ps_ctx* c, cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return PS_OK;
+  if (c) c->err = std::string(what) + ": " + cudaGetErrorString(e);
+  return PS_ERR_CUDA;
+}
+
+namespace {
+
+size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+size_t elem_bytes(const ps_config& g) { return g.dtype == PS_DTYPE_F32 ? 4 : 2; }
+
+ps_status check_config(const ps_config* g) {
+  if (!g) return PS_ERR_INVALID_ARG;
+  if (g->dtype != PS_DTYPE_F32 && g->dtype != PS_DTYPE_BF16) return PS_ERR_INVALID_ARG;
+  if (g->hidden <= 0 || g->n_heads <= 0 || g->n_kv_heads <= 0 || g->ffn <= 0 || g->vocab <= 0)
+    return PS_ERR_INVALID_ARG;
+  if (g->k_masks < 0 || g->k_masks > PS_MAX_MASKS) return PS_ERR_INVALID_ARG;
+  if (g->max_batch < 1 || g->max_batch > PS_MAX_BATCH) return PS_ERR_INVALID_ARG;
+  if (g->max_ctx < g->k_masks + 1) return PS_ERR_INVALID_ARG;
+  if (!(g->rope_base > 1.f) || !(g->rms_eps >= 0.f)) return PS_ERR_INVALID_ARG;
+  if (g->head_dim != 64 && g->head_dim != 128) return PS_ERR_UNSUPPORTED;
+  if (g->hidden % 8 || g->ffn % 8) return PS_ERR_UNSUPPORTED;
+  if (g->n_heads % g->n_kv_heads) return PS_ERR_UNSUPPORTED;
+  return PS_OK;
+}
+
+// Walks the workspace layout; with c == nullptr only the size is computed.
+size_t carve(const ps_config& g, ps_ctx* c, char* base) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = off;
+    off = align_up(off + bytes);
+    return base ? base + at : nullptr;
+  };
+  const size_t H = g.hidden, Hq = (size_t)g.n_heads * g.head_dim,
+               Hkv = (size_t)g.n_kv_heads * g.head_dim, F = g.ffn, V = g.vocab;
+  const size_t R = g.k_masks + 1;
+  const size_t Md = (size_t)g.max_batch * R;                      // rows of a draft step
+  const size_t Mx = std::max<size_t>(Md, kAppendChunk);           // rows of fc / norm / kv
+  const size_t kv = (size_t)g.max_batch * g.n_kv_heads * g.max_ctx * g.head_dim * elem_bytes(g);
+  void* kc = take(kv);
+  void* vc = take(kv);
+  void* status = take(256);
+  void* tickets = take(sizeof(unsigned) * PS_MAX_BATCH);
+  void* vrec = take(sizeof(VerifyRec) * PS_MAX_BATCH * (PS_MAX_MASKS + 2));
+  void* x_in = take(Mx * 2 * H * 4);
+  void* x0 = take(Mx * H * 4);
+  void* xn = take(Mx * H * 4);
+  void* q = take(Md * Hq * 4);
+  void* kv_tmp = take(Mx * 2 * Hkv * 4);
+  void* attn = take(Md * Hq * 4);
+  void* a = take(Md * H * 4);
+  void* an = take(Md * H * 4);
+  void* gate = take(Md * F * 4);
+  void* up = take(Md * F * 4);
+  void* hdn = take(Md * H * 4);
+  void* hn = take(Md * H * 4);
+  void* logits = take(Md * V * 4);
+  void* st_hidden = take((size_t)g.max_batch * H * elem_bytes(g));
+  void* st_tok = take((size_t)g.max_batch * 4);
+  void* st_tlogits = take(Md * V * 4);
+  void* st_dlogits = take(Md * V * 4);
+  void* st_top = take(Md * 8);  // arg-max ids, then their logits
+  void* st_res = take((size_t)g.max_batch * (R + 3) * 4);
+  if (c) {
+    c->kcache = kc; c->vcache = vc; c->dev_status = (int*)status; c->tickets = (unsigned*)tickets;
+    c->vrec = (VerifyRec*)vrec;
+    c->x_in = (float*)x_in; c->x0 = (float*)x0; c->xn = (float*)xn; c->q = (float*)q;
+    c->kv_tmp = (float*)kv_tmp; c->attn = (float*)attn; c->a = (float*)a; c->an = (float*)an;
+    c->gate = (float*)gate; c->up = (float*)up; c->hdn = (float*)hdn; c->hn = (float*)hn;
+    c->logits = (float*)logits;
+    c->st_hidden = st_hidden; c->st_tok = (int*)st_tok; c->st_tlogits = (float*)st_tlogits;
+    c->st_dlogits = (float*)st_dlogits; c->st_top = (int*)st_top; c->st_res = (int*)st_res;
+    c->max_rows = (int)Md;
+  }
+  return off;
+}
+
+ps_status check_slots(ps_ctx* c, int B, const int* seq_slot) {
+  if (B < 1 || B > c->cfg.max_batch || !seq_slot) return fail(c, PS_ERR_INVALID_ARG, "bad batch");
+  bool seen[PS_MAX_BATCH] = {false};
+  for (int b = 0; b < B; ++b) {
+    int s = seq_slot[b];
+    if (s < 0 || s >= c->cfg.max_batch || seen[s])
+      return fail(c, PS_ERR_INVALID_ARG, "slot out of range or used twice");
+    seen[s] = true;
+  }
+  return PS_OK;
+}
+
+}  // namespace
+}  // namespace ps
+
+using namespace ps;
+
+extern "C" {
+
+size_t ps_workspace_bytes(const ps_config* cfg) {
+  if (check_config(cfg) != PS_OK) return 0;
+  return carve(*cfg, nullptr, nullptr);
+}
+
+ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* w, void* workspace,
+                  size_t workspace_bytes, void* stream) {
+  if (!out || !w || !workspace) return PS_ERR_INVALID_ARG;
+  ps_status s = check_config(cfg);
+  if (s != PS_OK) return s;
+  if (((uintptr_t)workspace & 255) != 0) return PS_ERR_INVALID_ARG;
+  if (workspace_bytes < carve(*cfg, nullptr, nullptr)) return PS_ERR_CAPACITY;
+  const void* need[] = {w->embed, w->w_fc, w->g_in, w->w_q, w->w_k, w->w_v, w->w_o, w->g_post,
+                        w->w_gate, w->w_up, w->w_down, w->g_final, w->w_lm};
+  for (const void* p : need)
+    if (!p) return PS_ERR_INVALID_ARG;
+  if (cfg->k_masks > 0 && (!w->mask_embed || !w->mask_feat)) return PS_ERR_INVALID_ARG;
+  if ((cfg->flags & PS_FLAG_FC_BIAS) && !w->b_fc) return PS_ERR_INVALID_ARG;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return PS_ERR_CUDA;
+  ps_ctx* c = new ps_ctx();
+  c->cfg = *cfg;
+  c->w = *w;
+  c->device = dev;
+  c->ws = (char*)workspace;
+  c->ws_bytes = workspace_bytes;
+  c->launches = 0;
+  c->len.assign(cfg->max_batch, 0);
+  carve(*cfg, c, c->ws);
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemsetAsync(c->dev_status, 0, 256, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * PS_MAX_BATCH, st);
+  if (e != cudaSuccess) {
+    delete c;
+    return PS_ERR_CUDA;
+  }
+  *out = c;
+  return PS_OK;
+}
+
+void ps_destroy(ps_ctx* c) { delete c; }
+
+const char* ps_last_error(ps_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+long long ps_launch_count(ps_ctx* c) { return c ? c->launches : 0; }
+
+ps_status ps_kv_len(ps_ctx* c, int slot, int* len) {
+  if (!c || !len || slot < 0 || slot >= c->cfg.max_batch) return PS_ERR_INVALID_ARG;
+  *len = c->len[slot];
+  return PS_OK;
+}
+
+ps_status ps_kv_reset(ps_ctx* c, int slot) {
+  if (!c || slot < 0 || slot >= c->cfg.max_batch) return PS_ERR_INVALID_ARG;
+  c->len[slot] = 0;
+  return PS_OK;
+}
+
+ps_status ps_kv_export(ps_ctx* c, int slot, void* K, void* V, void* stream) {
+  if (!c || !K || !V || slot < 0 || slot >= c->cfg.max_batch) return PS_ERR_INVALID_ARG;
+  return launch_kv_copy(c, slot, c->len[slot], K, V, false, (cudaStream_t)stream);
+}
+
+ps_status ps_kv_import(ps_ctx* c, int slot, int len, const void* K, const void* V, void* stream) {
+  if (!c || slot < 0 || slot >= c->cfg.max_batch || len < 0) return PS_ERR_INVALID_ARG;
+  if (len > 0 && (!K || !V)) return PS_ERR_INVALID_ARG;
+  if (len > c->cfg.max_ctx) return fail(c, PS_ERR_CAPACITY, "import exceeds max_ctx");
+  ps_status s = launch_kv_copy(c, slot, len, (void*)K, (void*)V, true, (cudaStream_t)stream);
+  if (s == PS_OK) c->len[slot] = len;
+  return s;
+}
+
+ps_status ps_poll(ps_ctx* c, void* stream) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, c->dev_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->dev_status, 0, sizeof(int), st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_check(c, e, "ps_poll");
+  if (word & kStatTimeout) return fail(c, PS_ERR_TIMEOUT, "a bounded device wait expired");
+  if (word & kStatNonfinite) return fail(c, PS_ERR_NONFINITE, "non-finite logits in ps_verify");
+  return PS_OK;
+}
+
+ps_status ps_kv_append(ps_ctx* c, int B, const int* seq_slot, const int* n_new,
+                       const int* row_offset, const void* hidden, const int* tokens, void* stream) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  ps_status s = check_slots(c, B, seq_slot);
+  if (s != PS_OK) return s;
+  if (!n_new || !row_offset) return fail(c, PS_ERR_INVALID_ARG, "null n_new / row_offset");
+  if (row_offset[0] != 0) return fail(c, PS_ERR_INVALID_ARG, "row_offset[0] must be 0");
+  for (int b = 0; b < B; ++b) {
+    if (n_new[b] < 0 || row_offset[b + 1] != row_offset[b] + n_new[b])
+      return fail(c, PS_ERR_INVALID_ARG, "row_offset does not match n_new");
+    if (c->len[seq_slot[b]] + n_new[b] > c->cfg.max_ctx)
+      return fail(c, PS_ERR_CAPACITY, "append exceeds max_ctx");
+  }
+  int total = row_offset[B];
+  if (total == 0) return PS_OK;
+  if (!hidden || !tokens) return fail(c, PS_ERR_INVALID_ARG, "null hidden / tokens");
+  SeqMap sm;
+  std::memset(&sm, 0, sizeof(sm));
+  sm.B = B;
+  for (int b = 0; b < B; ++b) {
+    sm.slot[b] = seq_slot[b];
+    sm.len[b] = c->len[seq_slot[b]];
+    sm.row_off[b] = row_offset[b];
+  }
+  sm.row_off[B] = total;
+  for (int r0 = 0; r0 < total; r0 += kAppendChunk) {
+    sm.row_base = r0;
+    int rows = std::min(kAppendChunk, total - r0);
+    s = plain_kv_append(c, sm, rows, hidden, tokens, (cudaStream_t)stream);
+    if (s != PS_OK) return s;
+  }
+  for (int b = 0; b < B; ++b) c->len[seq_slot[b]] += n_new[b];
+  return PS_OK;
+}
+
+ps_status ps_draft_step(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,
+                        const int* token_last, int top_n, int* top_ids, float* top_logit,
+                        float* row_max, float* row_lse, float* logits_out, float* feat_out,
+                        void* stream) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  ps_status s = check_slots(c, B, seq_slot);
+  if (s != PS_OK) return s;
+  if (!hidden_last || !token_last) return fail(c, PS_ERR_INVALID_ARG, "null hidden / token");
+  if (top_n < 0 || top_n > PS_MAX_TOP_N || top_n > c->cfg.vocab)
+    return fail(c, PS_ERR_INVALID_ARG, "top_n out of range");
+  if (top_n > 0 && (!top_ids || !top_logit)) return fail(c, PS_ERR_INVALID_ARG, "null top-n output");
+  const int R = c->cfg.k_masks + 1;
+  SeqMap sm;
+  std::memset(&sm, 0, sizeof(sm));
+  sm.B = B;
+  for (int b = 0; b < B; ++b) {
+    sm.slot[b] = seq_slot[b];
+    sm.len[b] = c->len[seq_slot[b]];
+    sm.row_off[b] = b * R;
+    if (sm.len[b] + R > c->cfg.max_ctx) return fail(c, PS_ERR_CAPACITY, "no room for the draft rows");
+  }
+  sm.row_off[B] = B * R;
+  return plain_draft_step(c, sm, B, hidden_last, token_last, top_n, top_ids, top_logit, row_max,
+                          row_lse, logits_out, feat_out, (cudaStream_t)stream);
+}
+
+ps_status ps_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draft_tokens,
+                    const float* draft_logits, const float* target_logits, float temperature,
+                    uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
+                    void* stream) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  if (B < 1 || B > PS_MAX_BATCH) return fail(c, PS_ERR_INVALID_ARG, "bad batch");
+  if (n_draft < 1 || n_draft > PS_MAX_MASKS + 1) return fail(c, PS_ERR_INVALID_ARG, "bad n_draft");
+  if (n_target != n_draft && n_target != n_draft + 1)
+    return fail(c, PS_ERR_INVALID_ARG, "n_target must be n_draft or n_draft+1");
+  if (!draft_tokens || !target_logits || !accept_len || !out_tokens || !n_out)
+    return fail(c, PS_ERR_INVALID_ARG, "null pointer");
+  if (!(temperature >= 0.f)) return fail(c, PS_ERR_INVALID_ARG, "temperature must be >= 0");
+  return launch_verify(c, B, n_draft, n_target, draft_tokens, draft_logits, target_logits,
+                       temperature, seed, offset, accept_len, out_tokens, n_out,
+                       (cudaStream_t)stream);
+}
+
+ps_status ps_round_host(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,
+                        const int* token_last, const float* target_logits, float temperature,
+                        uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,
+                        int* n_out, void* stream) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  ps_status s = check_slots(c, B, seq_slot);
+  if (s != PS_OK) return s;
+  if (!hidden_last || !token_last || !target_logits || !accept_len || !out_tokens || !n_out)
+    return fail(c, PS_ERR_INVALID_ARG, "null pointer");
+  cudaStream_t st = (cudaStream_t)stream;
+  const ps_config& g = c->cfg;
+  const int R = g.k_masks + 1;
+  const size_t eb = g.dtype == PS_DTYPE_F32 ? 4 : 2;
+  cudaError_t e;
+  e = cudaMemcpyAsync(c->st_hidden, hidden_last, (size_t)B * g.hidden * eb, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(c->st_tok, token_last, (size_t)B * 4, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(c->st_tlogits, target_logits, (size_t)B * R * g.vocab * 4,
+                        cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return cuda_check(c, e, "ps_round_host h2d");
+  // top_n = 1: top_ids is then exactly the [B][k+1] chain of arg-max drafts.
+  s = ps_draft_step(c, B, seq_slot, c->st_hidden, c->st_tok, 1, c->st_top, (float*)(c->st_top + (size_t)c->max_rows),
+                    nullptr, nullptr, c->st_dlogits, nullptr, st);
+  if (s != PS_OK) return s;
+  int* r_acc = c->st_res;
+  int* r_n = c->st_res + B;
+  int* r_out = c->st_res + 2 * B;
+  s = ps_verify(c, B, R, R, c->st_top, c->st_dlogits, c->st_tlogits, temperature, seed, offset,
+                r_acc, r_out, r_n, st);
+  if (s != PS_OK) return s;
+  e = cudaMemcpyAsync(accept_len, r_acc, (size_t)B * 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(n_out, r_n, (size_t)B * 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(out_tokens, r_out, (size_t)B * (R + 1) * 4, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  return cuda_check(c, e, "ps_round_host d2h");
+}
+
+}  // extern "C"

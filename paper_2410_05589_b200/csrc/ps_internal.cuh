@@ -1,0 +1,90 @@
+// Internal declarations shared by the translation units of the library.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "ps.h"
+
+namespace ps {
+
+constexpr int kMaxRowsPerSeq = PS_MAX_MASKS + 1;  // rows of one sequence in a draft step
+constexpr int kAppendChunk = 256;                 // rows handled per pass of ps_kv_append
+
+// Which sequence each row of a launch belongs to.  Passed by value as a kernel parameter.
+// Row m (0-based within the launch) belongs to the sequence b with
+// row_off[b] <= m + row_base < row_off[b+1]; its index inside the sequence is
+// j = m + row_base - row_off[b] and its absolute position is len[b] + j.
+struct SeqMap {
+  int B;
+  int row_base;
+  int slot[PS_MAX_BATCH];
+  int len[PS_MAX_BATCH];
+  int row_off[PS_MAX_BATCH + 1];
+};
+
+__device__ __forceinline__ void seq_of_row(const SeqMap& s, int m, int& b, int& j) {
+  int g = m + s.row_base;
+  int lo = 0, hi = s.B - 1;
+  while (lo < hi) {  // last b with row_off[b] <= g (empty sequences are skipped by taking the last)
+    int mid = (lo + hi + 1) >> 1;
+    if (s.row_off[mid] <= g) lo = mid; else hi = mid - 1;
+  }
+  b = lo;
+  j = g - s.row_off[lo];
+}
+
+// Device status word values (bit flags).
+constexpr int kStatNonfinite = 1;
+constexpr int kStatTimeout = 2;
+
+struct VerifyRec {  // one per (sequence, position): result of the acceptance test
+  int accept;       // bit 0: accepted; bit 1: a non-finite logit was met
+  int token;        // token to emit if this position ends the chain
+};
+
+}  // namespace ps
+
+struct ps_ctx {
+  ps_config cfg;
+  ps_weights w;
+  int device;
+  char* ws;
+  size_t ws_bytes;
+  int max_rows;    // rows the activation buffers hold
+  // workspace slices
+  void* kcache;    // [max_batch][n_kv_heads][max_ctx][head_dim] storage dtype, post-RoPE
+  void* vcache;
+  int* dev_status;
+  unsigned* tickets;        // [max_batch] arrival counters of the verify kernel (zero between calls)
+  ps::VerifyRec* vrec;      // [max_batch][PS_MAX_MASKS+2]
+  float *x_in, *x0, *xn, *q, *kv_tmp, *attn, *a, *an, *gate, *up, *hdn, *hn, *logits;
+  // staging for ps_round_host
+  void* st_hidden; int* st_tok; float* st_tlogits; float* st_dlogits; int* st_top; int* st_res;
+  std::vector<int> len;     // committed positions per slot (host is the source of truth)
+  long long launches;
+  std::string err;
+};
+
+namespace ps {
+
+ps_status fail(ps_ctx* c, ps_status s, const std::string& what);
+ps_status cuda_check(ps_ctx* c, cudaError_t e, const char* what);
+
+// ---- unfused kernels with fp32 activations (all dtypes, all shapes) -----------------------
+ps_status plain_kv_append(ps_ctx* c, const SeqMap& sm, int rows, const void* hidden,
+                          const int* tokens, cudaStream_t st);
+ps_status plain_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last,
+                           const int* token_last, int top_n, int* top_ids, float* top_logit,
+                           float* row_max, float* row_lse, float* logits_out, float* feat_out,
+                           cudaStream_t st);
+ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draft_tokens,
+                        const float* draft_logits, const float* target_logits, float temperature,
+                        uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,
+                        int* n_out, cudaStream_t st);
+ps_status launch_kv_copy(ps_ctx* c, int slot, int len, void* K, void* V, bool to_cache,
+                         cudaStream_t st);
+}  // namespace ps

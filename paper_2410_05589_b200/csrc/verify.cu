@@ -1,0 +1,352 @@
+// ps_verify: speculative-sampling acceptance for a drafted chain (Eq. 1; Algorithm 1 with one
+// child per node).  One thread block per (position, sequence) evaluates its row pair
+// speculatively: softmax statistics of the target and draft rows, the test r < min(1, p/q),
+// and -- if the test fails or the row is the extra target row -- the token that would be
+// emitted there (residual max(0, p-q) normalised, or p itself).  The last block of a sequence
+// to finish walks the positions in order and writes accept_len / out_tokens / n_out.
+// Nothing spins: blocks only take a ticket, the last arriver does the merge.
+#include <cfloat>
+
+#include "ps_internal.cuh"
+
+namespace ps {
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+constexpr int kSeg = 128;  // elements per warp-wide segment of the inverse-CDF search
+
+// Philox-4x32 with 10 rounds (Salmon et al., SC'11): counter (c0..c3), key (k0,k1).
+__device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t (&c)[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0 = __umulhi(0xD2511F53u, c[0]), lo0 = 0xD2511F53u * c[0];
+    uint32_t hi1 = __umulhi(0xCD9E8D57u, c[2]), lo1 = 0xCD9E8D57u * c[2];
+    uint32_t n0 = hi1 ^ c[1] ^ k0, n2 = hi0 ^ c[3] ^ k1;
+    c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+}
+
+__global__ void k_philox_fill(uint32_t k0, uint32_t k1, const uint32_t* ctr, uint32_t* out, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint32_t c[4] = {ctr[4 * i], ctr[4 * i + 1], ctr[4 * i + 2], ctr[4 * i + 3]};
+  philox4x32_10(k0, k1, c);
+  for (int j = 0; j < 4; ++j) out[4 * i + j] = c[j];
+}
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+struct Scratch {
+  float fmax[kWarps];
+  int imax[kWarps];
+  double dsum[kWarps];
+  int flag[kWarps];
+  float bc_f;
+  int bc_i;
+  double bc_d;
+  int bc_flag;
+};
+
+// Max over a row with NaN treated as -inf, ties to the lower index; also reports whether the
+// row holds a NaN or +inf (or nothing above -inf).  Result broadcast to all threads.
+__device__ void row_argmax(const float* row, int V, Scratch& s, float& vmax, int& imax, int& bad) {
+  float bv = -INFINITY;
+  int bi = 0x7fffffff, bd = 0;
+  for (int v = threadIdx.x; v < V; v += kThreads) {
+    float x = row[v];
+    if (x != x || x == INFINITY) bd = 1;
+    if (x != x) x = -INFINITY;
+    if (x > bv || (x == bv && v < bi)) { bv = x; bi = v; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+    int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    bd |= __shfl_xor_sync(0xffffffffu, bd, o);
+    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+  }
+  int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) { s.fmax[warp] = bv; s.imax[warp] = bi; s.flag[warp] = bd; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kWarps; ++w) {
+      if (s.fmax[w] > bv || (s.fmax[w] == bv && s.imax[w] < bi)) { bv = s.fmax[w]; bi = s.imax[w]; }
+      bd |= s.flag[w];
+    }
+    if (bv == -INFINITY) bd = 1;  // an all -inf row has no distribution
+    s.bc_f = bv; s.bc_i = bi; s.bc_flag = bd;
+  }
+  __syncthreads();
+  vmax = s.bc_f; imax = s.bc_i; bad = s.bc_flag;
+  __syncthreads();
+}
+
+// sum_v exp((row[v] - vmax) / T), accumulated in double, broadcast to all threads.
+__device__ double row_sumexp(const float* row, int V, float vmax, double inv_t, Scratch& s) {
+  double acc = 0.0;
+  for (int v = threadIdx.x; v < V; v += kThreads)
+    acc += (double)expf((float)(((double)row[v] - (double)vmax) * inv_t));
+  acc = warp_sum_d(acc);
+  if ((threadIdx.x & 31) == 0) s.dsum[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w = 0; w < kWarps; ++w) t += s.dsum[w];
+    s.bc_d = t;
+  }
+  __syncthreads();
+  double r = s.bc_d;
+  __syncthreads();
+  return r;
+}
+
+// Weight of token v in the distribution to sample: max(0, p_v - q_v), or p_v when use_q == 0.
+// q is softmax(drow/T) when drow != nullptr, else the point mass on x.
+__device__ __forceinline__ float weight_of(int v, const float* trow, const float* drow, int x,
+                                           int use_q, float tmax, float dmax, double inv_t,
+                                           float inv_st, float inv_sd) {
+  float p = expf((float)(((double)trow[v] - (double)tmax) * inv_t)) * inv_st;
+  if (!use_q) return p;
+  float q = drow ? expf((float)(((double)drow[v] - (double)dmax) * inv_t)) * inv_sd
+                 : (v == x ? 1.f : 0.f);
+  return fmaxf(p - q, 0.f);
+}
+
+// Inverse-CDF draw with uniform u from the weights above: the first v whose running sum
+// exceeds u * total.  seg_sum: shared array of ceil(V / kSeg) doubles.  Returns the token to
+// all threads; returns -1 if the total weight is not positive.
+__device__ int sample_weights(const float* trow, const float* drow, int x, int use_q, int V,
+                              float tmax, float dmax, double inv_t, double st, double sd,
+                              double u, double* seg_sum, Scratch& s) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nseg = (V + kSeg - 1) / kSeg;
+  const float inv_st = (float)(1.0 / st), inv_sd = (float)(1.0 / sd);
+  constexpr int E = kSeg / 32;
+  for (int g = warp; g < nseg; g += kWarps) {
+    double a = 0.0;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      int v = g * kSeg + lane * E + e;
+      if (v < V) a += (double)weight_of(v, trow, drow, x, use_q, tmax, dmax, inv_t, inv_st, inv_sd);
+    }
+    a = warp_sum_d(a);
+    if (lane == 0) seg_sum[g] = a;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    // lane owns segments [lane*c, lane*c + c)
+    int c = (nseg + 31) / 32;
+    int g_lo = min(nseg, lane * c), g_hi = min(nseg, lane * c + c);
+    double mine = 0.0;
+    for (int g = g_lo; g < g_hi; ++g) mine += seg_sum[g];
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      double t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    double total = __shfl_sync(0xffffffffu, incl, 31);
+    double target = u * total;
+    int token = -1;
+    if (total > 0.0) {  // uniform across the warp
+      // first lane whose inclusive sum exceeds the target, else the last lane with weight
+      unsigned over = __ballot_sync(0xffffffffu, incl > target);
+      unsigned pos = __ballot_sync(0xffffffffu, mine > 0.0);
+      int src = over ? __ffs(over) - 1 : (pos ? 31 - __clz(pos) : 0);
+      int gsel = -1;
+      double gbase = 0.0;
+      if (lane == src) {
+        double run = incl - mine;
+        int last_pos = -1;
+        double last_base = 0.0;
+        for (int g = g_lo; g < g_hi; ++g) {
+          if (seg_sum[g] > 0.0) { last_pos = g; last_base = run; }
+          if (run + seg_sum[g] > target) { gsel = g; gbase = run; break; }
+          run += seg_sum[g];
+        }
+        if (gsel < 0) { gsel = last_pos; gbase = last_base; }
+      }
+      gsel = __shfl_sync(0xffffffffu, gsel, src);
+      gbase = __shfl_sync(0xffffffffu, gbase, src);
+      // inside the segment: lane owns E consecutive tokens
+      float wv[E];
+      double lsum = 0.0;
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        int v = gsel * kSeg + lane * E + e;
+        wv[e] = (gsel >= 0 && v < V) ? weight_of(v, trow, drow, x, use_q, tmax, dmax, inv_t, inv_st, inv_sd) : 0.f;
+        lsum += (double)wv[e];
+      }
+      double linc = lsum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        double t = __shfl_up_sync(0xffffffffu, linc, o);
+        if (lane >= o) linc += t;
+      }
+      unsigned over2 = __ballot_sync(0xffffffffu, gbase + linc > target);
+      unsigned pos2 = __ballot_sync(0xffffffffu, lsum > 0.0);
+      int src2 = over2 ? __ffs(over2) - 1 : (pos2 ? 31 - __clz(pos2) : 0);
+      int pick = -1;
+      if (lane == src2 && gsel >= 0 && (over2 | pos2)) {
+        double run2 = gbase + linc - lsum;
+        int lastp = -1;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          if (wv[e] > 0.f) lastp = e;
+          run2 += (double)wv[e];
+          if (pick < 0 && run2 > target) pick = e;
+        }
+        if (pick < 0) pick = lastp;
+        pick = pick < 0 ? -1 : gsel * kSeg + lane * E + pick;
+      }
+      token = __shfl_sync(0xffffffffu, pick, src2);
+    }
+    if (lane == 0) s.bc_i = token;
+  }
+  __syncthreads();
+  int tok = s.bc_i;
+  __syncthreads();
+  return tok;
+}
+
+struct VerifyArgs {
+  int B, n_draft, n_target, V;
+  const int* draft_tokens;
+  const float* draft_logits;
+  const float* target_logits;
+  float temperature;
+  uint32_t key0, key1, off_lo, off_hi;
+  int* accept_len;
+  int* out_tokens;
+  int* n_out;
+  VerifyRec* rec;      // [B][PS_MAX_MASKS+2]
+  unsigned* tickets;   // [B], zero on entry and on exit
+  int* status;
+};
+
+__global__ void __launch_bounds__(kThreads) k_verify(VerifyArgs a) {
+  extern __shared__ double seg_sum[];
+  __shared__ Scratch s;
+  __shared__ int s_last;
+  const int i = blockIdx.x, b = blockIdx.y, V = a.V;
+  const bool bonus = i >= a.n_draft;
+  const float* trow = a.target_logits + ((size_t)b * a.n_target + i) * V;
+  const float* drow = (!bonus && a.draft_logits) ? a.draft_logits + ((size_t)b * a.n_draft + i) * V
+                                                 : nullptr;
+  int x = bonus ? -1 : a.draft_tokens[(size_t)b * a.n_draft + i];
+  int accept = 0, token = -1, bad = 0;
+
+  float tmax; int targ, tbad;
+  row_argmax(trow, V, s, tmax, targ, tbad);
+  if (a.temperature == 0.f) {
+    accept = (!bonus && x == targ) ? 1 : 0;
+    token = targ;
+  } else {
+    double inv_t = 1.0 / (double)a.temperature;
+    float dmax = 0.f; int darg, dbad = 0;
+    if (drow) row_argmax(drow, V, s, dmax, darg, dbad);
+    bad = tbad | dbad;
+    if (bad) {
+      token = targ;
+    } else {
+      double st = row_sumexp(trow, V, tmax, inv_t, s);
+      double sd = drow ? row_sumexp(drow, V, dmax, inv_t, s) : 1.0;
+      uint32_t c[4] = {(uint32_t)i, (uint32_t)b, a.off_lo, a.off_hi};
+      philox4x32_10(a.key0, a.key1, c);
+      double r = (double)(c[0] >> 8) * (1.0 / 16777216.0);
+      double u2 = (double)(c[1] >> 8) * (1.0 / 16777216.0);
+      if (!bonus) {
+        bool in_range = x >= 0 && x < V;
+        double logp = in_range ? ((double)trow[x] - (double)tmax) * inv_t - log(st) : -INFINITY;
+        double logq = drow ? (in_range ? ((double)drow[x] - (double)dmax) * inv_t - log(sd) : -INFINITY)
+                           : 0.0;
+        double diff = logp - logq;
+        double ratio = (diff != diff) ? 0.0 : exp(fmin(diff, 0.0));
+        accept = r < ratio ? 1 : 0;
+      }
+      if (!accept) {  // uniform across the block: every thread computed the same decision
+        token = sample_weights(trow, drow, x, bonus ? 0 : 1, V, tmax, dmax, inv_t, st, sd, u2,
+                               seg_sum, s);
+        if (token < 0)
+          token = sample_weights(trow, drow, x, 0, V, tmax, dmax, inv_t, st, sd, u2, seg_sum, s);
+        if (token < 0) token = targ;
+      }
+    }
+  }
+
+  if (threadIdx.x == 0) {
+    VerifyRec* rec = a.rec + (size_t)b * (PS_MAX_MASKS + 2);
+    rec[i].accept = accept | (bad << 1);
+    rec[i].token = token;
+    __threadfence();
+    unsigned t = atomicAdd(&a.tickets[b], 1u);
+    s_last = (t == (unsigned)a.n_target - 1u);
+  }
+  __syncthreads();
+  if (s_last && threadIdx.x == 0) {
+    __threadfence();
+    volatile VerifyRec* rec = a.rec + (size_t)b * (PS_MAX_MASKS + 2);
+    int* out = a.out_tokens + (size_t)b * (a.n_draft + 1);
+    int acc = 0, any_bad = 0, emitted = -1;
+    while (acc < a.n_draft) {
+      int f = rec[acc].accept;
+      any_bad |= (f >> 1) & 1;
+      if (!(f & 1)) { emitted = rec[acc].token; break; }
+      out[acc] = a.draft_tokens[(size_t)b * a.n_draft + acc];
+      ++acc;
+    }
+    if (acc == a.n_draft && a.n_target == a.n_draft + 1) {
+      any_bad |= (rec[acc].accept >> 1) & 1;
+      emitted = rec[acc].token;
+    }
+    int n = acc;
+    if (emitted >= 0) out[n++] = emitted;
+    for (int j = n; j <= a.n_draft; ++j) out[j] = -1;
+    a.accept_len[b] = acc;
+    a.n_out[b] = n;
+    if (any_bad) atomicOr(a.status, kStatNonfinite);
+    a.tickets[b] = 0u;
+  }
+}
+
+}  // namespace
+
+ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draft_tokens,
+                        const float* draft_logits, const float* target_logits, float temperature,
+                        uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,
+                        int* n_out, cudaStream_t st) {
+  VerifyArgs a;
+  a.B = B; a.n_draft = n_draft; a.n_target = n_target; a.V = c->cfg.vocab;
+  a.draft_tokens = draft_tokens; a.draft_logits = draft_logits; a.target_logits = target_logits;
+  a.temperature = temperature;
+  a.key0 = (uint32_t)seed; a.key1 = (uint32_t)(seed >> 32);
+  a.off_lo = (uint32_t)offset; a.off_hi = (uint32_t)(offset >> 32);
+  a.accept_len = accept_len; a.out_tokens = out_tokens; a.n_out = n_out;
+  a.rec = c->vrec; a.tickets = c->tickets; a.status = c->dev_status;
+  size_t smem = (size_t)((a.V + kSeg - 1) / kSeg) * sizeof(double);
+  if (smem > 160 * 1024) return fail(c, PS_ERR_UNSUPPORTED, "vocab too large for ps_verify");
+  if (smem > 40 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k_verify, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_check(c, e, "verify smem");
+  }
+  k_verify<<<dim3(n_target, B), kThreads, smem, st>>>(a);
+  c->launches++;
+  return cuda_check(c, cudaGetLastError(), "k_verify");
+}
+
+}  // namespace ps
+
+extern "C" ps_status ps_philox_fill(const uint32_t key[2], const uint32_t* ctr, uint32_t* out, int n,
+                                    void* stream) {
+  if (!key || !ctr || !out || n < 0) return PS_ERR_INVALID_ARG;
+  if (n == 0) return PS_OK;
+  ps::k_philox_fill<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>(key[0], key[1], ctr, out, n);
+  return cudaGetLastError() == cudaSuccess ? PS_OK : PS_ERR_CUDA;
+}
