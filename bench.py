@@ -1,0 +1,407 @@
+#!/usr/bin/env python
+"""Benchmark of the ParallelSpec hot path: ps_draft_step + ps_verify steps per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 13b|7b|33b|tiny]
+    python bench.py --impl reference ...      # the CPU checker timed on the host cores
+
+One "step" = one parallel draft step (all k+1 rows, logits stored) followed by one verify
+call on synthetic target logits, for the workload's batch.  N > 1 (under torchrun) runs N
+independent replicas, one per GPU, with no data-path collective.  Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "draft+verify steps/sec"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126 << 20
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="13b", choices=["13b", "7b", "33b", "tiny", "mini"])
+    ap.add_argument("--temperature", type=float, default=1.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def stage_bytes(s, B, lens):
+    """Algorithmic bytes each stage must move per step (weights once, KV once, logits written
+    once by the LM head and read once by verify together with the target logits)."""
+    e = 4 if s.dtype == 0 else 2
+    H, F, V = s.hidden, s.ffn, s.vocab
+    Hq, Hkv = s.n_heads * s.head_dim, s.n_kv_heads * s.head_dim
+    M = B * (s.k_masks + 1)
+    return {
+        "fc_norm": e * 2 * H * H,
+        "qkv_rope": e * (Hq * H + 2 * Hkv * H),
+        "attention": e * 2 * Hkv * int(sum(lens)),
+        "o_proj": e * H * Hq,
+        "ffn": e * 3 * H * F,
+        "lm_head": e * V * H + 4 * M * V,
+        "verify": 8 * M * V,
+    }
+
+
+def max_over_ranks(x: float, device="cuda") -> float:
+    """Slowest rank's value (every rank gets it).  Replicas exchange nothing else."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_steps_per_s(world: int, steps_per_rank: int, slowest_ms: float) -> float:
+    """Whole-job throughput of N independent replicas: all steps over the slowest rank's time."""
+    return world * steps_per_rank / (slowest_ms * 1e-3)
+
+
+class ClockSampler(threading.Thread):
+    """Reads SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, device_index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            h = None
+            for i in range(pynvml.nvmlDeviceGetCount()):
+                hi = pynvml.nvmlDeviceGetHandleByIndex(i)
+                u = pynvml.nvmlDeviceGetUUID(hi)
+                u = u.decode() if isinstance(u, bytes) else u
+                if uuid in u or u.replace("GPU-", "") == uuid:
+                    h = hi
+            self.h = h if h is not None else pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.nv = pynvml
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_setup(s, B, lens):
+    import oracle
+    import synth
+    from synth import bf16_bits_to_f32
+
+    W = synth.weights(s)
+    max_ctx = int(max(lens)) + s.rows
+    o = oracle.Oracle(oracle.OracleConfig(s.dtype, s.hidden, s.n_heads, s.n_kv_heads, s.head_dim,
+                                          s.ffn, s.vocab, s.k_masks, B, max_ctx, s.rope_base,
+                                          s.rms_eps), W)
+    for b in range(B):
+        K, V = synth.kv_rows(s, ("kv", b), int(lens[b]))
+        if s.dtype == 1:
+            K, V = bf16_bits_to_f32(K), bf16_bits_to_f32(V)
+        o.kv_import(b, K.astype("float64"), V.astype("float64"))
+    return o
+
+
+def oracle_time_step(o, s, b, k_use, hidden_last, token_last, target, T):
+    """Seconds of one oracle draft step (k_use+1 rows) + verify on those rows, sequence b."""
+    import numpy as np
+
+    import oracle
+
+    t0 = time.perf_counter()
+    out = o.draft_step(b, hidden_last[b:b + 1], int(token_last[b]), k_use=k_use)
+    lg = out["logits"].astype(np.float32)[None]
+    toks = lg.argmax(-1).astype(np.int32)
+    oracle.verify(toks, lg, target[b:b + 1, :k_use + 1], T, 1, 0)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(s, B, lens, hidden_last, token_last, target, T, budget_s):
+    """The CPU checker, as it stands, on a bounded sample of the same workload."""
+    import oracle
+
+    o = oracle_setup(s, B, lens)
+    R = s.rows
+    # first: one row of sequence 0 to size the sample
+    t_row = oracle_time_step(o, s, 0, 0, hidden_last, token_last, target, T)
+    full_step = t_row * R * B
+    if full_step <= budget_s:
+        n_seq, k_use = B, s.k_masks
+    elif t_row * R <= budget_s:
+        n_seq, k_use = max(1, int(budget_s / (t_row * R))), s.k_masks
+    else:
+        n_seq, k_use = 1, max(0, int(budget_s / t_row) - 1)
+    t = 0.0
+    for b in range(n_seq):
+        t += oracle_time_step(o, s, b, k_use, hidden_last, token_last, target, T)
+    rows_done = n_seq * (k_use + 1)
+    est_step = t * (B * R) / rows_done
+    sample = (f"{n_seq} of {B} sequences x {k_use + 1} of {R} rows of one draft+verify step "
+              f"({t:.1f} s), scaled by rows to a full step")
+    return {"value": 1.0 / est_step, "unit": "steps/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "sample": sample}
+
+
+def run_reference(args):
+    """--impl reference: the CPU checker timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import numpy as np
+
+    import oracle
+    import synth
+
+    s = synth.CONFIGS[args.workload]
+    B = s.batch
+    lens = synth.ctx_lengths(s, B)
+    o = oracle_setup(s, B, lens)
+    hl, tl = synth.hidden_states(s, "last", B), synth.token_ids(s, "last", B)
+    tgt = (synth.zipf_logits(s.seed, "tgt0", B, s.rows, s.vocab) if s.logits_kind == "zipf"
+           else synth.gauss_logits(s.seed, "tgt0", (B, s.rows, s.vocab)))
+    R = s.rows
+    t_row = oracle_time_step(o, s, 0, 0, hl, tl, tgt, args.temperature)
+    total_steps = args.steps + args.warmup
+    budget = 150.0 / max(1, total_steps)
+    k_use = min(s.k_masks, max(0, int(budget / t_row) - 1))
+    n_seq = 1 if t_row * (k_use + 1) * 2 > budget else min(B, max(1, int(budget / (t_row * (k_use + 1)))))
+    times = []
+    for i in range(total_steps):
+        t = sum(oracle_time_step(o, s, b, k_use, hl, tl, tgt, args.temperature) for b in range(n_seq))
+        if i >= args.warmup:
+            times.append(t)
+    per_step = (sum(times) / len(times)) * (B * R) / (n_seq * (k_use + 1))
+    value = 1.0 / per_step
+    sample = (f"each step: {n_seq} of {B} sequences x {k_use + 1} of {R} rows of the oracle's draft "
+              f"step + verify, scaled by rows to a full step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "steps/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(s, B, lens),
+        "cpu_baseline": {"value": value, "unit": "steps/s", "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "drafted_tokens_per_s": value * B * R,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(s, B, lens):
+    return {
+        "workload": f"{s.name}: H{s.hidden} heads{s.n_heads}x{s.head_dim} F{s.ffn} V{s.vocab} "
+                    f"B{B} k{s.k_masks} ctx{int(min(lens))}-{int(max(lens))} "
+                    f"{'fp32' if s.dtype == 0 else 'bf16'}",
+        "batch": B, "k_masks": s.k_masks, "rows_per_step": B * s.rows,
+        "verify": "n_draft=n_target=k+1, draft logits stored, Zipf(1.1)-biased target logits",
+    }
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2410_05589_b200 as ps
+    import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    s = synth.CONFIGS[args.workload]
+    B, R, V, T = s.batch, s.rows, s.vocab, args.temperature
+    lens = synth.ctx_lengths(s, B)
+    W = synth.weights(s)
+    kv_bytes_seq = 2 * s.n_kv_heads * s.head_dim * int(lens.mean()) * (4 if s.dtype == 0 else 2)
+    # rotate over enough distinct KV sets that consecutive steps never find their KV in L2
+    n_sets = 1 if kv_bytes_seq * B > 2 * L2_BYTES else max(2, min(16, -(-2 * L2_BYTES // max(1, kv_bytes_seq * B))))
+    n_sets = min(n_sets, 128 // B)
+    g = ps.drafter_from_shape(s, W, max_batch=B * n_sets, max_ctx=int(lens.max()) + R)
+    del W
+    for i in range(n_sets):
+        for b in range(B):
+            K, Vv = synth.kv_rows(s, ("kv", b), int(lens[b]))
+            g.kv_import(i * B + b, ps.to_device(K), ps.to_device(Vv))
+    hl_np, tl_np = synth.hidden_states(s, "last", B), synth.token_ids(s, "last", B)
+    tgt_np = [(synth.zipf_logits(s.seed, f"tgt{i}", B, R, V) if s.logits_kind == "zipf"
+               else synth.gauss_logits(s.seed, f"tgt{i}", (B, R, V))) for i in range(min(n_sets, 4))]
+    hl, tl = ps.to_device(hl_np), ps.to_device(tl_np)
+    tgt = [ps.to_device(t) for t in tgt_np]
+    slots = [[i * B + b for b in range(B)] for i in range(n_sets)]
+    d_out, v_out = {}, {}
+
+    def step(i):
+        o = g.draft_step(slots[i % n_sets], hl, tl, top_n=1, want_logits=True, out=d_out)
+        g.verify(o["top_ids"].view(B, R), o["logits"], tgt[i % len(tgt)], T, 1, i, out=v_out)
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    l0 = g.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    launches = g.launch_count() - l0
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1))
+    assert g.poll() == 0, "device status word set during the timed region"
+    n_accept = float(v_out["n_out"].float().mean().item())
+
+    # ---- per-stage times (CUDA events recorded by the library between stages) -------------
+    g.profile(True)
+    n_prof = min(args.steps, 200)
+    for i in range(n_prof):
+        step(i)
+    torch.cuda.synchronize()
+    prof = g.profile_read()
+    g.profile(False)
+    sb = stage_bytes(s, B, lens)
+    peak, peak_kind = measured_peak()
+    stages = {}
+    for name, (tot, cnt) in prof.items():
+        if cnt and name in sb:
+            us = tot / cnt * 1e3
+            stages[name] = {"us": round(us, 2), "gbs": round(sb[name] / (us * 1e-6) / 1e9, 1)}
+    dom = max(stages, key=lambda k: stages[k]["us"]) if stages else None
+    step_bytes = sum(sb.values())
+    roofline = None
+    if dom:
+        roofline = {
+            "bound": "hbm", "kernel": dom, "achieved": stages[dom]["gbs"], "peak": peak,
+            "unit": "GB/s", "frac": round(stages[dom]["gbs"] / peak, 4), "traffic": None,
+            "peak_kind": f"of {peak_kind}", "bytes_per_launch": sb[dom],
+        }
+
+    # ---- end to end through the host-buffer entry point -----------------------------------
+    hl_h = torch.from_numpy(hl_np.view(np.int16) if hl_np.dtype == np.uint16 else hl_np).pin_memory()
+    tl_h = torch.from_numpy(tl_np).pin_memory()
+    tgt_h = [torch.from_numpy(t).pin_memory() for t in tgt_np]
+    r_out = {}
+    n_e2e = min(args.steps, 500)
+    for i in range(3):
+        g.round_host(slots[i % n_sets], hl_h, tl_h, tgt_h[i % len(tgt_h)], T, 1, i, out=r_out)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for i in range(n_e2e):
+        g.round_host(slots[i % n_sets], hl_h, tl_h, tgt_h[i % len(tgt_h)], T, 1, i, out=r_out)
+    torch.cuda.synchronize()
+    e2e_s = max_over_ranks(time.perf_counter() - t0)
+    eb = 4 if s.dtype == 0 else 2
+    e2e = {"value": aggregate_steps_per_s(world, n_e2e, e2e_s * 1e3), "unit": "steps/s",
+           "h2d_bytes_per_step": B * s.hidden * eb + B * 4 + B * R * V * 4,
+           "d2h_bytes_per_step": B * (R + 3) * 4, "steps": n_e2e}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(s, B, lens, hl_np, tl_np, tgt_np[0], T, args.cpu_seconds)
+
+    if rank == 0:
+        ms_per_step = ms / args.steps
+        value = aggregate_steps_per_s(world, args.steps, ms)
+        gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if s.dtype == 0 else "bf16", "data": "synthetic",
+            "config": dict(workload_config(s, B, lens),
+                           l2="weights exceed L2 and are streamed every step; KV caches rotate over "
+                              f"{n_sets} distinct sets, target logits over {len(tgt)} buffers",
+                           parallelism="replicas" if world > 1 else "single GPU"),
+            "drafted_tokens_per_s": value * B * R,
+            "step_bytes": step_bytes, "step_gbs": round(gbs, 1),
+            "hbm_frac_of_measured": round(gbs / peak, 4),
+            "hbm_frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
+            "mean_tokens_per_round": n_accept,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "stages": stages, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

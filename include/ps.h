@@ -191,6 +191,15 @@ ps_status ps_poll(ps_ctx* ctx, void* stream);
 /* Number of kernel launches the context has enqueued so far (host counter). */
 long long ps_launch_count(ps_ctx* ctx);
 
+/* Stage timing.  ps_profile(ctx, 1) makes every later call record a CUDA event after each
+ * stage it enqueues (a few microseconds of overhead per stage); ps_profile(ctx, 0) stops.
+ * ps_profile_read waits for the recorded events and returns, per stage name, the summed time
+ * and the number of intervals since profiling was switched on or last read.
+ *   names     host [max_stages][32] chars;  total_ms, count: host [max_stages];  n_stages: host */
+ps_status ps_profile(ps_ctx* ctx, int enable);
+ps_status ps_profile_read(ps_ctx* ctx, int max_stages, char* names, float* total_ms, int* count,
+                          int* n_stages);
+
 /* Text of the last error of this context (host string owned by the context). */
 const char* ps_last_error(ps_ctx* ctx);
 void ps_destroy(ps_ctx* ctx);

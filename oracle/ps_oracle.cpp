@@ -30,6 +30,9 @@
 #include <cstring>
 #include <limits>
 #include <vector>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 
 namespace {
 
@@ -234,6 +237,15 @@ int inverse_cdf(const std::vector<double>& w, double W, double u, double* margin
 }  // namespace
 
 extern "C" {
+
+// Threads the row loops use (for reporting next to timings).
+int pso_num_threads() {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
 
 void* pso_create(const Config* cfg, const Weights* w) {
   Ctx* C = new Ctx();

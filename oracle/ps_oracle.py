@@ -189,6 +189,11 @@ class Oracle:
         return out
 
 
+def num_threads() -> int:
+    """OpenMP threads the oracle's row loops run on."""
+    return _load().pso_num_threads()
+
+
 def row_stats(logits: np.ndarray, top_n: int):
     logits = np.ascontiguousarray(logits, dtype=np.float64)
     n, V = logits.shape

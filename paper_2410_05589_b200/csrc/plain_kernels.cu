@@ -346,6 +346,7 @@ ps_status fc_norm_kv(ps_ctx* c, const SeqMap& sm, int rows, int all_real, const 
   const ps_config& g = c->cfg;
   const ps_weights& w = c->w;
   int H = g.hidden, Hq = g.n_heads * g.head_dim, Hkv = g.n_kv_heads * g.head_dim;
+  prof_mark(c, st, "begin");
   k_gather<WT><<<rows, 256, 0, st>>>(sm, all_real, (const WT*)w.embed, (const WT*)w.mask_embed,
                                      (const WT*)w.mask_feat, (const WT*)hidden, tokens, H, g.vocab,
                                      c->x_in);
@@ -355,6 +356,7 @@ ps_status fc_norm_kv(ps_ctx* c, const SeqMap& sm, int rows, int all_real, const 
   if ((s = linear<WT>(c, c->x_in, 2 * H, w.w_fc, bias, nullptr, 0, c->x0, H, rows, H, 2 * H, st))) return s;
   k_rmsnorm<WT><<<rows, 256, 0, st>>>(c->x0, (const WT*)w.g_in, H, g.rms_eps, c->xn);
   c->launches++;
+  prof_mark(c, st, "fc_norm");
   if (with_q)
     if ((s = linear<WT>(c, c->xn, H, w.w_q, nullptr, nullptr, 0, c->q, Hq, rows, Hq, H, st))) return s;
   if ((s = linear<WT>(c, c->xn, H, w.w_k, nullptr, nullptr, 0, c->kv_tmp, 2 * Hkv, rows, Hkv, H, st))) return s;
@@ -363,6 +365,7 @@ ps_status fc_norm_kv(ps_ctx* c, const SeqMap& sm, int rows, int all_real, const 
       sm, with_q ? c->q : nullptr, c->kv_tmp, (WT*)c->kcache, (WT*)c->vcache, g.n_heads,
       g.n_kv_heads, g.head_dim, g.max_ctx, g.rope_base);
   c->launches++;
+  prof_mark(c, st, "qkv_rope");
   return cuda_check(c, cudaGetLastError(), "fc_norm_kv");
 }
 
@@ -385,7 +388,9 @@ ps_status draft_impl(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last
     k_attention<WT, 128><<<ag, 128, 0, st>>>(sm, c->q, (const WT*)c->kcache, (const WT*)c->vcache,
                                              g.n_heads, g.n_kv_heads, g.max_ctx, c->attn);
   c->launches++;
+  prof_mark(c, st, "attention");
   if ((s = linear<WT>(c, c->attn, Hq, w.w_o, nullptr, c->x0, H, c->a, H, M, H, Hq, st))) return s;
+  prof_mark(c, st, "o_proj");
   k_rmsnorm<WT><<<M, 256, 0, st>>>(c->a, (const WT*)w.g_post, H, g.rms_eps, c->an);
   c->launches++;
   if ((s = linear<WT>(c, c->an, H, w.w_gate, nullptr, nullptr, 0, c->gate, F, M, F, H, st))) return s;
@@ -395,6 +400,7 @@ ps_status draft_impl(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last
   c->launches++;
   float* hdn = feat_out ? feat_out : c->hdn;
   if ((s = linear<WT>(c, c->gate, F, w.w_down, nullptr, c->a, H, hdn, H, M, H, F, st))) return s;
+  prof_mark(c, st, "ffn");
   k_rmsnorm<WT><<<M, 256, 0, st>>>(hdn, (const WT*)w.g_final, H, g.rms_eps, c->hn);
   c->launches++;
   float* logits = logits_out ? logits_out : c->logits;
@@ -403,6 +409,7 @@ ps_status draft_impl(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last
     k_row_stats<<<M, 256, 0, st>>>(logits, V, top_n, top_ids, top_logit, row_max, row_lse);
     c->launches++;
   }
+  prof_mark(c, st, "lm_head");
   return cuda_check(c, cudaGetLastError(), "draft_step");
 }
 

@@ -18,6 +18,18 @@ ps_status cuda_check(ps_ctx* c, cudaError_t e, const char* what) {
   return PS_ERR_CUDA;
 }
 
+void prof_mark(ps_ctx* c, cudaStream_t st, const char* name) {
+  if (!c->prof) return;
+  if (c->prof_used == c->prof_ev.size()) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return;
+    c->prof_ev.push_back(e);
+    c->prof_name.push_back(name);
+  }
+  c->prof_name[c->prof_used] = name;
+  cudaEventRecord(c->prof_ev[c->prof_used++], st);
+}
+
 namespace {
 
 size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -150,7 +162,47 @@ ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* w, void*
   return PS_OK;
 }
 
-void ps_destroy(ps_ctx* c) { delete c; }
+void ps_destroy(ps_ctx* c) {
+  if (!c) return;
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+  delete c;
+}
+
+ps_status ps_profile(ps_ctx* c, int enable) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  c->prof = enable != 0;
+  c->prof_used = 0;
+  return PS_OK;
+}
+
+ps_status ps_profile_read(ps_ctx* c, int max_stages, char* names, float* total_ms, int* count,
+                          int* n_stages) {
+  if (!c || !names || !total_ms || !count || !n_stages || max_stages < 1) return PS_ERR_INVALID_ARG;
+  int n = 0;
+  for (size_t i = 1; i < c->prof_used; ++i) {
+    const char* nm = c->prof_name[i];
+    if (!std::strcmp(nm, "begin")) continue;   // an interval that ends at a "begin" mark is idle time
+    float ms = 0.f;
+    cudaError_t e = cudaEventSynchronize(c->prof_ev[i]);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, c->prof_ev[i - 1], c->prof_ev[i]);
+    if (e != cudaSuccess) return cuda_check(c, e, "ps_profile_read");
+    int j = 0;
+    while (j < n && std::strncmp(names + 32 * j, nm, 31)) ++j;
+    if (j == n) {
+      if (n == max_stages) continue;
+      std::strncpy(names + 32 * n, nm, 31);
+      names[32 * n + 31] = 0;
+      total_ms[n] = 0.f;
+      count[n] = 0;
+      ++n;
+    }
+    total_ms[j] += ms;
+    count[j] += 1;
+  }
+  *n_stages = n;
+  c->prof_used = 0;
+  return PS_OK;
+}
 
 const char* ps_last_error(ps_ctx* c) { return c ? c->err.c_str() : "null context"; }
 

@@ -67,12 +67,19 @@ struct ps_ctx {
   std::vector<int> len;     // committed positions per slot (host is the source of truth)
   long long launches;
   std::string err;
+  // optional stage timing (ps_profile): events recorded between stages
+  bool prof = false;
+  std::vector<cudaEvent_t> prof_ev;
+  std::vector<const char*> prof_name;   // name of the stage that ENDS at the event
+  size_t prof_used = 0;
 };
 
 namespace ps {
 
 ps_status fail(ps_ctx* c, ps_status s, const std::string& what);
 ps_status cuda_check(ps_ctx* c, cudaError_t e, const char* what);
+// Records a timing event that closes stage `name` (no-op unless profiling is on).
+void prof_mark(ps_ctx* c, cudaStream_t st, const char* name);
 
 // ---- unfused kernels with fp32 activations (all dtypes, all shapes) -----------------------
 ps_status plain_kv_append(ps_ctx* c, const SeqMap& sm, int rows, const void* hidden,

@@ -336,8 +336,10 @@ ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* 
     cudaError_t e = cudaFuncSetAttribute(k_verify, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_check(c, e, "verify smem");
   }
+  prof_mark(c, st, "begin");
   k_verify<<<dim3(n_target, B), kThreads, smem, st>>>(a);
   c->launches++;
+  prof_mark(c, st, "verify");
   return cuda_check(c, cudaGetLastError(), "k_verify");
 }
 

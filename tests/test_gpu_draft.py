@@ -1,0 +1,152 @@
+"""Parity of ps_draft_step / ps_kv_append with the CPU oracle (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from harness import Pair, as_f64, check_top, logits_close
+
+pytestmark = pytest.mark.gpu
+
+
+def _compare_step(p, top_n=4, seqs=None):
+    got = p.gpu_step(top_n=top_n)
+    s = p.s
+    worst = 0.0
+    for b in (p.oracle_seqs if seqs is None else seqs):
+        want = p.oracle_step(b)
+        e = logits_close(got["logits"][b], want["logits"], s.dtype)
+        worst = max(worst, e)
+        assert e <= 1.0, (b, e)
+        ef = logits_close(got["feat"][b], want["feat"], s.dtype)
+        assert ef <= 1.0, (b, "feat", ef)
+        for j in range(s.rows):
+            wl = want["logits"][j]
+            m = wl.max()
+            lse = m + np.log(np.exp(wl - m).sum())
+            tol = 1e-4 * max(abs(m), 1.0) if s.dtype == 0 else 1e-2 + 2e-2 * abs(m)
+            assert abs(got["row_max"][b, j] - m) <= tol
+            assert abs(got["row_lse"][b, j] - lse) <= tol + 2e-2 * (s.dtype == 1)
+            # statistics are those of the logits the kernel itself produced
+            gl = got["logits"][b, j].astype(np.float64)
+            assert abs(got["row_max"][b, j] - gl.max()) <= 1e-6 * max(1.0, abs(gl.max()))
+            assert abs(got["row_lse"][b, j] - (gl.max() + np.log(np.exp(gl - gl.max()).sum()))) <= 1e-4
+            check_top(got["top_ids"][b, j], got["top_logit"][b, j], wl, s.dtype)
+            # internal consistency: exact ranking of the kernel's own logits
+            order = np.lexsort((np.arange(s.vocab), -got["logits"][b, j]))[:top_n]
+            assert np.array_equal(got["top_ids"][b, j], order)
+    return worst
+
+
+def test_tiny_fp32_config():
+    p = Pair(synth.CONFIGS["tiny"], 1)
+    _compare_step(p)
+
+
+def test_tiny_fp32_with_bias_and_no_context():
+    p = Pair(synth.CONFIGS["tiny"], 1, with_bias=True, lens=[0])
+    _compare_step(p)
+
+
+def test_mini32_ragged_batch():
+    s = synth.CONFIGS["mini32"]
+    p = Pair(s, 3, lens=[5, 77, 0])
+    _compare_step(p, top_n=8)
+
+
+def test_mini_bf16_ragged_batch():
+    s = synth.CONFIGS["mini"]
+    p = Pair(s, s.batch)
+    _compare_step(p, top_n=8)
+
+
+def test_mini_bf16_more_masks_and_gqa():
+    s = synth.CONFIGS["mini"].with_(k_masks=8, n_kv_heads=2, batch=2, ctx_lo=130, ctx_hi=300)
+    p = Pair(s, 2)
+    _compare_step(p, top_n=1)
+
+
+def test_kv_append_matches_oracle_cache_and_is_incremental():
+    s = synth.CONFIGS["mini"]
+    p = Pair(s, 2, lens=[40, 9])
+    for b in range(2):
+        Ko, Vo = p.o.kv_export(b)
+        Kg, Vg = p.g.kv_export(b)
+        Kg, Vg = Kg.float().cpu().numpy(), Vg.float().cpu().numpy()
+        # bf16 cache: a one-ulp difference (2^-8 relative) is a rounding-boundary flip
+        assert np.abs(Kg - Ko).max() <= 2e-2 * np.abs(Ko).max()
+        assert (np.abs(Kg - Ko) <= 2.0 ** -7 * np.abs(Ko) + 1e-3).all()
+        assert (np.abs(Vg - Vo) <= 2.0 ** -7 * np.abs(Vo) + 1e-3).all()
+    # appending in two calls gives the same cache bits as one call
+    import paper_2410_05589_b200 as ps
+    g2 = ps.drafter_from_shape(s, p.W, max_batch=1, max_ctx=64)
+    h, t = synth.hidden_states(s, ("ctx", 0), 40), synth.token_ids(s, ("ctx", 0), 40)
+    g2.kv_append([0], [17], ps.to_device(h[:17]), ps.to_device(t[:17]))
+    g2.kv_append([0], [23], ps.to_device(h[17:]), ps.to_device(t[17:]))
+    K2, V2 = g2.kv_export(0)
+    K1, V1 = p.g.kv_export(0)
+    assert torch.equal(K1, K2) and torch.equal(V1, V2)
+    assert g2.kv_len(0) == 40
+
+
+def test_step_is_idempotent_and_prefix_invariant_in_batch():
+    s = synth.CONFIGS["mini"]
+    p = Pair(s, 3)
+    a = p.gpu_step()
+    b = p.gpu_step()
+    for k in ("logits", "feat", "top_ids", "row_lse"):
+        assert np.array_equal(a[k], b[k])
+    assert [p.g.kv_len(i) for i in range(3)] == [int(x) for x in p.lens]
+    # a sequence's result does not depend on its batch neighbours or its slot order
+    out = p.g.draft_step([2, 0], p.to_device(p.hidden_last[[2, 0]]), p.to_device(p.token_last[[2, 0]]),
+                         top_n=1)
+    torch.cuda.synchronize()
+    lg = out["logits"].cpu().numpy()
+    assert np.array_equal(lg[0], a["logits"][2]) and np.array_equal(lg[1], a["logits"][0])
+
+
+def test_argument_errors_return_status():
+    import paper_2410_05589_b200 as ps
+    s = synth.CONFIGS["mini32"]
+    p = Pair(s, 2, lens=[3, 4])
+    g = p.g
+    hl, tl = p.to_device(p.hidden_last), p.to_device(p.token_last)
+    with pytest.raises(ps.PsError) as e:
+        g.draft_step([0, 0], hl, tl)
+    assert e.value.status == -1
+    with pytest.raises(ps.PsError) as e:
+        g.draft_step([0, 5], hl, tl)
+    assert e.value.status == -1
+    with pytest.raises(ps.PsError) as e:
+        g.draft_step([0, 1], hl, tl, top_n=9)
+    assert e.value.status == -1
+    big = 200
+    with pytest.raises(ps.PsError) as e:
+        g.kv_append([0], [big], p.to_device(synth.hidden_states(s, "x", big)),
+                    p.to_device(synth.token_ids(s, "x", big)))
+    assert e.value.status == -3
+    assert g.kv_len(0) == 3
+    # the context is still usable
+    assert np.isfinite(p.gpu_step()["logits"]).all()
+    with pytest.raises(ps.PsError):
+        ps.Drafter(dtype=1, hidden=100, n_heads=2, n_kv_heads=2, head_dim=50, ffn=64, vocab=10,
+                   k_masks=1, max_batch=1, max_ctx=8, weights={})
+
+
+@pytest.mark.parametrize("name", ["7b", "13b"])
+def test_full_size_batch1(name):
+    """The 7B- and 13B-shaped batch-1 workloads at full size; context built by ps_kv_append on
+    the GPU and imported into the oracle (appends are checked above), oracle rows one by one."""
+    s = synth.CONFIGS[name]
+    p = Pair(s, 1, context="import")
+    _compare_step(p, top_n=1)
+    # the last 8 context rows again, this time produced by ps_kv_append at full size
+    L = int(p.lens[0])
+    h, t = synth.hidden_states(s, "tail", 8), synth.token_ids(s, "tail", 8)
+    p.g.kv_append([0], [8], p.to_device(h), p.to_device(t))
+    assert p.o.kv_append(0, h, t) == 0
+    Ko, Vo = p.o.kv_export(0)
+    Kg, Vg = p.g.kv_export(0)
+    Kg, Vg = Kg.float().cpu().numpy(), Vg.float().cpu().numpy()
+    assert (np.abs(Kg[L:] - Ko[L:]) <= 2.0 ** -7 * np.abs(Ko[L:]) + 1e-2).all()
+    assert (np.abs(Vg[L:] - Vo[L:]) <= 2.0 ** -7 * np.abs(Vo[L:]) + 1e-2).all()
