@@ -190,13 +190,15 @@ def cpu_baseline(s, B, lens, hidden_last, token_last, target, T, budget_s):
         n_seq, k_use = max(1, int(budget_s / (t_row * R))), s.k_masks
     else:
         n_seq, k_use = 1, max(0, int(budget_s / t_row) - 1)
-    t = 0.0
-    for b in range(n_seq):
-        t += oracle_time_step(o, s, b, k_use, hidden_last, token_last, target, T)
-    rows_done = n_seq * (k_use + 1)
+    t, reps = 0.0, 0
+    while reps == 0 or (t < 0.7 * budget_s and reps < 200):   # repeat short samples up to the budget
+        for b in range(n_seq):
+            t += oracle_time_step(o, s, b, k_use, hidden_last, token_last, target, T)
+        reps += 1
+    rows_done = reps * n_seq * (k_use + 1)
     est_step = t * (B * R) / rows_done
-    sample = (f"{n_seq} of {B} sequences x {k_use + 1} of {R} rows of one draft+verify step "
-              f"({t:.1f} s), scaled by rows to a full step")
+    sample = (f"{reps} x ({n_seq} of {B} sequences x {k_use + 1} of {R} rows of one draft+verify "
+              f"step), {t:.1f} s of CPU work, scaled by rows to a full step")
     return {"value": 1.0 / est_step, "unit": "steps/s", "cores": oracle.num_threads(),
             "kind": "oracle", "sample": sample}
 

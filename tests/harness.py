@@ -20,13 +20,14 @@ def as_f64(a, dtype):
 class Pair:
     """Oracle + CUDA drafter with identical weights and identical caches."""
 
-    def __init__(self, s, B, with_bias=False, context="append", lens=None, flags=0, oracle_seqs=None):
+    def __init__(self, s, B, with_bias=False, context="append", lens=None, flags=0, oracle_seqs=None,
+                 extra_ctx=0):
         import paper_2410_05589_b200 as ps
 
         self.s, self.B = s, B
         self.W = synth.weights(s, with_bias=with_bias)
         self.lens = synth.ctx_lengths(s, B) if lens is None else np.asarray(lens, np.int32)
-        max_ctx = int(self.lens.max()) + s.k_masks + 1
+        max_ctx = int(self.lens.max()) + s.k_masks + 1 + extra_ctx
         self.oracle_seqs = list(range(B)) if oracle_seqs is None else list(oracle_seqs)
         self.o = oracle_for(s, self.W, B, max_ctx)
         self.g = ps.drafter_from_shape(s, self.W, max_batch=B, max_ctx=max_ctx, flags=flags)

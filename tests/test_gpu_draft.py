@@ -138,7 +138,7 @@ def test_full_size_batch1(name):
     """The 7B- and 13B-shaped batch-1 workloads at full size; context built by ps_kv_append on
     the GPU and imported into the oracle (appends are checked above), oracle rows one by one."""
     s = synth.CONFIGS[name]
-    p = Pair(s, 1, context="import")
+    p = Pair(s, 1, context="import", extra_ctx=8)
     _compare_step(p, top_n=1)
     # the last 8 context rows again, this time produced by ps_kv_append at full size
     L = int(p.lens[0])
