@@ -50,6 +50,7 @@ enum {
   PS_FLAG_UNFUSED_KERNELS = 2   /* force the unfused fp32-activation kernels (debugging aid) */
 };
 enum { PS_MAX_BATCH = 128, PS_MAX_MASKS = 15, PS_MAX_TOP_N = 8 };
+enum { PS_STATIC_MAX_BATCH = 128, PS_STATIC_MAX_VOCAB = 262144 }; /* limits of ps_verify_static */
 
 typedef struct ps_config {
   int dtype;      /* PS_DTYPE_* */
@@ -209,6 +210,42 @@ void ps_destroy(ps_ctx* ctx);
  * check that the device stream equals the published generator word for word. */
 ps_status ps_philox_fill(const uint32_t key[2], const uint32_t* ctr, uint32_t* out, int n,
                          void* stream);
+
+/* ps_verify without a context and without any allocation.  (The paper has no counterpart:
+ * this entry point exists for the way the library is embedded, not for the method.)
+ *
+ * Who needs it: code that runs where device memory may no longer be requested -- an inference
+ * server that has handed its whole memory budget to a pool at start-up and forbids later
+ * cudaMalloc calls, a plugin inside someone else's allocator-controlled process, a region
+ * where an allocation would synchronise the device and stall other streams.  Such callers
+ * cannot create a ps_ctx (it needs a workspace) just to run the acceptance test.
+ *
+ * What it does: exactly what ps_verify does, with the same arguments plus the vocabulary size,
+ * but the kernel's scratch (per-sequence arrival counters and per-position records, about
+ * 18 KB) lives in a fixed array inside the library's device image.  Every GPU that loads the
+ * library holds that array until the process exits.  The call itself performs no cudaMalloc,
+ * cudaFree or other allocating routine; inputs and outputs are still the caller's.
+ *
+ * Limits (PS_ERR_CAPACITY with a message in `err` beyond them): B <= PS_STATIC_MAX_BATCH,
+ * n_draft <= PS_MAX_MASKS+1, vocab <= PS_STATIC_MAX_VOCAB.
+ *
+ * Sharing: there is ONE array per GPU and every call uses it.  It keeps the previous call's
+ * contents; the counters that must start at zero are cleared on `stream` before the kernel.
+ * Two calls whose kernels may overlap on the same GPU (different streams, different threads)
+ * race on it and give wrong results: serialise them.
+ *
+ * First call on a device: looks up the array's device address once (with that device current)
+ * and caches it.  Make that first call outside any stream capture.
+ *
+ *   nonfinite_flag  device [1] int or NULL: bit 0 is OR-ed in when a NaN/+inf logit was met in
+ *                   an examined row (the caller zeroes it beforehand)
+ *   err             host buffer for an error text, or NULL;  err_cap its size in bytes
+ * All other arguments as in ps_verify. */
+ps_status ps_verify_static(int vocab, int B, int n_draft, int n_target, const int* draft_tokens,
+                           const float* draft_logits, const float* target_logits,
+                           float temperature, uint64_t seed, uint64_t offset, int* accept_len,
+                           int* out_tokens, int* n_out, int* nonfinite_flag, char* err,
+                           size_t err_cap, void* stream);
 
 #ifdef __cplusplus
 }

@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     PsError,
     load_library,
     philox_fill,
+    verify_static,
 )
 from .build import build  # noqa: F401
 from .synth_bridge import drafter_from_shape, to_device  # noqa: F401

@@ -29,6 +29,7 @@ EXPORTS = (
     "ps_workspace_bytes", "ps_init", "ps_kv_append", "ps_draft_step", "ps_verify", "ps_round_host",
     "ps_kv_len", "ps_kv_reset", "ps_kv_export", "ps_kv_import", "ps_poll", "ps_launch_count",
     "ps_last_error", "ps_destroy", "ps_philox_fill", "ps_profile", "ps_profile_read",
+    "ps_verify_static",
 )
 
 
@@ -87,6 +88,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.ps_philox_fill.argtypes = [C.POINTER(C.c_uint32), vp, vp, C.c_int, vp]
     lib.ps_profile.argtypes = [vp, C.c_int]
     lib.ps_profile_read.argtypes = [vp, C.c_int, C.c_char_p, C.POINTER(C.c_float), ip, ip]
+    lib.ps_verify_static.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, C.c_float,
+                                     C.c_uint64, C.c_uint64, vp, vp, vp, vp, C.c_char_p, C.c_size_t, vp]
     _lib = lib
     return lib
 
@@ -119,6 +122,29 @@ def philox_fill(key, ctr: torch.Tensor) -> torch.Tensor:
     rc = lib.ps_philox_fill(k, _dptr(ctr), _dptr(out), ctr.shape[0], _stream())
     if rc != PS_OK:
         raise PsError(rc)
+    return out
+
+
+def verify_static(draft_tokens: torch.Tensor, draft_logits, target_logits: torch.Tensor,
+                  temperature: float, seed: int, offset: int, out: dict, nonfinite_flag=None,
+                  stream=None) -> dict:
+    """ps_verify_static: the acceptance test for callers that may not allocate device memory.
+
+    Needs no Drafter and no workspace; the kernel's scratch is a fixed array inside the library
+    (one per GPU, shared by all calls, so calls must not overlap on a GPU).  ``out`` must hold the
+    caller's preallocated CUDA int32 tensors ``accept_len`` [B], ``out_tokens`` [B][n_draft+1] and
+    ``n_out`` [B]: this wrapper allocates nothing either.
+    """
+    lib = load_library()
+    B, n_draft = draft_tokens.shape
+    _, n_target, vocab = target_logits.shape
+    err = C.create_string_buffer(256)
+    rc = lib.ps_verify_static(vocab, B, n_draft, n_target, _dptr(draft_tokens), _dptr(draft_logits),
+                              _dptr(target_logits), float(temperature), seed, offset,
+                              _dptr(out["accept_len"]), _dptr(out["out_tokens"]), _dptr(out["n_out"]),
+                              _dptr(nonfinite_flag), err, 256, _stream(stream))
+    if rc != PS_OK:
+        raise PsError(rc, err.value.decode())
     return out
 
 

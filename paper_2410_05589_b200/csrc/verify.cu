@@ -6,6 +6,8 @@
 // to finish walks the positions in order and writes accept_len / out_tokens / n_out.
 // Nothing spins: blocks only take a ticket, the last arriver does the merge.
 #include <cfloat>
+#include <cstdio>
+#include <mutex>
 
 #include "ps_internal.cuh"
 
@@ -351,4 +353,97 @@ extern "C" ps_status ps_philox_fill(const uint32_t key[2], const uint32_t* ctr, 
   if (n == 0) return PS_OK;
   ps::k_philox_fill<<<(n + 255) / 256, 256, 0, (cudaStream_t)stream>>>(key[0], key[1], ctr, out, n);
   return cudaGetLastError() == cudaSuccess ? PS_OK : PS_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------
+// ps_verify_static: the same kernel with its scratch in a fixed device array of this library
+// instead of a caller-allocated workspace, for callers that must not allocate.
+namespace ps {
+namespace {
+
+struct StaticScratch {
+  unsigned tickets[PS_STATIC_MAX_BATCH];                       // must be zero when a call starts
+  VerifyRec rec[PS_STATIC_MAX_BATCH * (PS_MAX_MASKS + 2)];     // fully rewritten by every call
+  int status_sink;                                             // takes the flag when the caller passes none
+};
+
+// About 18 KB, held by every GPU that loads the library until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the array on the CURRENT device, looked up once per device.  The array's
+// name is only a host-side handle here; a kernel must be given the address obtained below.
+cudaError_t static_scratch_address(StaticScratch** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_ptr[dev] = p;
+  }
+  *out = (StaticScratch*)g_static_ptr[dev];
+  return cudaSuccess;
+}
+
+ps_status static_fail(char* err, size_t cap, ps_status s, const char* text) {
+  if (err && cap) std::snprintf(err, cap, "%s", text);
+  return s;
+}
+
+}  // namespace
+}  // namespace ps
+
+extern "C" ps_status ps_verify_static(int vocab, int B, int n_draft, int n_target,
+                                      const int* draft_tokens, const float* draft_logits,
+                                      const float* target_logits, float temperature, uint64_t seed,
+                                      uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
+                                      int* nonfinite_flag, char* err, size_t err_cap, void* stream) {
+  using namespace ps;
+  if (err && err_cap) err[0] = 0;
+  if (!draft_tokens || !target_logits || !accept_len || !out_tokens || !n_out)
+    return static_fail(err, err_cap, PS_ERR_INVALID_ARG, "ps_verify_static: null pointer");
+  if (B < 1 || n_draft < 1 || vocab < 1)
+    return static_fail(err, err_cap, PS_ERR_INVALID_ARG, "ps_verify_static: sizes must be positive");
+  if (B > PS_STATIC_MAX_BATCH)
+    return static_fail(err, err_cap, PS_ERR_CAPACITY,
+                       "ps_verify_static: B exceeds PS_STATIC_MAX_BATCH (the fixed scratch holds 128 sequences)");
+  if (n_draft > PS_MAX_MASKS + 1)
+    return static_fail(err, err_cap, PS_ERR_CAPACITY,
+                       "ps_verify_static: n_draft exceeds PS_MAX_MASKS+1 (16 positions per sequence)");
+  if (vocab > PS_STATIC_MAX_VOCAB)
+    return static_fail(err, err_cap, PS_ERR_CAPACITY,
+                       "ps_verify_static: vocab exceeds PS_STATIC_MAX_VOCAB (262144)");
+  if (n_target != n_draft && n_target != n_draft + 1)
+    return static_fail(err, err_cap, PS_ERR_INVALID_ARG,
+                       "ps_verify_static: n_target must be n_draft or n_draft+1");
+  if (!(temperature >= 0.f))
+    return static_fail(err, err_cap, PS_ERR_INVALID_ARG, "ps_verify_static: temperature must be >= 0");
+  StaticScratch* sc = nullptr;
+  cudaError_t e = static_scratch_address(&sc);
+  if (e != cudaSuccess) return static_fail(err, err_cap, PS_ERR_CUDA, cudaGetErrorString(e));
+  cudaStream_t st = (cudaStream_t)stream;
+  // The arrival counters keep whatever the previous call left; they must start at zero.
+  e = cudaMemsetAsync(sc->tickets, 0, sizeof(sc->tickets), st);
+  if (e != cudaSuccess) return static_fail(err, err_cap, PS_ERR_CUDA, cudaGetErrorString(e));
+  VerifyArgs a;
+  a.B = B; a.n_draft = n_draft; a.n_target = n_target; a.V = vocab;
+  a.draft_tokens = draft_tokens; a.draft_logits = draft_logits; a.target_logits = target_logits;
+  a.temperature = temperature;
+  a.key0 = (uint32_t)seed; a.key1 = (uint32_t)(seed >> 32);
+  a.off_lo = (uint32_t)offset; a.off_hi = (uint32_t)(offset >> 32);
+  a.accept_len = accept_len; a.out_tokens = out_tokens; a.n_out = n_out;
+  a.rec = sc->rec; a.tickets = sc->tickets;
+  a.status = nonfinite_flag ? nonfinite_flag : &sc->status_sink;
+  size_t smem = (size_t)((vocab + kSeg - 1) / kSeg) * sizeof(double);   // <= 16 KB at the vocab limit
+  k_verify<<<dim3(n_target, B), kThreads, smem, st>>>(a);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return static_fail(err, err_cap, PS_ERR_CUDA, cudaGetErrorString(e));
+  return PS_OK;
 }
