@@ -189,6 +189,12 @@ ps_status ps_kv_import(ps_ctx* ctx, int slot, int len, const void* K, const void
  * PS_ERR_NONFINITE or PS_ERR_TIMEOUT. */
 ps_status ps_poll(ps_ctx* ctx, void* stream);
 
+/* Test helper: device address and size of one of the context's intermediate buffers after a
+ * draft step: "x0" (fc output, float [M][H]), "a" (attention block output, float [M][H]),
+ * "qkv" (float [M][Hq+2Hkv], before RoPE), "act" (float [M][F], silu(gate)*up).  The last two
+ * exist only on the fused bf16 path.  PS_ERR_INVALID_ARG for an unknown name. */
+ps_status ps_debug_buffer(ps_ctx* ctx, const char* name, void** ptr, size_t* bytes);
+
 /* Number of kernel launches the context has enqueued so far (host counter). */
 long long ps_launch_count(ps_ctx* ctx);
 

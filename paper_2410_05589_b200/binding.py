@@ -29,7 +29,7 @@ EXPORTS = (
     "ps_workspace_bytes", "ps_init", "ps_kv_append", "ps_draft_step", "ps_verify", "ps_round_host",
     "ps_kv_len", "ps_kv_reset", "ps_kv_export", "ps_kv_import", "ps_poll", "ps_launch_count",
     "ps_last_error", "ps_destroy", "ps_philox_fill", "ps_profile", "ps_profile_read",
-    "ps_verify_static",
+    "ps_verify_static", "ps_debug_buffer",
 )
 
 
@@ -88,6 +88,7 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.ps_philox_fill.argtypes = [C.POINTER(C.c_uint32), vp, vp, C.c_int, vp]
     lib.ps_profile.argtypes = [vp, C.c_int]
     lib.ps_profile_read.argtypes = [vp, C.c_int, C.c_char_p, C.POINTER(C.c_float), ip, ip]
+    lib.ps_debug_buffer.argtypes = [vp, C.c_char_p, C.POINTER(vp), C.POINTER(C.c_size_t)]
     lib.ps_verify_static.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, C.c_float,
                                      C.c_uint64, C.c_uint64, vp, vp, vp, vp, C.c_char_p, C.c_size_t, vp]
     _lib = lib
@@ -300,6 +301,19 @@ class Drafter:
         self._check(self.lib.ps_profile_read(self.h, n_max, names, ms, cnt, C.byref(n)))
         raw = names.raw
         return {raw[32 * i:32 * i + 32].split(b"\0")[0].decode(): (ms[i], cnt[i]) for i in range(n.value)}
+
+    def debug_buffer(self, name: str, dtype, shape) -> torch.Tensor:
+        """Copy of an intermediate buffer of the last draft step (test helper)."""
+        ptr, nbytes = C.c_void_p(), C.c_size_t()
+        self._check(self.lib.ps_debug_buffer(self.h, name.encode(), C.byref(ptr), C.byref(nbytes)))
+        base = self.workspace.data_ptr()
+        off = ptr.value - base
+        n = 1
+        for d in shape:
+            n *= d
+        elt = torch.empty((), dtype=dtype).element_size()
+        assert 0 <= off and n * elt <= nbytes.value and off + n * elt <= self.workspace.numel()
+        return self.workspace[off:off + n * elt].view(dtype).view(*shape).clone()
 
     def launch_count(self) -> int:
         return self.lib.ps_launch_count(self.h)

@@ -83,6 +83,7 @@ size_t carve(const ps_config& g, ps_ctx* c, char* base) {
   void* hdn = take(Md * H * 4);
   void* hn = take(Md * H * 4);
   void* logits = take(Md * V * 4);
+  void* fused = take(fused_scratch_bytes(g));
   void* st_hidden = take((size_t)g.max_batch * H * elem_bytes(g));
   void* st_tok = take((size_t)g.max_batch * 4);
   void* st_tlogits = take(Md * V * 4);
@@ -96,6 +97,7 @@ size_t carve(const ps_config& g, ps_ctx* c, char* base) {
     c->kv_tmp = (float*)kv_tmp; c->attn = (float*)attn; c->a = (float*)a; c->an = (float*)an;
     c->gate = (float*)gate; c->up = (float*)up; c->hdn = (float*)hdn; c->hn = (float*)hn;
     c->logits = (float*)logits;
+    c->fused_scratch = fused;
     c->st_hidden = st_hidden; c->st_tok = (int*)st_tok; c->st_tlogits = (float*)st_tlogits;
     c->st_dlogits = (float*)st_dlogits; c->st_top = (int*)st_top; c->st_res = (int*)st_res;
     c->max_rows = (int)Md;
@@ -152,7 +154,16 @@ ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* w, void*
   c->len.assign(cfg->max_batch, 0);
   carve(*cfg, c, c->ws);
   cudaStream_t st = (cudaStream_t)stream;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    delete c;
+    return PS_ERR_CUDA;
+  }
+  c->n_sm = std::min(prop.multiProcessorCount, kMaxSm);
+  c->smem_optin = (int)prop.sharedMemPerBlockOptin;
   cudaError_t e = cudaMemsetAsync(c->dev_status, 0, 256, st);
+  if (e == cudaSuccess)
+    e = cudaMemsetAsync(c->fused_scratch, 0, fused_scratch_bytes(*cfg), st);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * PS_MAX_BATCH, st);
   if (e != cudaSuccess) {
     delete c;
@@ -207,6 +218,15 @@ ps_status ps_profile_read(ps_ctx* c, int max_stages, char* names, float* total_m
 const char* ps_last_error(ps_ctx* c) { return c ? c->err.c_str() : "null context"; }
 
 long long ps_launch_count(ps_ctx* c) { return c ? c->launches : 0; }
+
+ps_status ps_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* bytes) {
+  if (!c || !name || !ptr || !bytes) return PS_ERR_INVALID_ARG;
+  const ps_config& g = c->cfg;
+  const size_t Md = (size_t)g.max_batch * (g.k_masks + 1);
+  if (!std::strcmp(name, "x0")) { *ptr = c->x0; *bytes = Md * g.hidden * 4; return PS_OK; }
+  if (!std::strcmp(name, "a")) { *ptr = c->a; *bytes = Md * g.hidden * 4; return PS_OK; }
+  return fused_debug_buffer(c, name, ptr, bytes);
+}
 
 ps_status ps_kv_len(ps_ctx* c, int slot, int* len) {
   if (!c || !len || slot < 0 || slot >= c->cfg.max_batch) return PS_ERR_INVALID_ARG;
@@ -304,6 +324,9 @@ ps_status ps_draft_step(ps_ctx* c, int B, const int* seq_slot, const void* hidde
     if (sm.len[b] + R > c->cfg.max_ctx) return fail(c, PS_ERR_CAPACITY, "no room for the draft rows");
   }
   sm.row_off[B] = B * R;
+  if (fused_supported(c, B * R))
+    return fused_draft_step(c, sm, B, hidden_last, token_last, top_n, top_ids, top_logit, row_max,
+                            row_lse, logits_out, feat_out, (cudaStream_t)stream);
   return plain_draft_step(c, sm, B, hidden_last, token_last, top_n, top_ids, top_logit, row_max,
                           row_lse, logits_out, feat_out, (cudaStream_t)stream);
 }

@@ -3,7 +3,9 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
+#include <cstring>
 #include <string>
 #include <vector>
 
@@ -13,6 +15,8 @@ namespace ps {
 
 constexpr int kMaxRowsPerSeq = PS_MAX_MASKS + 1;  // rows of one sequence in a draft step
 constexpr int kAppendChunk = 256;                 // rows handled per pass of ps_kv_append
+constexpr int kAttnMaxSplit = 16;                 // key-range splits of the fused attention
+constexpr int kMaxSm = 192;                       // bound used to size per-CTA scratch
 
 // Which sequence each row of a launch belongs to.  Passed by value as a kernel parameter.
 // Row m (0-based within the launch) belongs to the sequence b with
@@ -63,6 +67,9 @@ struct ps_ctx {
   ps::VerifyRec* vrec;      // [max_batch][PS_MAX_MASKS+2]
   float *x_in, *x0, *xn, *q, *kv_tmp, *attn, *a, *an, *gate, *up, *hdn, *hn, *logits;
   // staging for ps_round_host
+  void* fused_scratch;      // buffers of the fused bf16 path (see fused_kernels.cu)
+  int n_sm;                 // multiprocessors of the context's device
+  int smem_optin;           // opt-in shared memory per block
   void* st_hidden; int* st_tok; float* st_tlogits; float* st_dlogits; int* st_top; int* st_res;
   std::vector<int> len;     // committed positions per slot (host is the source of truth)
   long long launches;
@@ -85,6 +92,16 @@ void prof_mark(ps_ctx* c, cudaStream_t st, const char* name);
 ps_status plain_kv_append(ps_ctx* c, const SeqMap& sm, int rows, const void* hidden,
                           const int* tokens, cudaStream_t st);
 ps_status plain_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last,
+                           const int* token_last, int top_n, int* top_ids, float* top_logit,
+                           float* row_max, float* row_lse, float* logits_out, float* feat_out,
+                           cudaStream_t st);
+// ---- fused bf16 kernels for small M ---------------------------------------------------------
+bool fused_supported(const ps_ctx* c, int M);
+size_t fused_scratch_bytes(const ps_config& g);
+ps_status fused_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* bytes);
+ps_status launch_attn_split(ps_ctx* c, const SeqMap& sm, int B, const float* qkv, float* att_ml,
+                            float* att_o, int* n_split_out, cudaStream_t st);
+ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last,
                            const int* token_last, int top_n, int* top_ids, float* top_logit,
                            float* row_max, float* row_lse, float* logits_out, float* feat_out,
                            cudaStream_t st);
