@@ -34,11 +34,12 @@ struct LmPart {  // softmax / top-n summary of one CTA's vocabulary range for on
 struct GemmArgs {
   RowSrc rs;
   int N, K, M;
-  int pass_cols;   // k columns per pass (multiple of KC), chosen by the host
+  int pass_cols;   // k columns per pass (multiple of 64), chosen by the host
   int rows_cap;    // capacity (features per CTA, x2 when zipped) of the CTA accumulator
   // ---- prologue inputs
   const float* x_f32;  int ldx;        // PRO_NORM / PRO_F32: [M][ldx]
   const __nv_bfloat16* gain; float eps;
+  const float* ssq_in; int ssq_n;      // PRO_NORM: [ssq_n][M] partial sums of squares of x_f32 rows
   const __nv_bfloat16 *embed, *mask_embed, *mask_feat, *hidden;   // PRO_GATHER
   const int* tokens; int H, V, R;
   // PRO_ATTN: partial attention results [M][n_heads][n_split] (m, l) and [..][D] o
@@ -47,6 +48,7 @@ struct GemmArgs {
   float* out; int ldo;                 // EPI_STORE / EPI_SWIGLU: [M][ldo]
   const __nv_bfloat16* bias;
   const float* res; int ldr;
+  float* ssq_out;                      // EPI_STORE: [gridDim.x][M] partial sums of squares, or nullptr
   // EPI_LMHEAD
   float* logits_out;                   // [M][N] or nullptr
   LmPart* parts;                       // [gridDim.x][M]
@@ -61,70 +63,99 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// ---- prologues: the activation operand, columns [k0, k1), as hi/lo bf16 planes in shared memory
+// ---- prologues: the activation operand, columns [k0, k1), as fp32 planes in shared memory
+// One 8-column vector of row m starting at column k.
 template <int PRO>
-__device__ void load_acts(const GemmArgs& a, unsigned char* a_hi, unsigned char* a_lo, int apitch,
-                          const float* row_scale, int k0, int k1, int tid) {
-  const int M = a.M, vecs = (k1 - k0) / 8;
-  for (int idx = tid; idx < M * vecs; idx += kConsumerThreads) {
-    const int m = idx / vecs, v = idx - m * vecs;
-    const int k = k0 + v * 8;
-    const size_t off = (size_t)m * apitch + (size_t)v * 16;
-    if (PRO == PRO_GATHER) {
-      // row m = (b, j): j == 0 -> [embed[token_b] ; hidden_b], j >= 1 -> [mask_embed ; mask_feat][j-1]
-      const int H = a.H, b = m / a.R, j = m - b * a.R;
-      const int half = k >= H ? 1 : 0, kk = k - half * H;
-      const __nv_bfloat16* src;
-      if (j == 0) {
-        int tok = min(max(a.tokens[b], 0), a.V - 1);
-        src = half == 0 ? a.embed + (size_t)tok * H : a.hidden + (size_t)b * H;
-      } else {
-        src = (half == 0 ? a.mask_embed : a.mask_feat) + (size_t)(j - 1) * H;
-      }
-      *reinterpret_cast<uint4*>(a_hi + off) = *reinterpret_cast<const uint4*>(src + kk);
-      *reinterpret_cast<uint4*>(a_lo + off) = make_uint4(0, 0, 0, 0);   // inputs are exact bf16
-    } else if (PRO == PRO_NORM || PRO == PRO_F32) {
-      const float4* xp = reinterpret_cast<const float4*>(a.x_f32 + (size_t)m * a.ldx + k);
-      float4 x0 = xp[0], x1 = xp[1];
-      float x[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-      if (PRO == PRO_NORM) {
-        uint4 gq = *reinterpret_cast<const uint4*>(a.gain + k);
-        const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&gq);
-        const float s = row_scale[m];
+__device__ __forceinline__ void fetch8(const GemmArgs& a, int m, int k, float (&x)[8], uint4& raw) {
+  if (PRO == PRO_GATHER) {
+    // row m = (b, j): j == 0 -> [embed[token_b] ; hidden_b], j >= 1 -> [mask_embed ; mask_feat][j-1]
+    const int H = a.H, b = m / a.R, j = m - b * a.R;
+    const int half = k >= H ? 1 : 0, kk = k - half * H;
+    const __nv_bfloat16* src;
+    if (j == 0) {
+      int tok = min(max(a.tokens[b], 0), a.V - 1);
+      src = half == 0 ? a.embed + (size_t)tok * H : a.hidden + (size_t)b * H;
+    } else {
+      src = (half == 0 ? a.mask_embed : a.mask_feat) + (size_t)(j - 1) * H;
+    }
+    raw = *reinterpret_cast<const uint4*>(src + kk);
+  } else if (PRO == PRO_NORM || PRO == PRO_F32) {
+    const float4* xp = reinterpret_cast<const float4*>(a.x_f32 + (size_t)m * a.ldx + k);
+    float4 x0 = xp[0], x1 = xp[1];
+    x[0] = x0.x; x[1] = x0.y; x[2] = x0.z; x[3] = x0.w;
+    x[4] = x1.x; x[5] = x1.y; x[6] = x1.z; x[7] = x1.w;
+    if (PRO == PRO_NORM) raw = *reinterpret_cast<const uint4*>(a.gain + k);
+  } else {  // PRO_ATTN: merge the key splits of (row m, head h): o = sum_s w_s o_s / sum_s w_s l_s
+    const int D = a.D, S = a.n_split, nh = a.n_heads;
+    const int h = k / D, d0 = k - h * D;
+    const float* ml = a.att_ml + ((size_t)m * nh + h) * S * 2;
+    float mx = -FLT_MAX;
+    for (int s = 0; s < S; ++s) mx = fmaxf(mx, ml[2 * s]);
+    float den = 0.f;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          float2 gf = __bfloat1622float2(gp[i]);
-          x[2 * i] = x[2 * i] * s * gf.x;
-          x[2 * i + 1] = x[2 * i + 1] * s * gf.y;
+    for (int i = 0; i < 8; ++i) x[i] = 0.f;
+    for (int s = 0; s < S; ++s) {
+      float w = __expf(ml[2 * s] - mx);
+      den += w * ml[2 * s + 1];
+      const float4* op = reinterpret_cast<const float4*>(a.att_o + (((size_t)m * nh + h) * S + s) * D + d0);
+      float4 o0 = op[0], o1 = op[1];
+      x[0] += w * o0.x; x[1] += w * o0.y; x[2] += w * o0.z; x[3] += w * o0.w;
+      x[4] += w * o1.x; x[5] += w * o1.y; x[6] += w * o1.z; x[7] += w * o1.w;
+    }
+    const float inv = 1.f / den;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] *= inv;
+  }
+}
+
+template <int PRO>
+__device__ void load_acts(const GemmArgs& a, float* plane_a, float* plane_b, int ppitch,
+                          const float* row_scale, int k0, int k1, int tid) {
+  constexpr int U = 4;   // vectors in flight per thread: all loads are issued before any store
+  const int M = a.M, vecs = (k1 - k0) / 8, total = M * vecs;
+  for (int base = tid; base < total; base += U * kConsumerThreads) {
+    float x[U][8];
+    uint4 raw[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int idx = base + u * kConsumerThreads;
+      if (idx < total) {
+        const int m = idx / vecs, v = idx - m * vecs;
+        fetch8<PRO>(a, m, k0 + v * 8, x[u], raw[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int idx = base + u * kConsumerThreads;
+      if (idx < total) {
+        const int m = idx / vecs, v = idx - m * vecs;
+        const size_t off = (size_t)m * ppitch + (size_t)v * 4;
+        if (PRO == PRO_GATHER) {
+          const float2 p0 = widen2(raw[u].x), p1 = widen2(raw[u].y), p2 = widen2(raw[u].z),
+                       p3 = widen2(raw[u].w);
+          *reinterpret_cast<float4*>(plane_a + off) = make_float4(p0.x, p0.y, p1.x, p1.y);
+          *reinterpret_cast<float4*>(plane_b + off) = make_float4(p2.x, p2.y, p3.x, p3.y);
+        } else {
+          if (PRO == PRO_NORM) {
+            const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&raw[u]);
+            const float s = row_scale[m];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              float2 gf = __bfloat1622float2(gp[i]);
+              x[u][2 * i] = x[u][2 * i] * s * gf.x;
+              x[u][2 * i + 1] = x[u][2 * i + 1] * s * gf.y;
+            }
+          }
+          *reinterpret_cast<float4*>(plane_a + off) = make_float4(x[u][0], x[u][1], x[u][2], x[u][3]);
+          *reinterpret_cast<float4*>(plane_b + off) = make_float4(x[u][4], x[u][5], x[u][6], x[u][7]);
         }
       }
-      store_split8(a_hi, a_lo, off, x);
-    } else {  // PRO_ATTN: merge the key splits of (row m, head h): o = sum_s w_s o_s / sum_s w_s l_s
-      const int D = a.D, S = a.n_split, nh = a.n_heads;
-      const int h = k / D, d0 = k - h * D;
-      const float* ml = a.att_ml + ((size_t)m * nh + h) * S * 2;
-      float mx = -FLT_MAX;
-      for (int s = 0; s < S; ++s) mx = fmaxf(mx, ml[2 * s]);
-      float den = 0.f;
-      float x[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      for (int s = 0; s < S; ++s) {
-        float w = __expf(ml[2 * s] - mx);
-        den += w * ml[2 * s + 1];
-        const float4* op = reinterpret_cast<const float4*>(a.att_o + (((size_t)m * nh + h) * S + s) * D + d0);
-        float4 o0 = op[0], o1 = op[1];
-        x[0] += w * o0.x; x[1] += w * o0.y; x[2] += w * o0.z; x[3] += w * o0.w;
-        x[4] += w * o1.x; x[5] += w * o1.y; x[6] += w * o1.z; x[7] += w * o1.w;
-      }
-      const float inv = 1.f / den;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) x[i] *= inv;
-      store_split8(a_hi, a_lo, off, x);
     }
   }
 }
 
-// Shared-memory layout (dynamic): [Smem][red: 2 x 8 warps x 16 slot rows x 16 m floats]
-// [row scales][CTA accumulator: 16 m x rows_cap floats][act hi plane][act lo plane][ring]
+// Shared-memory layout (dynamic): [Smem][red: 2 x 8 warps x 8 slot rows x 16 m floats]
+// [row scales][CTA accumulator: 16 m x rows_cap floats][act plane a][act plane b][ring]
 constexpr int kRedFloats = kConsumerWarps * kSlotRows * kMaxM;   // one buffer
 
 struct Layout {
@@ -137,7 +168,7 @@ __host__ __device__ inline Layout make_layout(int M, int pass_cols, int rows_cap
   L.off_red = off; off += 2 * kRedFloats * 4;
   L.off_scale = off; off += 128;
   L.off_out = off; off += ((rows_cap * kMaxM * 4) + 127) & ~127;
-  const int plane = ((M * act_pitch(pass_cols)) + 127) & ~127;
+  const int plane = ((M * plane_pitch(pass_cols) * 4) + 127) & ~127;
   L.off_hi = off; off += plane;
   L.off_lo = off; off += plane;
   L.off_ring = off;
@@ -148,17 +179,17 @@ __host__ __device__ inline Layout make_layout(int M, int pass_cols, int rows_cap
 }
 
 // Smallest number of k passes whose activation planes leave room for kMinSlots ring slots.
-// Returns the columns per pass (multiple of KC) or 0 if even one chunk does not fit.
+// Returns the columns per pass (multiple of 64) or 0 if nothing fits.
 int choose_pass_cols(int M, int K, int rows_cap, int smem_limit) {
-  for (int n_pass = 1; n_pass <= (K + KC - 1) / KC; ++n_pass) {
-    int cols = ((K + n_pass - 1) / n_pass + KC - 1) / KC * KC;
+  for (int n_pass = 1; n_pass <= (K + 63) / 64; ++n_pass) {
+    int cols = ((K + n_pass - 1) / n_pass + 63) / 64 * 64;
     if (make_layout(M, std::min(cols, (K + 7) / 8 * 8), rows_cap, smem_limit).n_slots >= kMinSlots)
       return cols;
   }
   return 0;
 }
 
-template <int PRO, int EPI, bool UPPER>
+template <int PRO, int EPI, int MT>
 __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_limit) {
   extern __shared__ __align__(128) unsigned char smem[];
   Smem& sm = *reinterpret_cast<Smem*>(smem);
@@ -167,10 +198,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
   float* red = reinterpret_cast<float*>(smem + L.off_red);
   float* row_scale = reinterpret_cast<float*>(smem + L.off_scale);
   float* cta_out = reinterpret_cast<float*>(smem + L.off_out);   // [m][rows_cap]
-  unsigned char* a_hi = smem + L.off_hi;
-  unsigned char* a_lo = smem + L.off_lo;
+  float* plane_a = reinterpret_cast<float*>(smem + L.off_hi);
+  float* plane_b = reinterpret_cast<float*>(smem + L.off_lo);
   unsigned char* ring = smem + L.off_ring;
-  const int apitch = act_pitch(min(pass_cols, a.K));
+  const int ppitch = plane_pitch(min(pass_cols, a.K));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rows_cap = a.rows_cap, rows_half = rows_cap >> 1;
 
@@ -187,20 +218,18 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
 
   int n_begin, n_end;
   cta_range(a.N, blockIdx.x, gridDim.x, n_begin, n_end);
-  const int feat_per_tile = a.rs.zip ? 8 : 16;
   const int cnt = n_end - n_begin;
+  const int n_st = n_subtiles(a.rs, n_begin, n_end);
 
   if (warp == kConsumerWarps) {
     produce(a.rs, a.K, pass_cols, n_begin, n_end, ring, L.n_slots, sm, lane);
   } else {
-    if (PRO == PRO_NORM) {   // scale[m] = rsqrt(mean(x^2) + eps) over the whole row
+    if (PRO == PRO_NORM) {
+      // scale[m] = rsqrt(mean(x^2) + eps): the producing kernel left one partial sum of squares
+      // per CTA and row; they are added in a fixed order
       for (int m = warp; m < a.M; m += kConsumerWarps) {
-        const float4* xr = reinterpret_cast<const float4*>(a.x_f32 + (size_t)m * a.ldx);
         float ss = 0.f;
-        for (int i = lane; i < a.K / 4; i += 32) {
-          float4 v = xr[i];
-          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        }
+        for (int c = lane; c < a.ssq_n; c += 32) ss += a.ssq_in[(size_t)c * a.M + m];
         ss = warp_sum(ss);
         if (lane == 0) row_scale[m] = rsqrtf(ss / (float)a.K + a.eps);
       }
@@ -208,38 +237,35 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
     }
     int it = 0, buf = 0;
     bool alive = true;   // after a wait expired the loops still run (barriers stay matched) but do no work
-    const int g = lane >> 2, t = lane & 3;
     for (int k0 = 0; k0 < a.K; k0 += pass_cols) {
       const int k1 = min(a.K, k0 + pass_cols);
       consumer_sync();   // everyone is done reading the previous pass's planes
-      load_acts<PRO>(a, a_hi, a_lo, apitch, row_scale, k0, k1, tid);
+      load_acts<PRO>(a, plane_a, plane_b, ppitch, row_scale, k0, k1, tid);
       consumer_sync();
-      for (int n0 = n_begin; n0 < n_end; n0 += feat_per_tile, buf ^= 1) {
-        float acc[2][4];
+      for (int st = 0; st < n_st; ++st, buf ^= 1) {
+        float part[2][MT];
         if (alive)
-          alive = consume_tile<UPPER>(a_hi, a_lo, apitch, a.M, k1 - k0, ring, L.n_slots, sm, it, warp,
-                                      lane, acc);
+          alive = consume_tile<MT>(plane_a, plane_b, ppitch, k1 - k0, ring, L.n_slots, sm, it, warp,
+                                   lane, part);
         // partial sums of this warp's k-slice: red[buf][warp][slot row][m]
-        float* r = red + (size_t)buf * kRedFloats + (size_t)warp * kSlotRows * kMaxM;
+        if (lane < 4) {
+          float* r = red + (size_t)buf * kRedFloats + (size_t)warp * kSlotRows * kMaxM;
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-          r[(nt * 8 + 2 * t) * kMaxM + g] = acc[nt][0];
-          r[(nt * 8 + 2 * t + 1) * kMaxM + g] = acc[nt][1];
-          if (UPPER) {
-            r[(nt * 8 + 2 * t) * kMaxM + g + 8] = acc[nt][2];
-            r[(nt * 8 + 2 * t + 1) * kMaxM + g + 8] = acc[nt][3];
-          }
+          for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+              r[(lane + 4 * j) * kMaxM + m] = part[j][m];
         }
         consumer_sync();
-        // 256 threads = 16 slot rows x 16 m: add the 8 warps' partials into the CTA accumulator
+        // 128 threads = 8 slot rows x 16 m: add the 8 warps' partials into the CTA accumulator
         const int i = tid >> 4, m = tid & 15;
-        const int feat = a.rs.zip ? n0 + (i & 7) : n0 + i;
-        if (m < a.M && feat < n_end) {
+        const int feat = subtile_feature(a.rs, n_begin, st, i & 7);
+        if (i < kSlotRows && m < a.M && feat < n_end) {
           const float* rb = red + (size_t)buf * kRedFloats;
           float v = 0.f;
 #pragma unroll
           for (int w = 0; w < kConsumerWarps; ++w) v += rb[((size_t)w * kSlotRows + i) * kMaxM + m];
-          const int idx = (a.rs.zip && i >= 8 ? rows_half : 0) + (feat - n_begin);
+          const int idx = ((a.rs.zip && (st & 1)) ? rows_half : 0) + (feat - n_begin);
           float* dst = cta_out + (size_t)m * rows_cap + idx;
           *dst = (k0 == 0) ? v : *dst + v;
         }
@@ -249,12 +275,19 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
     const bool ok = !*(volatile int*)&sm.abort_flag;
     // ---- CTA-level epilogue over the accumulated features --------------------------------
     if (ok && EPI == EPI_STORE) {
-      for (int e = tid; e < a.M * cnt; e += kConsumerThreads) {
-        const int m = e / cnt, idx = e - m * cnt, n = n_begin + idx;
-        float v = cta_out[(size_t)m * rows_cap + idx];
-        if (a.bias) v += __bfloat162float(a.bias[n]);
-        if (a.res) v += a.res[(size_t)m * a.ldr + n];
-        a.out[(size_t)m * a.ldo + n] = v;
+      // warp per row m; also this CTA's share of the row's sum of squares for the next RMSNorm
+      for (int m = warp; m < a.M; m += kConsumerWarps) {
+        float ss = 0.f;
+        for (int idx = lane; idx < cnt; idx += 32) {
+          const int n = n_begin + idx;
+          float v = cta_out[(size_t)m * rows_cap + idx];
+          if (a.bias) v += __bfloat162float(a.bias[n]);
+          if (a.res) v += a.res[(size_t)m * a.ldr + n];
+          a.out[(size_t)m * a.ldo + n] = v;
+          ss += v * v;
+        }
+        ss = warp_sum(ss);
+        if (a.ssq_out && lane == 0) a.ssq_out[(size_t)blockIdx.x * a.M + m] = ss;
       }
     } else if (ok && EPI == EPI_SWIGLU) {
       for (int e = tid; e < a.M * cnt; e += kConsumerThreads) {
@@ -373,7 +406,14 @@ ps_status launch_gemm(ps_ctx* c, GemmArgs& a, cudaStream_t st) {
   if (a.pass_cols == 0) return fail(c, PS_ERR_UNSUPPORTED, "activation operand does not fit shared memory");
   Layout L = make_layout(a.M, std::min(a.pass_cols, a.K), a.rows_cap, smem_limit);
   a.status = c->dev_status;
-  auto kern = a.M > 8 ? k_ws_gemm<PRO, EPI, true> : k_ws_gemm<PRO, EPI, false>;
+  void (*kern)(GemmArgs, int) = nullptr;
+  switch (a.M) {   // the row count is a template parameter of the kernel
+#define PS_CASE(m) case m: kern = k_ws_gemm<PRO, EPI, m>; break;
+    PS_CASE(1) PS_CASE(2) PS_CASE(3) PS_CASE(4) PS_CASE(5) PS_CASE(6) PS_CASE(7) PS_CASE(8)
+    PS_CASE(9) PS_CASE(10) PS_CASE(11) PS_CASE(12) PS_CASE(13) PS_CASE(14) PS_CASE(15) PS_CASE(16)
+#undef PS_CASE
+    default: return fail(c, PS_ERR_UNSUPPORTED, "row count outside the fused kernels' range");
+  }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit);
   if (e != cudaSuccess) return cuda_check(c, e, "ws_gemm smem attribute");
   kern<<<n_cta, kThreads, L.total, st>>>(a, smem_limit);
@@ -383,6 +423,7 @@ ps_status launch_gemm(ps_ctx* c, GemmArgs& a, cudaStream_t st) {
 
 struct FusedScratch {
   float* qkv; float* att_ml; float* att_o; float* act; LmPart* parts; unsigned* ticket;
+  float* ssq[3];   // partial sums of squares of x0, a and hdn rows: [kMaxSm][kMaxM] each
   size_t bytes;
 };
 
@@ -402,6 +443,7 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
   s.act = (float*)take((size_t)kMaxM * g.ffn * 4);
   s.parts = (LmPart*)take((size_t)kMaxSm * kMaxM * sizeof(LmPart));
   s.ticket = (unsigned*)take(256);
+  for (int i = 0; i < 3; ++i) s.ssq[i] = (float*)take((size_t)kMaxSm * kMaxM * 4);
   s.bytes = off;
   return s;
 }
@@ -455,6 +497,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.embed = (BP)w.embed; a.mask_embed = (BP)w.mask_embed; a.mask_feat = (BP)w.mask_feat;
     a.hidden = (BP)hidden_last; a.tokens = token_last; a.H = H; a.V = V; a.R = R;
     a.out = c->x0; a.ldo = H; a.bias = (g.flags & PS_FLAG_FC_BIAS) ? (BP)w.b_fc : nullptr;
+    a.ssq_out = f.ssq[0];
     if ((s = launch_gemm<PRO_GATHER, EPI_STORE>(c, a, st))) return s;
   }
   prof_mark(c, st, "fc_norm");
@@ -464,6 +507,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.rs.rows[0] = Hq; a.rs.rows[1] = Hkv; a.rs.rows[2] = Hkv; a.rs.n_mats = 3;
     a.N = Hq + 2 * Hkv; a.K = H; a.M = M;
     a.x_f32 = c->x0; a.ldx = H; a.gain = (BP)w.g_in; a.eps = g.rms_eps;
+    a.ssq_in = f.ssq[0]; a.ssq_n = c->n_sm;
     a.out = f.qkv; a.ldo = Hq + 2 * Hkv;
     if ((s = launch_gemm<PRO_NORM, EPI_STORE>(c, a, st))) return s;
   }
@@ -477,6 +521,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.N = H; a.K = Hq; a.M = M;
     a.att_ml = f.att_ml; a.att_o = f.att_o; a.n_heads = g.n_heads; a.n_split = n_split; a.D = D;
     a.out = c->a; a.ldo = H; a.res = c->x0; a.ldr = H;
+    a.ssq_out = f.ssq[1];
     if ((s = launch_gemm<PRO_ATTN, EPI_STORE>(c, a, st))) return s;
   }
   prof_mark(c, st, "o_proj");
@@ -486,6 +531,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.rs.n_mats = 2; a.rs.zip = 1;
     a.N = F; a.K = H; a.M = M;
     a.x_f32 = c->a; a.ldx = H; a.gain = (BP)w.g_post; a.eps = g.rms_eps;
+    a.ssq_in = f.ssq[1]; a.ssq_n = c->n_sm;
     a.out = f.act; a.ldo = F;
     if ((s = launch_gemm<PRO_NORM, EPI_SWIGLU>(c, a, st))) return s;
   }
@@ -496,6 +542,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.N = H; a.K = F; a.M = M;
     a.x_f32 = f.act; a.ldx = F;
     a.out = hdn; a.ldo = H; a.res = c->a; a.ldr = H;
+    a.ssq_out = f.ssq[2];
     if ((s = launch_gemm<PRO_F32, EPI_STORE>(c, a, st))) return s;
   }
   prof_mark(c, st, "ffn");
@@ -504,6 +551,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.rs.W[0] = (BP)w.w_lm; a.rs.rows[0] = V; a.rs.n_mats = 1;
     a.N = V; a.K = H; a.M = M;
     a.x_f32 = hdn; a.ldx = H; a.gain = (BP)w.g_final; a.eps = g.rms_eps;
+    a.ssq_in = f.ssq[2]; a.ssq_n = c->n_sm;
     a.logits_out = logits_out; a.parts = f.parts; a.ticket = f.ticket;
     a.top_n = top_n; a.top_ids = top_ids; a.top_logit = top_logit; a.row_max = row_max; a.row_lse = row_lse;
     if ((s = launch_gemm<PRO_NORM, EPI_LMHEAD>(c, a, st))) return s;

@@ -1,17 +1,18 @@
 // Weight-streaming small-M GEMM for the bf16 drafter:  Y[m][n] = sum_k A[m][k] * W[n][k],
-// M = B*(k+1) <= 16 rows, W row-major bf16 (read exactly once from HBM), fp32 accumulation.
+// M = B*(k+1) <= 16 rows, W row-major bf16 (read exactly once from HBM), fp32 arithmetic.
 //
 // One CTA per SM owns a contiguous range of output features n (balanced to one row).  A
 // producer warp streams that range through a ring of shared-memory slots with bulk async
-// copies (cp.async.bulk + mbarrier transaction counts), 16 weight rows x KC columns per slot;
-// eight consumer warps split each slot along k and feed the tensor cores with
-// mma.sync.m16n8k16 (activation rows on the 16-wide axis, 8 weight rows per tile).
-//
-// Activations stay fp32-accurate although the tensor cores take bf16: each activation x is
-// held in shared memory as two bf16 planes, hi = bf16(x) and lo = bf16(x - hi), and every
-// weight fragment is multiplied with both (x*w = hi*w + lo*w up to 2^-17).  When M*K is too
-// large for shared memory the k range is processed in passes; partial sums of the CTA's
-// features stay in shared memory between passes.
+// copies (cp.async.bulk + mbarrier transaction counts), 8 weight rows x KC columns per slot,
+// one 4 KB copy per row (small bulk copies pay a fixed cost each and starve the memory system).
+// Eight consumer warps split each slot along k.  At these row counts the path is bound by HBM,
+// not by arithmetic: with M = 5 each weight needs 5 multiply-adds, about 45% of the fp32 rate
+// at full memory bandwidth, so the contraction runs on the fp32 pipes with packed
+// fma.rn.f32x2 (two k positions per instruction) on activations kept in shared memory as
+// fp32.  (Legacy mma.sync tiles were measured to cap this kernel near 4 TB/s on this part and
+// would need split bf16 activations to keep fp32 accuracy.)
+// When M*K is too large for shared memory the k range is processed in passes; partial sums of
+// the CTA's features stay in shared memory between passes.
 // Every wait is bounded: on expiry the kernel raises the device status word and returns.
 #pragma once
 #include <cuda_bf16.h>
@@ -26,14 +27,14 @@ namespace ws {
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;  // + one producer warp
-constexpr int KC = 512;                          // k-columns per slot
-constexpr int kSlotRows = 16;
-constexpr int kWPitch = KC * 2 + 64;             // bytes; = 64 mod 128 -> conflict-free 16-byte reads
+constexpr int KC = 2048;                         // k-columns per slot
+constexpr int kSlotRows = 8;
+constexpr int kWPitch = KC * 2 + 32;             // bytes; = 32 mod 128 -> conflict-free 16-byte reads
 constexpr int kSlotBytes = kSlotRows * kWPitch;
 constexpr int kMaxSlots = 12;
-constexpr int kMinSlots = 4;
-constexpr int kColsPerWarp = KC / kConsumerWarps;  // 64
-constexpr int kStepsPerWarp = kColsPerWarp / 32;   // 2
+constexpr int kMinSlots = 3;
+constexpr int kColsPerWarp = KC / kConsumerWarps;  // 256
+constexpr int kStepsPerWarp = kColsPerWarp / 64;   // 4: a warp covers 8 k-vectors of 8 per step
 constexpr long long kWaitCycles = 2000000000LL;    // ~1 s: bound of every mbarrier wait
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -90,15 +91,6 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 __device__ __forceinline__ void consumer_sync() {
   asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
 }
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                         uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
-      "{%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
 // ---- where the weight rows come from ---------------------------------------------------------
 // Logical output features are either the concatenation of up to three matrices (q|k|v) or, with
 // zip = 1, feature n is the PAIR (W[0] row n, W[1] row n) (gate, up).
@@ -109,16 +101,23 @@ struct RowSrc {
   int zip;
 };
 
-// Global address of slot row i (0..15) of the sub-tile that starts at logical feature n0; nullptr
-// if that row lies beyond n_end.  Sub-tiles hold 16 features (8 when zipped).
-__device__ __forceinline__ const __nv_bfloat16* slot_row_ptr(const RowSrc& rs, int n0, int i,
-                                                             int n_end, int K) {
-  if (rs.zip) {
-    int n = n0 + (i & 7);
-    return n < n_end ? rs.W[i >> 3] + (size_t)n * K : nullptr;
-  }
-  int n = n0 + i;
+// Sub-tiles hold 8 weight rows.  Plain / concatenated sources: sub-tile st covers features
+// n_begin + 8 st + i.  Zipped sources: sub-tiles alternate between the two matrices, st = 2 grp
+// + which covers rows n_begin + 8 grp + i of W[which].
+__device__ __forceinline__ int n_subtiles(const RowSrc& rs, int n_begin, int n_end) {
+  int groups = (n_end - n_begin + 7) >> 3;
+  return rs.zip ? 2 * groups : groups;
+}
+// Feature index of slot row i of sub-tile st (may be >= n_end: then the row does not exist).
+__device__ __forceinline__ int subtile_feature(const RowSrc& rs, int n_begin, int st, int i) {
+  return n_begin + 8 * (rs.zip ? (st >> 1) : st) + i;
+}
+// Global address of that row, nullptr if it lies beyond n_end.
+__device__ __forceinline__ const __nv_bfloat16* slot_row_ptr(const RowSrc& rs, int n_begin, int st,
+                                                             int i, int n_end, int K) {
+  int n = subtile_feature(rs, n_begin, st, i);
   if (n >= n_end) return nullptr;
+  if (rs.zip) return rs.W[st & 1] + (size_t)n * K;
   int m = 0;
   while (m + 1 < rs.n_mats && n >= rs.rows[m]) {
     n -= rs.rows[m];
@@ -134,12 +133,11 @@ struct Smem {
   int is_last;
 };
 
-// Activation pitch in bytes of one bf16 plane of `cols` columns: = 64 mod 128 so that the 8
-// threads of a quarter warp (two rows x four 16-byte columns) hit 32 distinct banks.
-__host__ __device__ inline int act_pitch(int cols) {
-  int raw = cols * 2;
-  return raw + ((64 - (raw & 127)) + 128) % 128;
-}
+// Activations of one pass live in two fp32 planes: element (m, k) sits in plane (k >> 2) & 1 at
+// float index m * plane_pitch(cols) + (k >> 3) * 4 + (k & 3).  A lane that needs the eight
+// activations k..k+7 of a row reads one float4 from each plane; the eight lanes of a warp that
+// work on neighbouring k-vectors read 128 contiguous bytes.
+__host__ __device__ inline int plane_pitch(int cols) { return cols / 2 + 4; }   // floats per row
 
 // Features [n_begin, n_end) of CTA `cta` out of `n_cta`, balanced to one feature.
 __host__ __device__ inline void cta_range(int N, int cta, int n_cta, int& n_begin, int& n_end) {
@@ -148,16 +146,17 @@ __host__ __device__ inline void cta_range(int N, int cta, int n_cta, int& n_begi
 }
 
 // Producer: streams every (pass, sub-tile, k-chunk) of the CTA's feature range through the ring.
-// Runs in one warp; lane i < 16 issues the copy of slot row i.  pass_cols is a multiple of KC.
+// Runs in one warp; lane i < 8 issues the copy of slot row i.  pass_cols is a multiple of 8.
 __device__ __forceinline__ void produce(const RowSrc& rs, int K, int pass_cols, int n_begin,
                                         int n_end, unsigned char* ring, int n_slots, Smem& sm,
                                         int lane) {
-  const int feat_per_tile = rs.zip ? 8 : 16;
+  const int n_st = n_subtiles(rs, n_begin, n_end);
   int it = 0;
   for (int k0 = 0; k0 < K; k0 += pass_cols) {
     const int k1 = min(K, k0 + pass_cols);
-    for (int n0 = n_begin; n0 < n_end; n0 += feat_per_tile) {
-      const __nv_bfloat16* src = lane < kSlotRows ? slot_row_ptr(rs, n0, lane, n_end, K) : nullptr;
+    for (int st = 0; st < n_st; ++st) {
+      const __nv_bfloat16* src =
+          lane < kSlotRows ? slot_row_ptr(rs, n_begin, st, lane, n_end, K) : nullptr;
       unsigned valid = __ballot_sync(0xffffffffu, src != nullptr);
       int n_valid = __popc(valid);
       for (int kc = k0; kc < k1; kc += KC, ++it) {
@@ -179,74 +178,83 @@ __device__ __forceinline__ void produce(const RowSrc& rs, int K, int pass_cols, 
   }
 }
 
-// Consumer: accumulates one sub-tile over the k range of the current pass (`cols_pass` columns)
-// into acc[ntile][4].  a_hi / a_lo: bf16 planes [M][cols_pass] with pitch apitch.  `it` is the
-// running chunk counter shared with the producer's schedule.  Returns false if a wait expired.
-template <bool kUpperRows>
-__device__ __forceinline__ bool consume_tile(const unsigned char* a_hi, const unsigned char* a_lo,
-                                             int apitch, int M, int cols_pass,
-                                             const unsigned char* ring, int n_slots, Smem& sm,
-                                             int& it, int warp, int lane, float (&acc)[2][4]) {
-  const int g = lane >> 2, t = lane & 3;
+// Two bf16 values packed in a 32-bit word, widened to a float pair (exact).
+__device__ __forceinline__ float2 widen2(uint32_t w) {
+  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+
+// Consumer: accumulates one sub-tile (8 weight rows) over the k range of the current pass
+// (`cols_pass` columns).  Lane = 4 * kq + r works on weight rows r and r + 4 and, in step s of
+// a chunk, on the k-vector (8 columns) number warp * 32 + s * 8 + kq.  On return lanes 0..3
+// (kq == 0) hold in out[j][m] the warp's partial sum for slot row r + 4 j and activation row m.
+// M (the number of activation rows) is a template parameter so that every loop unrolls and the
+// loads of a step are all issued before its multiply-adds.
+// `it` is the running chunk counter shared with the producer's schedule.  Returns false if a
+// wait expired.
+template <int M>
+__device__ __forceinline__ bool consume_tile(const float* plane_a, const float* plane_b, int ppitch,
+                                             int cols_pass, const unsigned char* ring, int n_slots,
+                                             Smem& sm, int& it, int warp, int lane,
+                                             float (&out)[2][M]) {
+  constexpr int MT = M;
+  const int r = lane & 3, kq = lane >> 2;
+  float2 acc[2][M];
 #pragma unroll
-  for (int i = 0; i < 2; ++i)
+  for (int j = 0; j < 2; ++j)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-  const bool row_lo = g < M, row_hi = kUpperRows && (g + 8 < M);
+    for (int m = 0; m < M; ++m) acc[j][m] = make_float2(0.f, 0.f);
   for (int c0 = 0; c0 < cols_pass; c0 += KC, ++it) {
     int slot = it % n_slots;
     uint32_t parity = (it / n_slots) & 1;
-    if (*(volatile int*)&sm.abort_flag) return false;
     if (!mbar_wait(&sm.full[slot], parity, &sm.abort_flag)) return false;
     const int cols = min(KC, cols_pass - c0);
-    const unsigned char* wbase = ring + (size_t)slot * kSlotBytes;
+    const unsigned char* w0 = ring + (size_t)slot * kSlotBytes + r * kWPitch;
+    const unsigned char* w1 = w0 + 4 * kWPitch;
 #pragma unroll
     for (int s = 0; s < kStepsPerWarp; ++s) {
-      int col = warp * kColsPerWarp + s * 32 + t * 8;     // column inside the chunk
-      if (warp * kColsPerWarp + s * 32 < cols) {          // warp-uniform
-        bool in = col < cols;
-        const uint4 z = make_uint4(0, 0, 0, 0);
-        uint4 b0 = in ? *reinterpret_cast<const uint4*>(wbase + g * kWPitch + col * 2) : z;
-        uint4 b1 = in ? *reinterpret_cast<const uint4*>(wbase + (g + 8) * kWPitch + col * 2) : z;
-        size_t aoff = (size_t)g * apitch + (size_t)(c0 + col) * 2;
-        uint4 h0 = (in && row_lo) ? *reinterpret_cast<const uint4*>(a_hi + aoff) : z;
-        uint4 l0 = (in && row_lo) ? *reinterpret_cast<const uint4*>(a_lo + aoff) : z;
-        uint4 h1 = z, l1 = z;
-        if (kUpperRows) {
-          size_t aoff1 = aoff + (size_t)8 * apitch;
-          h1 = (in && row_hi) ? *reinterpret_cast<const uint4*>(a_hi + aoff1) : z;
-          l1 = (in && row_hi) ? *reinterpret_cast<const uint4*>(a_lo + aoff1) : z;
+      const int col = warp * kColsPerWarp + s * 64 + kq * 8;     // column inside the chunk
+      if (col < cols) {
+        const uint4 q0 = *reinterpret_cast<const uint4*>(w0 + col * 2);
+        const uint4 q1 = *reinterpret_cast<const uint4*>(w1 + col * 2);
+        const int v4 = ((c0 + col) >> 3) * 4;
+        float4 xa[M], xb[M];
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+          xa[m] = *reinterpret_cast<const float4*>(plane_a + (size_t)m * ppitch + v4);
+          xb[m] = *reinterpret_cast<const float4*>(plane_b + (size_t)m * ppitch + v4);
         }
-        mma_bf16(acc[0], h0.x, h1.x, h0.y, h1.y, b0.x, b0.y);
-        mma_bf16(acc[0], h0.z, h1.z, h0.w, h1.w, b0.z, b0.w);
-        mma_bf16(acc[1], h0.x, h1.x, h0.y, h1.y, b1.x, b1.y);
-        mma_bf16(acc[1], h0.z, h1.z, h0.w, h1.w, b1.z, b1.w);
-        mma_bf16(acc[0], l0.x, l1.x, l0.y, l1.y, b0.x, b0.y);
-        mma_bf16(acc[0], l0.z, l1.z, l0.w, l1.w, b0.z, b0.w);
-        mma_bf16(acc[1], l0.x, l1.x, l0.y, l1.y, b1.x, b1.y);
-        mma_bf16(acc[1], l0.z, l1.z, l0.w, l1.w, b1.z, b1.w);
+        const float2 wa[4] = {widen2(q0.x), widen2(q0.y), widen2(q0.z), widen2(q0.w)};
+        const float2 wb[4] = {widen2(q1.x), widen2(q1.y), widen2(q1.z), widen2(q1.w)};
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+          const float2 x01 = make_float2(xa[m].x, xa[m].y), x23 = make_float2(xa[m].z, xa[m].w);
+          const float2 x45 = make_float2(xb[m].x, xb[m].y), x67 = make_float2(xb[m].z, xb[m].w);
+          acc[0][m] = __ffma2_rn(wa[0], x01, acc[0][m]);
+          acc[1][m] = __ffma2_rn(wb[0], x01, acc[1][m]);
+          acc[0][m] = __ffma2_rn(wa[1], x23, acc[0][m]);
+          acc[1][m] = __ffma2_rn(wb[1], x23, acc[1][m]);
+          acc[0][m] = __ffma2_rn(wa[2], x45, acc[0][m]);
+          acc[1][m] = __ffma2_rn(wb[2], x45, acc[1][m]);
+          acc[0][m] = __ffma2_rn(wa[3], x67, acc[0][m]);
+          acc[1][m] = __ffma2_rn(wb[3], x67, acc[1][m]);
+        }
       }
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.empty[slot]);
   }
-  return true;
-}
-
-// Splits fp32 values into the hi / lo bf16 planes, 8 consecutive columns at a time.
-__device__ __forceinline__ void store_split8(unsigned char* a_hi, unsigned char* a_lo, size_t off,
-                                             const float (&x)[8]) {
-  uint32_t h[4], l[4];
+  // even + odd k positions, then the eight k-vector lanes of each row (lane bits 2..4)
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    __nv_bfloat162 hh = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
-    float2 hf = __bfloat1622float2(hh);
-    __nv_bfloat162 ll = __floats2bfloat162_rn(x[2 * i] - hf.x, x[2 * i + 1] - hf.y);
-    h[i] = *reinterpret_cast<uint32_t*>(&hh);
-    l[i] = *reinterpret_cast<uint32_t*>(&ll);
-  }
-  *reinterpret_cast<uint4*>(a_hi + off) = make_uint4(h[0], h[1], h[2], h[3]);
-  *reinterpret_cast<uint4*>(a_lo + off) = make_uint4(l[0], l[1], l[2], l[3]);
+  for (int j = 0; j < 2; ++j)
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+      float v = acc[j][m].x + acc[j][m].y;
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      v += __shfl_xor_sync(0xffffffffu, v, 8);
+      v += __shfl_xor_sync(0xffffffffu, v, 16);
+      out[j][m] = v;
+    }
+  return true;
 }
 
 }  // namespace ws
