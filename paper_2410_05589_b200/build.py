@@ -44,7 +44,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
                 *[os.path.getmtime(h) for h in glob.glob(os.path.join(_PKG, "csrc", "*.cuh"))],
                 os.path.getmtime(os.path.join(_ROOT, "include", "ps.h")))):
             continue
-        cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(_ROOT, "include"), "-c", src, "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *os.environ.get("PS_NVCC_EXTRA", "").split(), "-I",
+               os.path.join(_ROOT, "include"), "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")

@@ -154,9 +154,10 @@ __device__ void load_acts(const GemmArgs& a, float* plane_a, float* plane_b, int
   }
 }
 
-// Shared-memory layout (dynamic): [Smem][red: 2 x 8 warps x 8 slot rows x 16 m floats]
-// [row scales][CTA accumulator: 16 m x rows_cap floats][act plane a][act plane b][ring]
-constexpr int kRedFloats = kConsumerWarps * kSlotRows * kMaxM;   // one buffer
+// Shared-memory layout (dynamic): [Smem][red: 2 x warps x 8 slot rows x ms(M) floats]
+// [row scales][CTA accumulator: M x rows_cap floats][act plane a][act plane b][ring]
+__host__ __device__ constexpr int m_stride(int M) { return M <= 8 ? 8 : 16; }
+__host__ __device__ constexpr int red_floats(int M) { return kConsumerWarps * kSlotRows * m_stride(M); }
 
 struct Layout {
   int off_red, off_scale, off_out, off_hi, off_lo, off_ring, n_slots, total;
@@ -165,9 +166,9 @@ struct Layout {
 __host__ __device__ inline Layout make_layout(int M, int pass_cols, int rows_cap, int smem_limit) {
   Layout L;
   int off = (int)((sizeof(Smem) + 127) & ~127u);
-  L.off_red = off; off += 2 * kRedFloats * 4;
+  L.off_red = off; off += 2 * red_floats(M) * 4;
   L.off_scale = off; off += 128;
-  L.off_out = off; off += ((rows_cap * kMaxM * 4) + 127) & ~127;
+  L.off_out = off; off += ((rows_cap * M * 4) + 127) & ~127;
   const int plane = ((M * plane_pitch(pass_cols) * 4) + 127) & ~127;
   L.off_hi = off; off += plane;
   L.off_lo = off; off += plane;
@@ -179,12 +180,13 @@ __host__ __device__ inline Layout make_layout(int M, int pass_cols, int rows_cap
 }
 
 // Smallest number of k passes whose activation planes leave room for kMinSlots ring slots.
-// Returns the columns per pass (multiple of 64) or 0 if nothing fits.
+// Passes are whole numbers of KC-column chunks so that every bulk copy but the last of a row
+// is a full chunk.  Returns the columns per pass or 0 if nothing fits.
 int choose_pass_cols(int M, int K, int rows_cap, int smem_limit) {
-  for (int n_pass = 1; n_pass <= (K + 63) / 64; ++n_pass) {
-    int cols = ((K + n_pass - 1) / n_pass + 63) / 64 * 64;
-    if (make_layout(M, std::min(cols, (K + 7) / 8 * 8), rows_cap, smem_limit).n_slots >= kMinSlots)
-      return cols;
+  const int n_chunks = (K + KC - 1) / KC;
+  for (int n_pass = 1; n_pass <= n_chunks; ++n_pass) {
+    int cols = (n_chunks + n_pass - 1) / n_pass * KC;
+    if (make_layout(M, std::min(cols, K), rows_cap, smem_limit).n_slots >= kMinSlots) return cols;
   }
   return 0;
 }
@@ -248,23 +250,24 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
           alive = consume_tile<MT>(plane_a, plane_b, ppitch, k1 - k0, ring, L.n_slots, sm, it, warp,
                                    lane, part);
         // partial sums of this warp's k-slice: red[buf][warp][slot row][m]
+        constexpr int MS = m_stride(MT), kRed = red_floats(MT);
         if (lane < 4) {
-          float* r = red + (size_t)buf * kRedFloats + (size_t)warp * kSlotRows * kMaxM;
+          float* r = red + (size_t)buf * kRed + (size_t)warp * kSlotRows * MS;
 #pragma unroll
           for (int j = 0; j < 2; ++j)
 #pragma unroll
             for (int m = 0; m < MT; ++m)
-              r[(lane + 4 * j) * kMaxM + m] = part[j][m];
+              r[(lane + 4 * j) * MS + m] = part[j][m];
         }
         consumer_sync();
-        // 128 threads = 8 slot rows x 16 m: add the 8 warps' partials into the CTA accumulator
-        const int i = tid >> 4, m = tid & 15;
+        // 8 slot rows x MS threads add the warps' partials into the CTA accumulator
+        const int i = tid / MS, m = tid % MS;
         const int feat = subtile_feature(a.rs, n_begin, st, i & 7);
         if (i < kSlotRows && m < a.M && feat < n_end) {
-          const float* rb = red + (size_t)buf * kRedFloats;
+          const float* rb = red + (size_t)buf * kRed;
           float v = 0.f;
 #pragma unroll
-          for (int w = 0; w < kConsumerWarps; ++w) v += rb[((size_t)w * kSlotRows + i) * kMaxM + m];
+          for (int w = 0; w < kConsumerWarps; ++w) v += rb[((size_t)w * kSlotRows + i) * MS + m];
           const int idx = ((a.rs.zip && (st & 1)) ? rows_half : 0) + (feat - n_begin);
           float* dst = cta_out + (size_t)m * rows_cap + idx;
           *dst = (k0 == 0) ? v : *dst + v;

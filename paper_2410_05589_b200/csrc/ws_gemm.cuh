@@ -5,7 +5,7 @@
 // producer warp streams that range through a ring of shared-memory slots with bulk async
 // copies (cp.async.bulk + mbarrier transaction counts), 8 weight rows x KC columns per slot,
 // one 4 KB copy per row (small bulk copies pay a fixed cost each and starve the memory system).
-// Eight consumer warps split each slot along k.  At these row counts the path is bound by HBM,
+// The consumer warps split each slot along k.  At these row counts the path is bound by HBM,
 // not by arithmetic: with M = 5 each weight needs 5 multiply-adds, about 45% of the fp32 rate
 // at full memory bandwidth, so the contraction runs on the fp32 pipes with packed
 // fma.rn.f32x2 (two k positions per instruction) on activations kept in shared memory as
@@ -24,7 +24,10 @@
 namespace ps {
 namespace ws {
 
-constexpr int kConsumerWarps = 8;
+#ifndef PS_CONSUMER_WARPS
+#define PS_CONSUMER_WARPS 8
+#endif
+constexpr int kConsumerWarps = PS_CONSUMER_WARPS;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;  // + one producer warp
 constexpr int KC = 2048;                         // k-columns per slot
@@ -33,8 +36,8 @@ constexpr int kWPitch = KC * 2 + 32;             // bytes; = 32 mod 128 -> confl
 constexpr int kSlotBytes = kSlotRows * kWPitch;
 constexpr int kMaxSlots = 12;
 constexpr int kMinSlots = 3;
-constexpr int kColsPerWarp = KC / kConsumerWarps;  // 256
-constexpr int kStepsPerWarp = kColsPerWarp / 64;   // 4: a warp covers 8 k-vectors of 8 per step
+constexpr int kColsPerWarp = KC / kConsumerWarps;
+constexpr int kStepsPerWarp = kColsPerWarp / 64;   // a warp covers 8 k-vectors of 8 columns per step
 constexpr long long kWaitCycles = 2000000000LL;    // ~1 s: bound of every mbarrier wait
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
