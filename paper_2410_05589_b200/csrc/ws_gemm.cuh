@@ -228,18 +228,18 @@ __device__ __forceinline__ bool consume_tile(const float* plane_a, const float* 
         }
         const float2 wa[4] = {widen2(q0.x), widen2(q0.y), widen2(q0.z), widen2(q0.w)};
         const float2 wb[4] = {widen2(q1.x), widen2(q1.y), widen2(q1.z), widen2(q1.w)};
+        // k pair outermost: 2 M independent accumulators between two uses of the same one
 #pragma unroll
-        for (int m = 0; m < M; ++m) {
-          const float2 x01 = make_float2(xa[m].x, xa[m].y), x23 = make_float2(xa[m].z, xa[m].w);
-          const float2 x45 = make_float2(xb[m].x, xb[m].y), x67 = make_float2(xb[m].z, xb[m].w);
-          acc[0][m] = __ffma2_rn(wa[0], x01, acc[0][m]);
-          acc[1][m] = __ffma2_rn(wb[0], x01, acc[1][m]);
-          acc[0][m] = __ffma2_rn(wa[1], x23, acc[0][m]);
-          acc[1][m] = __ffma2_rn(wb[1], x23, acc[1][m]);
-          acc[0][m] = __ffma2_rn(wa[2], x45, acc[0][m]);
-          acc[1][m] = __ffma2_rn(wb[2], x45, acc[1][m]);
-          acc[0][m] = __ffma2_rn(wa[3], x67, acc[0][m]);
-          acc[1][m] = __ffma2_rn(wb[3], x67, acc[1][m]);
+        for (int i = 0; i < 4; ++i) {
+#pragma unroll
+          for (int m = 0; m < M; ++m) {
+            const float2 x = i == 0 ? make_float2(xa[m].x, xa[m].y)
+                           : i == 1 ? make_float2(xa[m].z, xa[m].w)
+                           : i == 2 ? make_float2(xb[m].x, xb[m].y)
+                                    : make_float2(xb[m].z, xb[m].w);
+            acc[0][m] = __ffma2_rn(wa[i], x, acc[0][m]);
+            acc[1][m] = __ffma2_rn(wb[i], x, acc[1][m]);
+          }
         }
       }
     }
