@@ -84,6 +84,7 @@ size_t carve(const ps_config& g, ps_ctx* c, char* base) {
   void* hn = take(Md * H * 4);
   void* logits = take(Md * V * 4);
   void* fused = take(fused_scratch_bytes(g));
+  void* inv_freq = take(sizeof(double) * 64);
   void* st_hidden = take((size_t)g.max_batch * H * elem_bytes(g));
   void* st_tok = take((size_t)g.max_batch * 4);
   void* st_tlogits = take(Md * V * 4);
@@ -98,6 +99,7 @@ size_t carve(const ps_config& g, ps_ctx* c, char* base) {
     c->gate = (float*)gate; c->up = (float*)up; c->hdn = (float*)hdn; c->hn = (float*)hn;
     c->logits = (float*)logits;
     c->fused_scratch = fused;
+    c->rope_inv_freq = (double*)inv_freq;
     c->st_hidden = st_hidden; c->st_tok = (int*)st_tok; c->st_tlogits = (float*)st_tlogits;
     c->st_dlogits = (float*)st_dlogits; c->st_top = (int*)st_top; c->st_res = (int*)st_res;
     c->max_rows = (int)Md;
@@ -165,7 +167,7 @@ ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* w, void*
   if (e == cudaSuccess)
     e = cudaMemsetAsync(c->fused_scratch, 0, fused_scratch_bytes(*cfg), st);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * PS_MAX_BATCH, st);
-  if (e != cudaSuccess) {
+  if (e != cudaSuccess || launch_rope_table(c, st) != PS_OK) {
     delete c;
     return PS_ERR_CUDA;
   }
