@@ -63,7 +63,7 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// ---- prologues: the activation operand, columns [k0, k1), as fp32 planes in shared memory
+// ---- prologues: the activation operand, columns [k0, k1), as hi/lo bf16 planes in shared memory
 // One 8-column vector of row m starting at column k.
 template <int PRO>
 __device__ __forceinline__ void fetch8(const GemmArgs& a, int m, int k, float (&x)[8], uint4& raw) {
@@ -109,7 +109,7 @@ __device__ __forceinline__ void fetch8(const GemmArgs& a, int m, int k, float (&
 }
 
 template <int PRO>
-__device__ void load_acts(const GemmArgs& a, float* plane_a, float* plane_b, int ppitch,
+__device__ void load_acts(const GemmArgs& a, unsigned char* a_hi, unsigned char* a_lo, int apitch,
                           const float* row_scale, int k0, int k1, int tid) {
   constexpr int U = 4;   // vectors in flight per thread: all loads are issued before any store
   const int M = a.M, vecs = (k1 - k0) / 8, total = M * vecs;
@@ -129,12 +129,10 @@ __device__ void load_acts(const GemmArgs& a, float* plane_a, float* plane_b, int
       const int idx = base + u * kConsumerThreads;
       if (idx < total) {
         const int m = idx / vecs, v = idx - m * vecs;
-        const size_t off = (size_t)m * ppitch + (size_t)v * 4;
+        const size_t off = (size_t)m * apitch + (size_t)v * 16;
         if (PRO == PRO_GATHER) {
-          const float2 p0 = widen2(raw[u].x), p1 = widen2(raw[u].y), p2 = widen2(raw[u].z),
-                       p3 = widen2(raw[u].w);
-          *reinterpret_cast<float4*>(plane_a + off) = make_float4(p0.x, p0.y, p1.x, p1.y);
-          *reinterpret_cast<float4*>(plane_b + off) = make_float4(p2.x, p2.y, p3.x, p3.y);
+          *reinterpret_cast<uint4*>(a_hi + off) = raw[u];
+          *reinterpret_cast<uint4*>(a_lo + off) = make_uint4(0, 0, 0, 0);   // inputs are exact bf16
         } else {
           if (PRO == PRO_NORM) {
             const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&raw[u]);
@@ -146,18 +144,17 @@ __device__ void load_acts(const GemmArgs& a, float* plane_a, float* plane_b, int
               x[u][2 * i + 1] = x[u][2 * i + 1] * s * gf.y;
             }
           }
-          *reinterpret_cast<float4*>(plane_a + off) = make_float4(x[u][0], x[u][1], x[u][2], x[u][3]);
-          *reinterpret_cast<float4*>(plane_b + off) = make_float4(x[u][4], x[u][5], x[u][6], x[u][7]);
+          store_split8(a_hi, a_lo, off, x[u]);
         }
       }
     }
   }
 }
 
-// Shared-memory layout (dynamic): [Smem][red: 2 x warps x 8 slot rows x ms(M) floats]
-// [row scales][CTA accumulator: M x rows_cap floats][act plane a][act plane b][ring]
+// Shared-memory layout (dynamic): [Smem][red: 2 x warps x 16 sub-tile rows x ms(M) floats]
+// [row scales][CTA accumulator: M x rows_cap floats][act hi plane][act lo plane][ring]
 __host__ __device__ constexpr int m_stride(int M) { return M <= 8 ? 8 : 16; }
-__host__ __device__ constexpr int red_floats(int M) { return kConsumerWarps * kSlotRows * m_stride(M); }
+__host__ __device__ constexpr int red_floats(int M) { return kConsumerWarps * 16 * m_stride(M); }
 
 struct Layout {
   int off_red, off_scale, off_out, off_hi, off_lo, off_ring, n_slots, total;
@@ -169,7 +166,7 @@ __host__ __device__ inline Layout make_layout(int M, int pass_cols, int rows_cap
   L.off_red = off; off += 2 * red_floats(M) * 4;
   L.off_scale = off; off += 128;
   L.off_out = off; off += ((rows_cap * M * 4) + 127) & ~127;
-  const int plane = ((M * plane_pitch(pass_cols) * 4) + 127) & ~127;
+  const int plane = ((M * act_pitch(pass_cols)) + 127) & ~127;
   L.off_hi = off; off += plane;
   L.off_lo = off; off += plane;
   L.off_ring = off;
@@ -187,11 +184,12 @@ int choose_pass_cols(int M, int K, int rows_cap, int smem_limit) {
   for (int n_pass = 1; n_pass <= n_chunks; ++n_pass) {
     int cols = (n_chunks + n_pass - 1) / n_pass * KC;
     if (make_layout(M, std::min(cols, K), rows_cap, smem_limit).n_slots >= kMinSlots) return cols;
+    if (n_pass == n_chunks && make_layout(M, std::min(cols, K), rows_cap, smem_limit).n_slots >= 2) return cols;
   }
   return 0;
 }
 
-template <int PRO, int EPI, int MT>
+template <int PRO, int EPI, int NB>
 __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_limit) {
   extern __shared__ __align__(128) unsigned char smem[];
   Smem& sm = *reinterpret_cast<Smem*>(smem);
@@ -200,10 +198,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
   float* red = reinterpret_cast<float*>(smem + L.off_red);
   float* row_scale = reinterpret_cast<float*>(smem + L.off_scale);
   float* cta_out = reinterpret_cast<float*>(smem + L.off_out);   // [m][rows_cap]
-  float* plane_a = reinterpret_cast<float*>(smem + L.off_hi);
-  float* plane_b = reinterpret_cast<float*>(smem + L.off_lo);
+  unsigned char* a_hi = smem + L.off_hi;
+  unsigned char* a_lo = smem + L.off_lo;
   unsigned char* ring = smem + L.off_ring;
-  const int ppitch = plane_pitch(min(pass_cols, a.K));
+  const int apitch = act_pitch(min(pass_cols, a.K));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rows_cap = a.rows_cap, rows_half = rows_cap >> 1;
 
@@ -242,33 +240,36 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
     for (int k0 = 0; k0 < a.K; k0 += pass_cols) {
       const int k1 = min(a.K, k0 + pass_cols);
       consumer_sync();   // everyone is done reading the previous pass's planes
-      load_acts<PRO>(a, plane_a, plane_b, ppitch, row_scale, k0, k1, tid);
+      load_acts<PRO>(a, a_hi, a_lo, apitch, row_scale, k0, k1, tid);
       consumer_sync();
       for (int st = 0; st < n_st; ++st, buf ^= 1) {
-        float part[2][MT];
+        float part[NB][4];
         if (alive)
-          alive = consume_tile<MT>(plane_a, plane_b, ppitch, k1 - k0, ring, L.n_slots, sm, it, warp,
-                                   lane, part);
-        // partial sums of this warp's k-slice: red[buf][warp][slot row][m]
-        constexpr int MS = m_stride(MT), kRed = red_floats(MT);
-        if (lane < 4) {
-          float* r = red + (size_t)buf * kRed + (size_t)warp * kSlotRows * MS;
+          alive = consume_tile<NB>(a_hi, a_lo, apitch, a.M, k1 - k0, ring, L.n_slots, sm, it, warp, lane,
+                                   part);
+        // partial sums of this warp's k-slice: red[buf][warp][row of the sub-tile (0..15)][m]
+        constexpr int MS = 8 * NB, kRed = kConsumerWarps * 16 * MS;
+        {
+          const int g = lane >> 2, t = lane & 3;
+          float* r = red + (size_t)buf * kRed + (size_t)warp * 16 * MS;
 #pragma unroll
-          for (int j = 0; j < 2; ++j)
-#pragma unroll
-            for (int m = 0; m < MT; ++m)
-              r[(lane + 4 * j) * MS + m] = part[j][m];
+          for (int nb = 0; nb < NB; ++nb) {
+            r[g * MS + 8 * nb + 2 * t] = part[nb][0];
+            r[g * MS + 8 * nb + 2 * t + 1] = part[nb][1];
+            r[(g + 8) * MS + 8 * nb + 2 * t] = part[nb][2];
+            r[(g + 8) * MS + 8 * nb + 2 * t + 1] = part[nb][3];
+          }
         }
         consumer_sync();
-        // 8 slot rows x MS threads add the warps' partials into the CTA accumulator
+        // 16 sub-tile rows x MS threads add the warps' partials into the CTA accumulator
         const int i = tid / MS, m = tid % MS;
-        const int feat = subtile_feature(a.rs, n_begin, st, i & 7);
-        if (i < kSlotRows && m < a.M && feat < n_end) {
+        const int feat = subtile_feature(a.rs, n_begin, st, (i >> 3) & 1, i & 7);
+        if (i < 16 && m < a.M && feat < n_end) {
           const float* rb = red + (size_t)buf * kRed;
           float v = 0.f;
 #pragma unroll
-          for (int w = 0; w < kConsumerWarps; ++w) v += rb[((size_t)w * kSlotRows + i) * MS + m];
-          const int idx = ((a.rs.zip && (st & 1)) ? rows_half : 0) + (feat - n_begin);
+          for (int w = 0; w < kConsumerWarps; ++w) v += rb[((size_t)w * 16 + i) * MS + m];
+          const int idx = ((a.rs.zip && i >= 8) ? rows_half : 0) + (feat - n_begin);
           float* dst = cta_out + (size_t)m * rows_cap + idx;
           *dst = (k0 == 0) ? v : *dst + v;
         }
@@ -409,14 +410,7 @@ ps_status launch_gemm(ps_ctx* c, GemmArgs& a, cudaStream_t st) {
   if (a.pass_cols == 0) return fail(c, PS_ERR_UNSUPPORTED, "activation operand does not fit shared memory");
   Layout L = make_layout(a.M, std::min(a.pass_cols, a.K), a.rows_cap, smem_limit);
   a.status = c->dev_status;
-  void (*kern)(GemmArgs, int) = nullptr;
-  switch (a.M) {   // the row count is a template parameter of the kernel
-#define PS_CASE(m) case m: kern = k_ws_gemm<PRO, EPI, m>; break;
-    PS_CASE(1) PS_CASE(2) PS_CASE(3) PS_CASE(4) PS_CASE(5) PS_CASE(6) PS_CASE(7) PS_CASE(8)
-    PS_CASE(9) PS_CASE(10) PS_CASE(11) PS_CASE(12) PS_CASE(13) PS_CASE(14) PS_CASE(15) PS_CASE(16)
-#undef PS_CASE
-    default: return fail(c, PS_ERR_UNSUPPORTED, "row count outside the fused kernels' range");
-  }
+  auto kern = a.M > 8 ? k_ws_gemm<PRO, EPI, 2> : k_ws_gemm<PRO, EPI, 1>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit);
   if (e != cudaSuccess) return cuda_check(c, e, "ws_gemm smem attribute");
   kern<<<n_cta, kThreads, L.total, st>>>(a, smem_limit);
