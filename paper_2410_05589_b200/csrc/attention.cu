@@ -8,8 +8,8 @@
 // output channel for the P*V product.  q and the new k rows are rotated on the fly (RoPE, pair
 // (i, i + D/2), angle pos * base^(-2i/D), the angle formed and reduced in double); cached keys
 // are already rotated.  New k/v rows are rounded to bf16 as a cache row would be.
-// Output: un-normalised partial (max, sum, o) per (row, head, split); the o-projection's
-// prologue merges the splits.
+// Output: un-normalised partial (max, sum, o) per (row, head, split); the last split of a
+// (sequence, head) to finish merges them into the hi/lo bf16 planes the o-projection reads.
 #include <cfloat>
 
 #include "ps_internal.cuh"
@@ -46,7 +46,9 @@ __global__ void __launch_bounds__(kTile) k_attn_tile(SeqMap sm, const float* __r
                                                      int n_heads, int n_kv_heads, int max_ctx,
                                                      const double* __restrict__ inv_freq, int n_split,
                                                      float* __restrict__ att_ml,
-                                                     float* __restrict__ att_o) {
+                                                     float* __restrict__ att_o, unsigned* tickets,
+                                                     __nv_bfloat16* __restrict__ out_hi,
+                                                     __nv_bfloat16* __restrict__ out_lo) {
   constexpr int RMAX = kMaxRowsPerSeq, P = D + kPad, HALF = D / 2;
   extern __shared__ __align__(16) unsigned char att_smem[];
   const int h = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
@@ -217,6 +219,37 @@ __global__ void __launch_bounds__(kTile) k_attn_tile(SeqMap sm, const float* __r
       if (tid == 0) { att_ml[rec * 2] = run_m[j]; att_ml[rec * 2 + 1] = run_l[j]; }
     }
   }
+  // ---- the last split of this (sequence, head) to finish merges all of them and writes the
+  // attention output as hi/lo bf16 planes [row][n_heads * D] (no block waits for another)
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned tk = atomicAdd(&tickets[b * n_heads + h], 1u);
+    s_last = (tk == (unsigned)n_split - 1u);
+    if (s_last) tickets[b * n_heads + h] = 0u;
+  }
+  __syncthreads();
+  if (s_last && tid < D) {
+    __threadfence();
+    for (int j = 0; j < R; ++j) {
+      const size_t rec0 = ((size_t)(m0 + j) * n_heads + h) * n_split;
+      const volatile float* ml = att_ml + rec0 * 2;
+      float mx = -FLT_MAX;
+      for (int s = 0; s < n_split; ++s) mx = fmaxf(mx, ml[2 * s]);
+      float den = 0.f, num = 0.f;
+      for (int s = 0; s < n_split; ++s) {
+        const float w = __expf(ml[2 * s] - mx);
+        den += w * ml[2 * s + 1];
+        num += w * ((const volatile float*)att_o)[(rec0 + s) * D + tid];
+      }
+      const float x = num / den;
+      const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+      const size_t at = (size_t)(m0 + j) * n_heads * D + h * D + tid;
+      out_hi[at] = hi;
+      out_lo[at] = __float2bfloat16_rn(x - __bfloat162float(hi));
+    }
+  }
 }
 
 // inv_freq[i] = base^(-2i/D) in double, once per context.
@@ -238,9 +271,11 @@ ps_status launch_rope_table(ps_ctx* c, cudaStream_t st) {
 }
 
 // Chooses the number of key splits and launches the kernel.  qkv: float [M][Hq+2Hkv] before
-// RoPE.  Partials: att_ml [M][n_heads][n_split][2], att_o [M][n_heads][n_split][D].
+// RoPE.  Partials: att_ml [M][n_heads][n_split][2], att_o [M][n_heads][n_split][D]; merged
+// output planes out_hi / out_lo: bf16 [M][n_heads * D]; tickets: [B][n_heads], zero between calls.
 ps_status launch_attn_split(ps_ctx* c, const SeqMap& sm, int B, const float* qkv, float* att_ml,
-                            float* att_o, int* n_split_out, cudaStream_t st) {
+                            float* att_o, unsigned* tickets, __nv_bfloat16* out_hi,
+                            __nv_bfloat16* out_lo, cudaStream_t st) {
   const ps_config& g = c->cfg;
   const int R = g.k_masks + 1, D = g.head_dim, Hq = g.n_heads * D, Hkv = g.n_kv_heads * D;
   typedef const __nv_bfloat16* BP;
@@ -249,7 +284,6 @@ ps_status launch_attn_split(ps_ctx* c, const SeqMap& sm, int B, const float* qkv
   // enough blocks for about three per SM, never less than one tile of keys per split
   int want = (3 * c->n_sm + B * g.n_heads - 1) / (B * g.n_heads);
   int n_split = std::max(1, std::min(std::min(want, kAttnMaxSplit), (max_len + kTile - 1) / kTile));
-  *n_split_out = n_split;
   dim3 grid(g.n_heads, n_split, B);
   const size_t bytes = attn_smem_bytes(R, D);
   cudaError_t e = D == 64 ? cudaFuncSetAttribute(k_attn_tile<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes)
@@ -258,11 +292,11 @@ ps_status launch_attn_split(ps_ctx* c, const SeqMap& sm, int B, const float* qkv
   if (D == 64)
     k_attn_tile<64><<<grid, kTile, bytes, st>>>(sm, qkv, Hq + 2 * Hkv, Hq, Hkv, (BP)c->kcache, (BP)c->vcache,
                                                 g.n_heads, g.n_kv_heads, g.max_ctx, c->rope_inv_freq, n_split,
-                                                att_ml, att_o);
+                                                att_ml, att_o, tickets, out_hi, out_lo);
   else
     k_attn_tile<128><<<grid, kTile, bytes, st>>>(sm, qkv, Hq + 2 * Hkv, Hq, Hkv, (BP)c->kcache, (BP)c->vcache,
                                                  g.n_heads, g.n_kv_heads, g.max_ctx, c->rope_inv_freq, n_split,
-                                                 att_ml, att_o);
+                                                 att_ml, att_o, tickets, out_hi, out_lo);
   c->launches++;
   return cuda_check(c, cudaGetLastError(), "k_attn_tile");
 }

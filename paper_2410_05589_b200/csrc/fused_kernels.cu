@@ -1,14 +1,19 @@
 // Fused bf16 draft step for small M = B*(k+1) <= 16 (Sec. 4.1 "Inference", Sec. 4.3):
 // every projection is a launch of the weight-streaming GEMM (ws_gemm.cuh) with the neighbouring
-// element-wise work folded into its prologue / epilogue:
-//   fc        prologue = gather of [embedding ; feature] / [MASK] rows     epilogue = store x0
-//   q|k|v     prologue = RMSNorm(x0)                                       epilogue = store
-//   o         prologue = merge of the attention splits                     epilogue = + x0
-//   gate|up   prologue = RMSNorm(a)                                        epilogue = silu(g)*u
-//   down      prologue = copy                                              epilogue = + a
-//   LM head   prologue = RMSNorm(hdn)   epilogue = logits, per-CTA softmax/top-n partials,
-//                                                  merged by the last CTA to finish
-// Activations travel between the launches in fp32 (L2-resident, a few hundred KB).
+// element-wise work folded into its epilogue:
+//   fc        input = [embedding ; feature] / [MASK] rows (gathered by bulk copies)
+//             epilogue: x0 (+ bias), planes of x0 * g_in, partial sums of squares
+//   q|k|v     input = planes of x0 * g_in       epilogue: * rms scale of x0
+//   o         input = planes of the merged attention output (written by the attention kernel)
+//             epilogue: a = x0 + ., planes of a * g_post, partial sums of squares
+//   gate|up   input = planes of a * g_post      epilogue: * rms scale, silu(g)*u as planes
+//   down      input = planes of silu(g)*u       epilogue: hdn = a + ., planes of hdn * g_final
+//   LM head   input = planes of hdn * g_final   epilogue: * rms scale, logits, per-CTA
+//             softmax/top-n summaries merged by the last CTA to finish
+// "Planes" are the hi/lo bf16 split of an fp32 activation, kept in global memory ([M][width],
+// L2 resident) so that the next launch fetches its operand with a few bulk copies instead of
+// converting it with thread code.  RMSNorm's row scale is a scalar per row, so it is applied
+// to the product: W (s x * g) = s (W (x * g)).
 #include <algorithm>
 #include <cfloat>
 
@@ -19,7 +24,6 @@ namespace {
 
 using namespace ws;
 
-enum Pro { PRO_GATHER = 0, PRO_NORM = 1, PRO_F32 = 2, PRO_ATTN = 3 };
 enum Epi { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_LMHEAD = 2 };
 
 constexpr int kMaxM = 16;
@@ -34,21 +38,22 @@ struct LmPart {  // softmax / top-n summary of one CTA's vocabulary range for on
 struct GemmArgs {
   RowSrc rs;
   int N, K, M;
-  int pass_cols;   // k columns per pass (multiple of 64), chosen by the host
+  int pass_cols;   // k columns per pass (multiple of KC), chosen by the host
   int rows_cap;    // capacity (features per CTA, x2 when zipped) of the CTA accumulator
-  // ---- prologue inputs
-  const float* x_f32;  int ldx;        // PRO_NORM / PRO_F32: [M][ldx]
-  const __nv_bfloat16* gain; float eps;
-  const float* ssq_in; int ssq_n;      // PRO_NORM: [ssq_n][M] partial sums of squares of x_f32 rows
-  const __nv_bfloat16 *embed, *mask_embed, *mask_feat, *hidden;   // PRO_GATHER
+  // ---- activation operand: planes [M][ld_in] bf16 in global memory, or (gather) rows of
+  // [embed[token] ; hidden] for the first row of a sequence and [mask_embed ; mask_feat] after it
+  const __nv_bfloat16 *in_hi, *in_lo; int ld_in;
+  const __nv_bfloat16 *embed, *mask_embed, *mask_feat, *hidden;
   const int* tokens; int H, V, R;
-  // PRO_ATTN: partial attention results [M][n_heads][n_split] (m, l) and [..][D] o
-  const float* att_ml; const float* att_o; int n_heads, n_split, D;
+  // ---- RMSNorm row scale from [ssq_n][M] partial sums of squares (nullptr: no scaling)
+  const float* ssq_in; int ssq_n; float eps;
   // ---- epilogue outputs
-  float* out; int ldo;                 // EPI_STORE / EPI_SWIGLU: [M][ldo]
+  float* out; int ldo;                 // fp32 [M][ldo] (optional for EPI_SWIGLU)
   const __nv_bfloat16* bias;
   const float* res; int ldr;
-  float* ssq_out;                      // EPI_STORE: [gridDim.x][M] partial sums of squares, or nullptr
+  float* ssq_out;                      // [gridDim.x][M] partial sums of squares of out, or nullptr
+  __nv_bfloat16 *out_hi, *out_lo; int ld_plane;   // planes of out * gain_next, or nullptr
+  const __nv_bfloat16* gain_next;                 // nullptr: no gain
   // EPI_LMHEAD
   float* logits_out;                   // [M][N] or nullptr
   LmPart* parts;                       // [gridDim.x][M]
@@ -63,99 +68,15 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// ---- prologues: the activation operand, columns [k0, k1), as hi/lo bf16 planes in shared memory
-// One 8-column vector of row m starting at column k.
-template <int PRO>
-__device__ __forceinline__ void fetch8(const GemmArgs& a, int m, int k, float (&x)[8], uint4& raw) {
-  if (PRO == PRO_GATHER) {
-    // row m = (b, j): j == 0 -> [embed[token_b] ; hidden_b], j >= 1 -> [mask_embed ; mask_feat][j-1]
-    const int H = a.H, b = m / a.R, j = m - b * a.R;
-    const int half = k >= H ? 1 : 0, kk = k - half * H;
-    const __nv_bfloat16* src;
-    if (j == 0) {
-      int tok = min(max(a.tokens[b], 0), a.V - 1);
-      src = half == 0 ? a.embed + (size_t)tok * H : a.hidden + (size_t)b * H;
-    } else {
-      src = (half == 0 ? a.mask_embed : a.mask_feat) + (size_t)(j - 1) * H;
-    }
-    raw = *reinterpret_cast<const uint4*>(src + kk);
-  } else if (PRO == PRO_NORM || PRO == PRO_F32) {
-    const float4* xp = reinterpret_cast<const float4*>(a.x_f32 + (size_t)m * a.ldx + k);
-    float4 x0 = xp[0], x1 = xp[1];
-    x[0] = x0.x; x[1] = x0.y; x[2] = x0.z; x[3] = x0.w;
-    x[4] = x1.x; x[5] = x1.y; x[6] = x1.z; x[7] = x1.w;
-    if (PRO == PRO_NORM) raw = *reinterpret_cast<const uint4*>(a.gain + k);
-  } else {  // PRO_ATTN: merge the key splits of (row m, head h): o = sum_s w_s o_s / sum_s w_s l_s
-    const int D = a.D, S = a.n_split, nh = a.n_heads;
-    const int h = k / D, d0 = k - h * D;
-    const float* ml = a.att_ml + ((size_t)m * nh + h) * S * 2;
-    float mx = -FLT_MAX;
-    for (int s = 0; s < S; ++s) mx = fmaxf(mx, ml[2 * s]);
-    float den = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) x[i] = 0.f;
-    for (int s = 0; s < S; ++s) {
-      float w = __expf(ml[2 * s] - mx);
-      den += w * ml[2 * s + 1];
-      const float4* op = reinterpret_cast<const float4*>(a.att_o + (((size_t)m * nh + h) * S + s) * D + d0);
-      float4 o0 = op[0], o1 = op[1];
-      x[0] += w * o0.x; x[1] += w * o0.y; x[2] += w * o0.z; x[3] += w * o0.w;
-      x[4] += w * o1.x; x[5] += w * o1.y; x[6] += w * o1.z; x[7] += w * o1.w;
-    }
-    const float inv = 1.f / den;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) x[i] *= inv;
-  }
+// hi = bf16(x), lo = bf16(x - hi)
+__device__ __forceinline__ void split_store(__nv_bfloat16* hi, __nv_bfloat16* lo, float x) {
+  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+  *hi = h;
+  *lo = __float2bfloat16_rn(x - __bfloat162float(h));
 }
 
-template <int PRO>
-__device__ void load_acts(const GemmArgs& a, unsigned char* a_hi, unsigned char* a_lo, int apitch,
-                          const float* row_scale, int k0, int k1, int tid) {
-  constexpr int U = 4;   // vectors in flight per thread: all loads are issued before any store
-  const int M = a.M, vecs = (k1 - k0) / 8, total = M * vecs;
-  for (int base = tid; base < total; base += U * kConsumerThreads) {
-    float x[U][8];
-    uint4 raw[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int idx = base + u * kConsumerThreads;
-      if (idx < total) {
-        const int m = idx / vecs, v = idx - m * vecs;
-        fetch8<PRO>(a, m, k0 + v * 8, x[u], raw[u]);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int idx = base + u * kConsumerThreads;
-      if (idx < total) {
-        const int m = idx / vecs, v = idx - m * vecs;
-        const size_t off = (size_t)m * apitch + (size_t)v * 16;
-        if (PRO == PRO_GATHER) {
-          *reinterpret_cast<uint4*>(a_hi + off) = raw[u];
-          *reinterpret_cast<uint4*>(a_lo + off) = make_uint4(0, 0, 0, 0);   // inputs are exact bf16
-        } else {
-          if (PRO == PRO_NORM) {
-            const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&raw[u]);
-            const float s = row_scale[m];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              float2 gf = __bfloat1622float2(gp[i]);
-              x[u][2 * i] = x[u][2 * i] * s * gf.x;
-              x[u][2 * i + 1] = x[u][2 * i + 1] * s * gf.y;
-            }
-          }
-          store_split8(a_hi, a_lo, off, x[u]);
-        }
-      }
-    }
-  }
-}
-
-// Shared-memory layout (dynamic): [Smem][red: 2 x warps x 16 sub-tile rows x ms(M) floats]
+// Shared-memory layout (dynamic): [Smem][red: 2 x warps x 16 sub-tile rows x 8 NB floats]
 // [row scales][CTA accumulator: M x rows_cap floats][act hi plane][act lo plane][ring]
-__host__ __device__ constexpr int m_stride(int M) { return M <= 8 ? 8 : 16; }
-__host__ __device__ constexpr int red_floats(int M) { return kConsumerWarps * 16 * m_stride(M); }
-
 struct Layout {
   int off_red, off_scale, off_out, off_hi, off_lo, off_ring, n_slots, total;
 };
@@ -163,7 +84,7 @@ struct Layout {
 __host__ __device__ inline Layout make_layout(int M, int pass_cols, int rows_cap, int smem_limit) {
   Layout L;
   int off = (int)((sizeof(Smem) + 127) & ~127u);
-  L.off_red = off; off += 2 * red_floats(M) * 4;
+  L.off_red = off; off += 2 * kConsumerWarps * 16 * (M <= 8 ? 8 : 16) * 4;
   L.off_scale = off; off += 128;
   L.off_out = off; off += ((rows_cap * M * 4) + 127) & ~127;
   const int plane = ((M * act_pitch(pass_cols)) + 127) & ~127;
@@ -171,25 +92,71 @@ __host__ __device__ inline Layout make_layout(int M, int pass_cols, int rows_cap
   L.off_lo = off; off += plane;
   L.off_ring = off;
   int n = (smem_limit - off) / kSlotBytes;
+  n &= ~1;                                   // slots are used in pairs
   L.n_slots = n > kMaxSlots ? kMaxSlots : n;
   L.total = off + (L.n_slots > 0 ? L.n_slots : 0) * kSlotBytes;
   return L;
 }
 
-// Smallest number of k passes whose activation planes leave room for kMinSlots ring slots.
-// Passes are whole numbers of KC-column chunks so that every bulk copy but the last of a row
-// is a full chunk.  Returns the columns per pass or 0 if nothing fits.
+// Smallest number of k passes whose activation planes leave room for kMinSlots ring slots (at
+// the largest pass count two slots are enough).  Passes are whole numbers of KC-column chunks
+// so that every bulk copy but the last of a row is a full chunk.  Returns the columns per pass
+// or 0 if nothing fits.
 int choose_pass_cols(int M, int K, int rows_cap, int smem_limit) {
   const int n_chunks = (K + KC - 1) / KC;
   for (int n_pass = 1; n_pass <= n_chunks; ++n_pass) {
-    int cols = (n_chunks + n_pass - 1) / n_pass * KC;
-    if (make_layout(M, std::min(cols, K), rows_cap, smem_limit).n_slots >= kMinSlots) return cols;
-    if (n_pass == n_chunks && make_layout(M, std::min(cols, K), rows_cap, smem_limit).n_slots >= 2) return cols;
+    const int cols = (n_chunks + n_pass - 1) / n_pass * KC;
+    const int slots = make_layout(M, std::min(cols, K), rows_cap, smem_limit).n_slots;
+    if (slots >= kMinSlots || (n_pass == n_chunks && slots >= 2)) return cols;
   }
   return 0;
 }
 
-template <int PRO, int EPI, int NB>
+// Plane loader (one warp): fetches the activation operand of every pass with bulk copies, one
+// per row and plane.  Lanes 0..15 own the hi plane rows, lanes 16..31 the lo plane rows.
+template <bool GATHER>
+__device__ __forceinline__ void load_planes(const GemmArgs& a, unsigned char* a_hi, unsigned char* a_lo,
+                                            int apitch, Smem& sm, int lane) {
+  const int m = lane & 15, plane = lane >> 4;
+  const bool active = m < a.M && !(GATHER && plane == 1);
+  const __nv_bfloat16 *src_e = nullptr, *src_f = nullptr;   // gather: embedding half, feature half
+  if (GATHER && active) {
+    const int b = m / a.R, j = m - b * a.R;
+    if (j == 0) {
+      const int tok = min(max(a.tokens[b], 0), a.V - 1);
+      src_e = a.embed + (size_t)tok * a.H;
+      src_f = a.hidden + (size_t)b * a.H;
+    } else {
+      src_e = a.mask_embed + (size_t)(j - 1) * a.H;
+      src_f = a.mask_feat + (size_t)(j - 1) * a.H;
+    }
+  }
+  int pass = 0;
+  for (int k0 = 0; k0 < a.K; k0 += a.pass_cols, ++pass) {
+    const int k1 = min(a.K, k0 + a.pass_cols);
+    int ok = 1;
+    if (lane == 0) {
+      if (pass > 0) ok = mbar_wait(&sm.planes_empty, (pass - 1) & 1, &sm.abort_flag) ? 1 : 0;
+      if (ok) mbar_arrive_expect_tx(&sm.planes_full, (uint32_t)((GATHER ? 1 : 2) * a.M * (k1 - k0) * 2));
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (!ok) return;
+    if (!active) continue;
+    unsigned char* dst = (plane ? a_lo : a_hi) + (size_t)m * apitch;
+    if (GATHER) {
+      const int e0 = max(k0, 0), e1 = min(k1, a.H);           // part inside the embedding half
+      if (e1 > e0) bulk_g2s(dst + (size_t)(e0 - k0) * 2, src_e + e0, (uint32_t)((e1 - e0) * 2), &sm.planes_full);
+      const int f0 = max(k0, a.H), f1 = min(k1, 2 * a.H);     // part inside the feature half
+      if (f1 > f0)
+        bulk_g2s(dst + (size_t)(f0 - k0) * 2, src_f + (f0 - a.H), (uint32_t)((f1 - f0) * 2), &sm.planes_full);
+    } else {
+      const __nv_bfloat16* src = (plane ? a.in_lo : a.in_hi) + (size_t)m * a.ld_in + k0;
+      bulk_g2s(dst, src, (uint32_t)((k1 - k0) * 2), &sm.planes_full);
+    }
+  }
+}
+
+template <bool GATHER, int EPI, int NB>
 __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_limit) {
   extern __shared__ __align__(128) unsigned char smem[];
   Smem& sm = *reinterpret_cast<Smem*>(smem);
@@ -210,6 +177,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
       mbar_init(&sm.full[i], 1);
       mbar_init(&sm.empty[i], kConsumerWarps);
     }
+    mbar_init(&sm.planes_full, 1);
+    mbar_init(&sm.planes_empty, 1);
     sm.abort_flag = 0;
     sm.is_last = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -223,30 +192,31 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
 
   if (warp == kConsumerWarps) {
     produce(a.rs, a.K, pass_cols, n_begin, n_end, ring, L.n_slots, sm, lane);
+  } else if (warp == kConsumerWarps + 1) {
+    load_planes<GATHER>(a, a_hi, a_lo, apitch, sm, lane);
   } else {
-    if (PRO == PRO_NORM) {
-      // scale[m] = rsqrt(mean(x^2) + eps): the producing kernel left one partial sum of squares
-      // per CTA and row; they are added in a fixed order
-      for (int m = warp; m < a.M; m += kConsumerWarps) {
+    // scale[m] = rsqrt(mean(x^2) + eps): the producing kernel left one partial sum of squares per
+    // CTA and row; they are added in a fixed order.  Needed only by the epilogue.
+    for (int m = warp; m < a.M; m += kConsumerWarps) {
+      float sc = 1.f;
+      if (a.ssq_in) {
         float ss = 0.f;
         for (int c = lane; c < a.ssq_n; c += 32) ss += a.ssq_in[(size_t)c * a.M + m];
         ss = warp_sum(ss);
-        if (lane == 0) row_scale[m] = rsqrtf(ss / (float)a.K + a.eps);
+        sc = rsqrtf(ss / (float)a.K + a.eps);
       }
-      consumer_sync();
+      if (lane == 0) row_scale[m] = sc;
     }
-    int it = 0, buf = 0;
+    int it = 0, buf = 0, pass = 0;
     bool alive = true;   // after a wait expired the loops still run (barriers stay matched) but do no work
-    for (int k0 = 0; k0 < a.K; k0 += pass_cols) {
+    for (int k0 = 0; k0 < a.K; k0 += pass_cols, ++pass) {
       const int k1 = min(a.K, k0 + pass_cols);
-      consumer_sync();   // everyone is done reading the previous pass's planes
-      load_acts<PRO>(a, a_hi, a_lo, apitch, row_scale, k0, k1, tid);
-      consumer_sync();
+      if (alive) alive = mbar_wait(&sm.planes_full, pass & 1, &sm.abort_flag);
       for (int st = 0; st < n_st; ++st, buf ^= 1) {
         float part[NB][4];
         if (alive)
-          alive = consume_tile<NB>(a_hi, a_lo, apitch, a.M, k1 - k0, ring, L.n_slots, sm, it, warp, lane,
-                                   part);
+          alive = consume_tile<NB, !GATHER>(a_hi, a_lo, apitch, a.M, k1 - k0, ring, L.n_slots, sm, it,
+                                            warp, lane, part);
         // partial sums of this warp's k-slice: red[buf][warp][row of the sub-tile (0..15)][m]
         constexpr int MS = 8 * NB, kRed = kConsumerWarps * 16 * MS;
         {
@@ -274,21 +244,27 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
           *dst = (k0 == 0) ? v : *dst + v;
         }
       }
+      consumer_sync();                              // every warp is done with this pass's planes
+      if (tid == 0) mbar_arrive(&sm.planes_empty);
     }
-    consumer_sync();
     const bool ok = !*(volatile int*)&sm.abort_flag;
     // ---- CTA-level epilogue over the accumulated features --------------------------------
     if (ok && EPI == EPI_STORE) {
       // warp per row m; also this CTA's share of the row's sum of squares for the next RMSNorm
       for (int m = warp; m < a.M; m += kConsumerWarps) {
+        const float sc = row_scale[m];
         float ss = 0.f;
         for (int idx = lane; idx < cnt; idx += 32) {
           const int n = n_begin + idx;
-          float v = cta_out[(size_t)m * rows_cap + idx];
+          float v = cta_out[(size_t)m * rows_cap + idx] * sc;
           if (a.bias) v += __bfloat162float(a.bias[n]);
           if (a.res) v += a.res[(size_t)m * a.ldr + n];
           a.out[(size_t)m * a.ldo + n] = v;
           ss += v * v;
+          if (a.out_hi) {
+            const float gv = a.gain_next ? v * __bfloat162float(a.gain_next[n]) : v;
+            split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, gv);
+          }
         }
         ss = warp_sum(ss);
         if (a.ssq_out && lane == 0) a.ssq_out[(size_t)blockIdx.x * a.M + m] = ss;
@@ -296,18 +272,25 @@ __global__ void __launch_bounds__(kThreads, 1) k_ws_gemm(GemmArgs a, int smem_li
     } else if (ok && EPI == EPI_SWIGLU) {
       for (int e = tid; e < a.M * cnt; e += kConsumerThreads) {
         const int m = e / cnt, idx = e - m * cnt, n = n_begin + idx;
-        const float gv = cta_out[(size_t)m * rows_cap + idx];
-        const float uv = cta_out[(size_t)m * rows_cap + rows_half + idx];
-        a.out[(size_t)m * a.ldo + n] = gv / (1.f + __expf(-gv)) * uv;
+        const float sc = row_scale[m];
+        const float gv = cta_out[(size_t)m * rows_cap + idx] * sc;
+        const float uv = cta_out[(size_t)m * rows_cap + rows_half + idx] * sc;
+        const float act = gv / (1.f + __expf(-gv)) * uv;
+        if (a.out) a.out[(size_t)m * a.ldo + n] = act;
+        split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, act);
       }
     } else if (ok && EPI == EPI_LMHEAD) {
-      if (a.logits_out)
-        for (int e = tid; e < a.M * cnt; e += kConsumerThreads) {
-          const int m = e / cnt, idx = e - m * cnt;
-          a.logits_out[(size_t)m * a.N + n_begin + idx] = cta_out[(size_t)m * rows_cap + idx];
-        }
+      for (int e = tid; e < a.M * cnt; e += kConsumerThreads) {
+        const int m = e / cnt, idx = e - m * cnt;
+        const float v = cta_out[(size_t)m * rows_cap + idx] * row_scale[m];
+        cta_out[(size_t)m * rows_cap + idx] = v;
+        if (a.logits_out) a.logits_out[(size_t)m * a.N + n_begin + idx] = v;
+      }
+    }
+    if (EPI == EPI_LMHEAD) {
+      consumer_sync();
       // per-row summary of this CTA's vocabulary range: warp per row m
-      for (int m = warp; m < a.M; m += kConsumerWarps) {
+      for (int m = warp; m < a.M && ok; m += kConsumerWarps) {
         const float* lg = cta_out + (size_t)m * rows_cap;
         float mx = -FLT_MAX;
         for (int i = lane; i < cnt; i += 32) mx = fmaxf(mx, lg[i]);
@@ -401,7 +384,7 @@ int rows_cap_for(int N, int n_cta, bool zip) {
   return zip ? 2 * per : per;
 }
 
-template <int PRO, int EPI>
+template <bool GATHER, int EPI>
 ps_status launch_gemm(ps_ctx* c, GemmArgs& a, cudaStream_t st) {
   const int n_cta = c->n_sm;
   const int smem_limit = c->smem_optin;
@@ -410,7 +393,7 @@ ps_status launch_gemm(ps_ctx* c, GemmArgs& a, cudaStream_t st) {
   if (a.pass_cols == 0) return fail(c, PS_ERR_UNSUPPORTED, "activation operand does not fit shared memory");
   Layout L = make_layout(a.M, std::min(a.pass_cols, a.K), a.rows_cap, smem_limit);
   a.status = c->dev_status;
-  auto kern = a.M > 8 ? k_ws_gemm<PRO, EPI, 2> : k_ws_gemm<PRO, EPI, 1>;
+  auto kern = a.M > 8 ? k_ws_gemm<GATHER, EPI, 2> : k_ws_gemm<GATHER, EPI, 1>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_limit);
   if (e != cudaSuccess) return cuda_check(c, e, "ws_gemm smem attribute");
   kern<<<n_cta, kThreads, L.total, st>>>(a, smem_limit);
@@ -418,9 +401,13 @@ ps_status launch_gemm(ps_ctx* c, GemmArgs& a, cudaStream_t st) {
   return cuda_check(c, cudaGetLastError(), "k_ws_gemm");
 }
 
+struct Planes { __nv_bfloat16 *hi, *lo; };
+
 struct FusedScratch {
   float* qkv; float* att_ml; float* att_o; float* act; LmPart* parts; unsigned* ticket;
-  float* ssq[3];   // partial sums of squares of x0, a and hdn rows: [kMaxSm][kMaxM] each
+  unsigned* attn_tickets;   // [PS_MAX_BATCH][n_heads]
+  float* ssq[3];            // partial sums of squares of x0, a and hdn rows: [kMaxSm][kMaxM] each
+  Planes x0p, ap, hdnp, attnp, actp;
   size_t bytes;
 };
 
@@ -433,6 +420,12 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
     off += (bytes + 255) & ~(size_t)255;
     return base ? base + at : nullptr;
   };
+  auto planes = [&](size_t width) {
+    Planes p;
+    p.hi = (__nv_bfloat16*)take((size_t)kMaxM * width * 2);
+    p.lo = (__nv_bfloat16*)take((size_t)kMaxM * width * 2);
+    return p;
+  };
   FusedScratch s;
   s.qkv = (float*)take((size_t)kMaxM * (Hq + 2 * Hkv) * 4);
   s.att_ml = (float*)take((size_t)kMaxM * g.n_heads * kAttnMaxSplit * 2 * 4);
@@ -440,7 +433,10 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
   s.act = (float*)take((size_t)kMaxM * g.ffn * 4);
   s.parts = (LmPart*)take((size_t)kMaxSm * kMaxM * sizeof(LmPart));
   s.ticket = (unsigned*)take(256);
+  s.attn_tickets = (unsigned*)take((size_t)PS_MAX_BATCH * g.n_heads * 4);
   for (int i = 0; i < 3; ++i) s.ssq[i] = (float*)take((size_t)kMaxSm * kMaxM * 4);
+  s.x0p = planes(g.hidden); s.ap = planes(g.hidden); s.hdnp = planes(g.hidden);
+  s.attnp = planes(Hq); s.actp = planes(g.ffn);
   s.bytes = off;
   return s;
 }
@@ -482,7 +478,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
   const ps_config& g = c->cfg;
   const ps_weights& w = c->w;
   const int H = g.hidden, Hq = g.n_heads * g.head_dim, Hkv = g.n_kv_heads * g.head_dim, F = g.ffn,
-            V = g.vocab, R = g.k_masks + 1, M = B * R, D = g.head_dim;
+            V = g.vocab, R = g.k_masks + 1, M = B * R;
   typedef const __nv_bfloat16* BP;
   const FusedScratch f = carve_fused(g, (char*)c->fused_scratch);
   ps_status s;
@@ -495,7 +491,8 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.hidden = (BP)hidden_last; a.tokens = token_last; a.H = H; a.V = V; a.R = R;
     a.out = c->x0; a.ldo = H; a.bias = (g.flags & PS_FLAG_FC_BIAS) ? (BP)w.b_fc : nullptr;
     a.ssq_out = f.ssq[0];
-    if ((s = launch_gemm<PRO_GATHER, EPI_STORE>(c, a, st))) return s;
+    a.out_hi = f.x0p.hi; a.out_lo = f.x0p.lo; a.ld_plane = H; a.gain_next = (BP)w.g_in;
+    if ((s = launch_gemm<true, EPI_STORE>(c, a, st))) return s;
   }
   prof_mark(c, st, "fc_norm");
   {  // S2 q|k|v = W rms(x0)
@@ -503,23 +500,24 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.rs.W[0] = (BP)w.w_q; a.rs.W[1] = (BP)w.w_k; a.rs.W[2] = (BP)w.w_v;
     a.rs.rows[0] = Hq; a.rs.rows[1] = Hkv; a.rs.rows[2] = Hkv; a.rs.n_mats = 3;
     a.N = Hq + 2 * Hkv; a.K = H; a.M = M;
-    a.x_f32 = c->x0; a.ldx = H; a.gain = (BP)w.g_in; a.eps = g.rms_eps;
-    a.ssq_in = f.ssq[0]; a.ssq_n = c->n_sm;
+    a.in_hi = f.x0p.hi; a.in_lo = f.x0p.lo; a.ld_in = H;
+    a.ssq_in = f.ssq[0]; a.ssq_n = c->n_sm; a.eps = g.rms_eps;
     a.out = f.qkv; a.ldo = Hq + 2 * Hkv;
-    if ((s = launch_gemm<PRO_NORM, EPI_STORE>(c, a, st))) return s;
+    if ((s = launch_gemm<false, EPI_STORE>(c, a, st))) return s;
   }
   prof_mark(c, st, "qkv_rope");
-  int n_split = 1;
-  if ((s = launch_attn_split(c, sm, B, f.qkv, f.att_ml, f.att_o, &n_split, st))) return s;
+  if ((s = launch_attn_split(c, sm, B, f.qkv, f.att_ml, f.att_o, f.attn_tickets, f.attnp.hi, f.attnp.lo, st)))
+    return s;
   prof_mark(c, st, "attention");
   {  // S4 a = x0 + W_o attn
     GemmArgs a{};
     a.rs.W[0] = (BP)w.w_o; a.rs.rows[0] = H; a.rs.n_mats = 1;
     a.N = H; a.K = Hq; a.M = M;
-    a.att_ml = f.att_ml; a.att_o = f.att_o; a.n_heads = g.n_heads; a.n_split = n_split; a.D = D;
+    a.in_hi = f.attnp.hi; a.in_lo = f.attnp.lo; a.ld_in = Hq;
     a.out = c->a; a.ldo = H; a.res = c->x0; a.ldr = H;
     a.ssq_out = f.ssq[1];
-    if ((s = launch_gemm<PRO_ATTN, EPI_STORE>(c, a, st))) return s;
+    a.out_hi = f.ap.hi; a.out_lo = f.ap.lo; a.ld_plane = H; a.gain_next = (BP)w.g_post;
+    if ((s = launch_gemm<false, EPI_STORE>(c, a, st))) return s;
   }
   prof_mark(c, st, "o_proj");
   {  // S5a act = silu(W_g rms(a)) * (W_u rms(a))
@@ -527,31 +525,33 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.rs.W[0] = (BP)w.w_gate; a.rs.W[1] = (BP)w.w_up; a.rs.rows[0] = F; a.rs.rows[1] = F;
     a.rs.n_mats = 2; a.rs.zip = 1;
     a.N = F; a.K = H; a.M = M;
-    a.x_f32 = c->a; a.ldx = H; a.gain = (BP)w.g_post; a.eps = g.rms_eps;
-    a.ssq_in = f.ssq[1]; a.ssq_n = c->n_sm;
+    a.in_hi = f.ap.hi; a.in_lo = f.ap.lo; a.ld_in = H;
+    a.ssq_in = f.ssq[1]; a.ssq_n = c->n_sm; a.eps = g.rms_eps;
     a.out = f.act; a.ldo = F;
-    if ((s = launch_gemm<PRO_NORM, EPI_SWIGLU>(c, a, st))) return s;
+    a.out_hi = f.actp.hi; a.out_lo = f.actp.lo; a.ld_plane = F;
+    if ((s = launch_gemm<false, EPI_SWIGLU>(c, a, st))) return s;
   }
   float* hdn = feat_out ? feat_out : c->hdn;
   {  // S5b hdn = a + W_d act
     GemmArgs a{};
     a.rs.W[0] = (BP)w.w_down; a.rs.rows[0] = H; a.rs.n_mats = 1;
     a.N = H; a.K = F; a.M = M;
-    a.x_f32 = f.act; a.ldx = F;
+    a.in_hi = f.actp.hi; a.in_lo = f.actp.lo; a.ld_in = F;
     a.out = hdn; a.ldo = H; a.res = c->a; a.ldr = H;
     a.ssq_out = f.ssq[2];
-    if ((s = launch_gemm<PRO_F32, EPI_STORE>(c, a, st))) return s;
+    a.out_hi = f.hdnp.hi; a.out_lo = f.hdnp.lo; a.ld_plane = H; a.gain_next = (BP)w.g_final;
+    if ((s = launch_gemm<false, EPI_STORE>(c, a, st))) return s;
   }
   prof_mark(c, st, "ffn");
   {  // S6 logits = W_lm rms(hdn), softmax statistics and top-n without a second pass over logits
     GemmArgs a{};
     a.rs.W[0] = (BP)w.w_lm; a.rs.rows[0] = V; a.rs.n_mats = 1;
     a.N = V; a.K = H; a.M = M;
-    a.x_f32 = hdn; a.ldx = H; a.gain = (BP)w.g_final; a.eps = g.rms_eps;
-    a.ssq_in = f.ssq[2]; a.ssq_n = c->n_sm;
+    a.in_hi = f.hdnp.hi; a.in_lo = f.hdnp.lo; a.ld_in = H;
+    a.ssq_in = f.ssq[2]; a.ssq_n = c->n_sm; a.eps = g.rms_eps;
     a.logits_out = logits_out; a.parts = f.parts; a.ticket = f.ticket;
     a.top_n = top_n; a.top_ids = top_ids; a.top_logit = top_logit; a.row_max = row_max; a.row_lse = row_lse;
-    if ((s = launch_gemm<PRO_NORM, EPI_LMHEAD>(c, a, st))) return s;
+    if ((s = launch_gemm<false, EPI_LMHEAD>(c, a, st))) return s;
   }
   prof_mark(c, st, "lm_head");
   return PS_OK;

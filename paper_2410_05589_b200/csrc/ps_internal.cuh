@@ -102,7 +102,8 @@ size_t fused_scratch_bytes(const ps_config& g);
 ps_status fused_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* bytes);
 ps_status launch_rope_table(ps_ctx* c, cudaStream_t st);
 ps_status launch_attn_split(ps_ctx* c, const SeqMap& sm, int B, const float* qkv, float* att_ml,
-                            float* att_o, int* n_split_out, cudaStream_t st);
+                            float* att_o, unsigned* tickets, __nv_bfloat16* out_hi,
+                            __nv_bfloat16* out_lo, cudaStream_t st);
 ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last,
                            const int* token_last, int top_n, int* top_ids, float* top_logit,
                            float* row_max, float* row_lse, float* logits_out, float* feat_out,

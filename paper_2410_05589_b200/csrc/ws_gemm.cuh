@@ -32,7 +32,7 @@ namespace ws {
 #endif
 constexpr int kConsumerWarps = PS_CONSUMER_WARPS;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;  // + one producer warp
+constexpr int kThreads = kConsumerThreads + 64;  // + the weight producer warp and the plane loader warp
 constexpr int KC = 2048;                         // k-columns per slot
 constexpr int kSlotRows = 8;
 constexpr int kWPitch = KC * 2 + 64;             // bytes; = 64 mod 128 -> conflict-free 16-byte reads
@@ -142,6 +142,8 @@ __device__ __forceinline__ const __nv_bfloat16* slot_row_ptr(const RowSrc& rs, i
 struct Smem {
   uint64_t full[kMaxSlots];
   uint64_t empty[kMaxSlots];
+  uint64_t planes_full;    // the activation planes of the current pass have landed
+  uint64_t planes_empty;   // every consumer is done with them
   int abort_flag;
   int is_last;
 };
@@ -209,7 +211,7 @@ __device__ __forceinline__ void produce(const RowSrc& rs, int K, int pass_cols, 
 // 8 nb + 2t, 2t+1; out[nb][2..3] = the same for half 1.
 // `it` is the running slot counter shared with the producer's schedule.  Returns false if a
 // wait expired.
-template <int NB>
+template <int NB, bool LO>
 __device__ __forceinline__ bool consume_tile(const unsigned char* a_hi, const unsigned char* a_lo,
                                              int apitch, int M, int cols_pass,
                                              const unsigned char* ring, int n_slots, Smem& sm,
@@ -247,11 +249,13 @@ __device__ __forceinline__ bool consume_tile(const unsigned char* a_hi, const un
         for (int nb = 0; nb < NB; ++nb) {
           const size_t ro = (size_t)8 * nb * apitch + (size_t)col * 2;
           const uint4 h = (in && row_ok[nb]) ? *reinterpret_cast<const uint4*>(ah + ro) : z;
-          const uint4 l = (in && row_ok[nb]) ? *reinterpret_cast<const uint4*>(al + ro) : z;
           mma_bf16(p[nb][0], q0.x, q1.x, q0.y, q1.y, h.x, h.y);
           mma_bf16(p[nb][1], q0.z, q1.z, q0.w, q1.w, h.z, h.w);
-          mma_bf16(p[nb][2], q0.x, q1.x, q0.y, q1.y, l.x, l.y);
-          mma_bf16(p[nb][3], q0.z, q1.z, q0.w, q1.w, l.z, l.w);
+          if (LO) {   // the lo plane is identically zero when the operand is exact bf16
+            const uint4 l = (in && row_ok[nb]) ? *reinterpret_cast<const uint4*>(al + ro) : z;
+            mma_bf16(p[nb][2], q0.x, q1.x, q0.y, q1.y, l.x, l.y);
+            mma_bf16(p[nb][3], q0.z, q1.z, q0.w, q1.w, l.z, l.w);
+          }
         }
       }
     }
@@ -266,22 +270,6 @@ __device__ __forceinline__ bool consume_tile(const unsigned char* a_hi, const un
 #pragma unroll
     for (int k = 0; k < 4; ++k) out[nb][k] = (p[nb][0][k] + p[nb][1][k]) + (p[nb][2][k] + p[nb][3][k]);
   return true;
-}
-
-// Splits fp32 values into the hi / lo bf16 planes, 8 consecutive columns at a time.
-__device__ __forceinline__ void store_split8(unsigned char* a_hi, unsigned char* a_lo, size_t off,
-                                             const float (&x)[8]) {
-  uint32_t h[4], l[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    __nv_bfloat162 hh = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
-    float2 hf = __bfloat1622float2(hh);
-    __nv_bfloat162 ll = __floats2bfloat162_rn(x[2 * i] - hf.x, x[2 * i + 1] - hf.y);
-    h[i] = *reinterpret_cast<uint32_t*>(&hh);
-    l[i] = *reinterpret_cast<uint32_t*>(&ll);
-  }
-  *reinterpret_cast<uint4*>(a_hi + off) = make_uint4(h[0], h[1], h[2], h[3]);
-  *reinterpret_cast<uint4*>(a_lo + off) = make_uint4(l[0], l[1], l[2], l[3]);
 }
 
 }  // namespace ws
