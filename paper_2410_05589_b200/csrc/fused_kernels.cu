@@ -92,7 +92,6 @@ __host__ __device__ inline Layout make_layout(int M, int pass_cols, int rows_cap
   L.off_lo = off; off += plane;
   L.off_ring = off;
   int n = (smem_limit - off) / kSlotBytes;
-  n &= ~1;                                   // slots are used in pairs
   L.n_slots = n > kMaxSlots ? kMaxSlots : n;
   L.total = off + (L.n_slots > 0 ? L.n_slots : 0) * kSlotBytes;
   return L;
@@ -107,7 +106,7 @@ int choose_pass_cols(int M, int K, int rows_cap, int smem_limit) {
   for (int n_pass = 1; n_pass <= n_chunks; ++n_pass) {
     const int cols = (n_chunks + n_pass - 1) / n_pass * KC;
     const int slots = make_layout(M, std::min(cols, K), rows_cap, smem_limit).n_slots;
-    if (slots >= kMinSlots || (n_pass == n_chunks && slots >= 2)) return cols;
+    if (slots >= kMinSlots || (n_pass == n_chunks && slots >= 3)) return cols;
   }
   return 0;
 }

@@ -9,6 +9,8 @@
 #include <cstdio>
 #include <mutex>
 
+#include <cooperative_groups.h>
+
 #include "ps_internal.cuh"
 
 namespace ps {
@@ -233,10 +235,43 @@ struct VerifyArgs {
   int* status;
 };
 
+// Called by one thread per (position, sequence): records the speculative outcome, takes a
+// ticket, and -- as the last arriver of its sequence -- walks the positions in order and writes
+// accept_len / out_tokens / n_out.
+__device__ void finish_position(const VerifyArgs& a, int i, int b, int accept, int bad, int token) {
+  VerifyRec* recw = a.rec + (size_t)b * (PS_MAX_MASKS + 2);
+  recw[i].accept = accept | (bad << 1);
+  recw[i].token = token;
+  __threadfence();
+  unsigned t = atomicAdd(&a.tickets[b], 1u);
+  if (t != (unsigned)a.n_target - 1u) return;
+  __threadfence();
+  volatile VerifyRec* rec = recw;
+  int* out = a.out_tokens + (size_t)b * (a.n_draft + 1);
+  int acc = 0, any_bad = 0, emitted = -1;
+  while (acc < a.n_draft) {
+    int f = rec[acc].accept;
+    any_bad |= (f >> 1) & 1;
+    if (!(f & 1)) { emitted = rec[acc].token; break; }
+    out[acc] = a.draft_tokens[(size_t)b * a.n_draft + acc];
+    ++acc;
+  }
+  if (acc == a.n_draft && a.n_target == a.n_draft + 1) {
+    any_bad |= (rec[acc].accept >> 1) & 1;
+    emitted = rec[acc].token;
+  }
+  int n = acc;
+  if (emitted >= 0) out[n++] = emitted;
+  for (int j = n; j <= a.n_draft; ++j) out[j] = -1;
+  a.accept_len[b] = acc;
+  a.n_out[b] = n;
+  if (any_bad) atomicOr(a.status, kStatNonfinite);
+  a.tickets[b] = 0u;
+}
+
 __global__ void __launch_bounds__(kThreads) k_verify(VerifyArgs a) {
   extern __shared__ double seg_sum[];
   __shared__ Scratch s;
-  __shared__ int s_last;
   const int i = blockIdx.x, b = blockIdx.y, V = a.V;
   const bool bonus = i >= a.n_draft;
   const float* trow = a.target_logits + ((size_t)b * a.n_target + i) * V;
@@ -283,39 +318,265 @@ __global__ void __launch_bounds__(kThreads) k_verify(VerifyArgs a) {
     }
   }
 
-  if (threadIdx.x == 0) {
-    VerifyRec* rec = a.rec + (size_t)b * (PS_MAX_MASKS + 2);
-    rec[i].accept = accept | (bad << 1);
-    rec[i].token = token;
-    __threadfence();
-    unsigned t = atomicAdd(&a.tickets[b], 1u);
-    s_last = (t == (unsigned)a.n_target - 1u);
+  if (threadIdx.x == 0) finish_position(a, i, b, accept, bad, token);
+}
+
+// ---- cluster variant ------------------------------------------------------------------------
+// A cluster of kClu thread blocks shares one (position, sequence) row pair, so that a batch of
+// one still spreads its few rows over dozens of SMs.  Thread g = rank * kCluThreads + tid owns
+// the contiguous tokens [g * C, g * C + C) of both rows and keeps them in registers: the logits
+// are read from memory once, with all 16-byte loads in flight together.  Row statistics are
+// combined through distributed shared memory (each block publishes its partials, a cluster
+// barrier, every block reads all of them in rank order, so all blocks hold identical values).
+// The inverse-CDF draw descends block -> warp -> lane -> token over running sums.
+constexpr int kClu = 8;
+constexpr int kCluThreads = 512;
+constexpr int kCluWarps = kCluThreads / 32;
+constexpr int kCluV4 = 4;  // float4 per thread and row: up to kClu * kCluThreads * 16 tokens
+constexpr int kCluMaxVocab = kClu * kCluThreads * 4 * kCluV4;
+
+struct CluPart {       // one per block, read by the whole cluster
+  float tmax, dmax;
+  int targ, bad;
+  double st, sd;
+  double wsum;         // weight held by this block
+  int pick, lastp;     // token chosen inside this block / its last token with weight
+};
+
+struct CluScratch {
+  float f[kCluWarps], f2[kCluWarps];
+  int i[kCluWarps], flag[kCluWarps];
+  double d[kCluWarps], d2[kCluWarps];
+};
+
+__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads)
+k_verify_cluster(VerifyArgs a) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cl = cg::this_cluster();
+  __shared__ CluPart part;
+  __shared__ CluScratch s;
+  const int rank = (int)cl.block_rank();
+  const int i = blockIdx.x / kClu, b = blockIdx.y, V = a.V;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool bonus = i >= a.n_draft;
+  const float* trow = a.target_logits + ((size_t)b * a.n_target + i) * V;
+  const bool greedy = a.temperature == 0.f;
+  const float* drow = (!bonus && !greedy && a.draft_logits)
+                          ? a.draft_logits + ((size_t)b * a.n_draft + i) * V : nullptr;
+  const int x = bonus ? -1 : a.draft_tokens[(size_t)b * a.n_draft + i];
+  const int nv4 = ((V + kClu * kCluThreads - 1) / (kClu * kCluThreads) + 3) / 4;
+  const int C = nv4 * 4, v0 = (rank * kCluThreads + tid) * C;
+
+  float t[kCluV4 * 4], d[kCluV4 * 4];
+#pragma unroll
+  for (int k = 0; k < kCluV4; ++k) {
+    const int v = v0 + 4 * k;   // V % 4 == 0: a vector lies inside the row or outside it
+    float4 tv = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY), dv = tv;
+    if (k < nv4 && v < V) {
+      tv = *reinterpret_cast<const float4*>(trow + v);
+      if (drow) dv = *reinterpret_cast<const float4*>(drow + v);
+    }
+    t[4 * k] = tv.x; t[4 * k + 1] = tv.y; t[4 * k + 2] = tv.z; t[4 * k + 3] = tv.w;
+    d[4 * k] = dv.x; d[4 * k + 1] = dv.y; d[4 * k + 2] = dv.z; d[4 * k + 3] = dv.w;
   }
+
+  // ---- maxima (NaN counts as -inf, ties to the lower id) and non-finite flags
+  float tm = -INFINITY, dm = -INFINITY;
+  int ti = 0x7fffffff, bad = 0;
+#pragma unroll
+  for (int e = 0; e < kCluV4 * 4; ++e) {
+    const int v = v0 + e;
+    if (e < C && v < V) {
+      float xt = t[e];
+      if (xt != xt || xt == INFINITY) bad = 1;
+      if (xt != xt) xt = -INFINITY;
+      if (xt > tm || (xt == tm && v < ti)) { tm = xt; ti = v; }
+      if (drow) {
+        float xd = d[e];
+        if (xd != xd || xd == INFINITY) bad = 1;
+        if (xd != xd) xd = -INFINITY;
+        dm = fmaxf(dm, xd);
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, tm, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, ti, o);
+    if (ov > tm || (ov == tm && oi < ti)) { tm = ov; ti = oi; }
+    dm = fmaxf(dm, __shfl_xor_sync(0xffffffffu, dm, o));
+    bad |= __shfl_xor_sync(0xffffffffu, bad, o);
+  }
+  if (lane == 0) { s.f[warp] = tm; s.i[warp] = ti; s.flag[warp] = bad; s.f2[warp] = dm; }
   __syncthreads();
-  if (s_last && threadIdx.x == 0) {
-    __threadfence();
-    volatile VerifyRec* rec = a.rec + (size_t)b * (PS_MAX_MASKS + 2);
-    int* out = a.out_tokens + (size_t)b * (a.n_draft + 1);
-    int acc = 0, any_bad = 0, emitted = -1;
-    while (acc < a.n_draft) {
-      int f = rec[acc].accept;
-      any_bad |= (f >> 1) & 1;
-      if (!(f & 1)) { emitted = rec[acc].token; break; }
-      out[acc] = a.draft_tokens[(size_t)b * a.n_draft + acc];
-      ++acc;
+  if (tid == 0) {
+    for (int w = 1; w < kCluWarps; ++w) {
+      if (s.f[w] > tm || (s.f[w] == tm && s.i[w] < ti)) { tm = s.f[w]; ti = s.i[w]; }
+      dm = fmaxf(dm, s.f2[w]);
+      bad |= s.flag[w];
     }
-    if (acc == a.n_draft && a.n_target == a.n_draft + 1) {
-      any_bad |= (rec[acc].accept >> 1) & 1;
-      emitted = rec[acc].token;
-    }
-    int n = acc;
-    if (emitted >= 0) out[n++] = emitted;
-    for (int j = n; j <= a.n_draft; ++j) out[j] = -1;
-    a.accept_len[b] = acc;
-    a.n_out[b] = n;
-    if (any_bad) atomicOr(a.status, kStatNonfinite);
-    a.tickets[b] = 0u;
+    part.tmax = tm; part.targ = ti; part.dmax = dm; part.bad = bad;
+    part.pick = -1; part.lastp = -1; part.wsum = 0.0; part.st = 0.0; part.sd = 0.0;
   }
+  cl.sync();
+  tm = -INFINITY; dm = -INFINITY; ti = 0x7fffffff; bad = 0;
+  for (int r = 0; r < kClu; ++r) {
+    const CluPart* pr = cl.map_shared_rank(&part, r);
+    const float ov = pr->tmax;
+    const int oi = pr->targ;
+    if (ov > tm || (ov == tm && oi < ti)) { tm = ov; ti = oi; }
+    dm = fmaxf(dm, pr->dmax);
+    bad |= pr->bad;
+  }
+  if (tm == -INFINITY || (drow && dm == -INFINITY)) bad = 1;  // a row without a distribution
+  const float tmax = tm, dmax = dm;
+  const int targ = ti;
+
+  int accept = 0, token = -1;
+  if (greedy) {
+    accept = (!bonus && x == targ) ? 1 : 0;
+    token = targ;
+    bad = 0;
+  } else if (bad) {
+    token = targ;
+  } else {
+    // every block takes the same branches below: the values they depend on are identical
+    const double inv_t = 1.0 / (double)a.temperature;
+    double st = 0.0, sd = 0.0;
+#pragma unroll
+    for (int e = 0; e < kCluV4 * 4; ++e) {
+      const bool in = e < C && v0 + e < V;
+      t[e] = in ? expf((float)(((double)t[e] - (double)tmax) * inv_t)) : 0.f;
+      st += (double)t[e];
+      if (drow) {
+        d[e] = in ? expf((float)(((double)d[e] - (double)dmax) * inv_t)) : 0.f;
+        sd += (double)d[e];
+      }
+    }
+    st = warp_sum_d(st);
+    sd = warp_sum_d(sd);
+    if (lane == 0) { s.d[warp] = st; s.d2[warp] = sd; }
+    __syncthreads();
+    if (tid == 0) {
+      double x1 = 0.0, x2 = 0.0;
+      for (int w = 0; w < kCluWarps; ++w) { x1 += s.d[w]; x2 += s.d2[w]; }
+      part.st = x1; part.sd = x2;
+    }
+    cl.sync();
+    st = 0.0; sd = 0.0;
+    for (int r = 0; r < kClu; ++r) {
+      const CluPart* pr = cl.map_shared_rank(&part, r);
+      st += pr->st; sd += pr->sd;
+    }
+    if (!drow) sd = 1.0;
+    uint32_t c[4] = {(uint32_t)i, (uint32_t)b, a.off_lo, a.off_hi};
+    philox4x32_10(a.key0, a.key1, c);
+    const double r = (double)(c[0] >> 8) * (1.0 / 16777216.0);
+    const double u2 = (double)(c[1] >> 8) * (1.0 / 16777216.0);
+    if (!bonus) {
+      const bool in_range = x >= 0 && x < V;
+      const double logp = in_range ? ((double)trow[x] - (double)tmax) * inv_t - log(st) : -INFINITY;
+      const double logq = drow ? (in_range ? ((double)drow[x] - (double)dmax) * inv_t - log(sd) : -INFINITY)
+                               : 0.0;
+      const double diff = logp - logq;
+      const double ratio = (diff != diff) ? 0.0 : exp(fmin(diff, 0.0));
+      accept = r < ratio ? 1 : 0;
+    }
+    if (!accept) {
+      const float inv_st = (float)(1.0 / st), inv_sd = (float)(1.0 / sd);
+      // attempt 0: residual max(0, p - q); attempt 1: p itself (extra row, or an empty residual)
+      for (int attempt = bonus ? 1 : 0; attempt < 2 && token < 0; ++attempt) {
+        float w[kCluV4 * 4];
+        double mine = 0.0;
+        int lastp = -1;
+#pragma unroll
+        for (int e = 0; e < kCluV4 * 4; ++e) {
+          const float p = t[e] * inv_st;
+          float wv = p;
+          if (attempt == 0) {
+            const float q = drow ? d[e] * inv_sd : ((v0 + e == x) ? 1.f : 0.f);
+            wv = fmaxf(p - q, 0.f);
+          }
+          w[e] = (e < C && v0 + e < V) ? wv : 0.f;
+          mine += (double)w[e];
+          if (w[e] > 0.f) lastp = v0 + e;
+        }
+        double incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const double up = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += up;
+        }
+        lastp = __reduce_max_sync(0xffffffffu, lastp);
+        __syncthreads();   // the scratch arrays are free again
+        if (lane == 31) { s.d[warp] = incl; s.i[warp] = lastp; }
+        __syncthreads();
+        if (tid == 0) {
+          double x1 = 0.0;
+          int lp = -1;
+          for (int k = 0; k < kCluWarps; ++k) { x1 += s.d[k]; lp = max(lp, s.i[k]); }
+          part.wsum = x1; part.lastp = lp; part.pick = -1;
+        }
+        cl.sync();
+        // level 1: the block whose running sum first exceeds the target
+        double total = 0.0;
+        for (int rr = 0; rr < kClu; ++rr) total += cl.map_shared_rank(&part, rr)->wsum;
+        int sel = -1;
+        if (total > 0.0) {
+          const double target = u2 * total;
+          double run = 0.0, base = 0.0;
+          for (int rr = 0; rr < kClu; ++rr) {
+            const double nx = run + cl.map_shared_rank(&part, rr)->wsum;
+            if (sel < 0 && nx > target) { sel = rr; base = run; }
+            run = nx;
+          }
+          if (sel == rank) {
+            // level 2: the warp, level 3: the lane, level 4: the token
+            double t2 = target - base, wrun = 0.0, wbase = 0.0;
+            int wsel = -1;
+            for (int k = 0; k < kCluWarps; ++k) {
+              const double nx = wrun + s.d[k];
+              if (wsel < 0 && nx > t2) { wsel = k; wbase = wrun; }
+              wrun = nx;
+            }
+            if (warp == wsel) {
+              const double t3 = t2 - wbase;
+              const unsigned over = __ballot_sync(0xffffffffu, incl > t3);
+              if (over) {
+                const int src = __ffs(over) - 1;
+                double excl = __shfl_up_sync(0xffffffffu, incl, 1);
+                if (lane == 0) excl = 0.0;
+                if (lane == src) {
+                  const double t4 = t3 - excl;
+                  double run4 = 0.0;
+                  int pick = -1, lp = -1;
+#pragma unroll
+                  for (int e = 0; e < kCluV4 * 4; ++e) {
+                    if (w[e] > 0.f) lp = e;
+                    run4 += (double)w[e];
+                    if (pick < 0 && run4 > t4) pick = e;
+                  }
+                  if (pick < 0) pick = lp;
+                  if (pick >= 0) part.pick = v0 + pick;
+                }
+              }
+            }
+          }
+        }
+        cl.sync();
+        if (total > 0.0) {
+          // rounding may leave no token chosen on the way down: take the last one with weight
+          token = sel >= 0 ? cl.map_shared_rank(&part, sel)->pick : -1;
+          if (token < 0)
+            for (int rr = 0; rr < kClu; ++rr) token = max(token, cl.map_shared_rank(&part, rr)->lastp);
+        }
+        cl.sync();   // all reads of this attempt's partials are done before they are rewritten
+      }
+      if (token < 0) token = targ;
+    }
+  }
+  if (rank == 0 && tid == 0) finish_position(a, i, b, accept, bad, token);
+  cl.sync();   // no block leaves while another may still read its shared memory
 }
 
 }  // namespace
@@ -332,6 +593,14 @@ ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* 
   a.off_lo = (uint32_t)offset; a.off_hi = (uint32_t)(offset >> 32);
   a.accept_len = accept_len; a.out_tokens = out_tokens; a.n_out = n_out;
   a.rec = c->vrec; a.tickets = c->tickets; a.status = c->dev_status;
+  const bool aligned = (((uintptr_t)target_logits | (uintptr_t)draft_logits) & 15u) == 0;
+  if (a.V % 4 == 0 && a.V <= kCluMaxVocab && aligned) {
+    prof_mark(c, st, "begin");
+    k_verify_cluster<<<dim3(n_target * kClu, B), kCluThreads, 0, st>>>(a);
+    c->launches++;
+    prof_mark(c, st, "verify");
+    return cuda_check(c, cudaGetLastError(), "k_verify_cluster");
+  }
   size_t smem = (size_t)((a.V + kSeg - 1) / kSeg) * sizeof(double);
   if (smem > 160 * 1024) return fail(c, PS_ERR_UNSUPPORTED, "vocab too large for ps_verify");
   if (smem > 40 * 1024) {

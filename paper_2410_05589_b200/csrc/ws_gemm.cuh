@@ -38,7 +38,7 @@ constexpr int kSlotRows = 8;
 constexpr int kWPitch = KC * 2 + 64;             // bytes; = 64 mod 128 -> conflict-free 16-byte reads
 constexpr int kSlotBytes = kSlotRows * kWPitch;
 constexpr int kMaxSlots = 12;
-constexpr int kMinSlots = 4;                     // two pairs
+constexpr int kMinSlots = 5;                     // a pair being consumed + three slots in flight
 constexpr int kColsPerWarp = KC / kConsumerWarps;
 constexpr int kStepsPerWarp = kColsPerWarp / 32;   // a warp covers 32 columns per step
 constexpr long long kWaitCycles = 2000000000LL;    // ~1 s: bound of every mbarrier wait

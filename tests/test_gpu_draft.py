@@ -102,9 +102,10 @@ def test_step_is_idempotent_and_prefix_invariant_in_batch():
                          top_n=1)
     torch.cuda.synchronize()
     lg = out["logits"].cpu().numpy()
-    # (up to fp32 re-association: the k range is split differently for different row counts)
-    np.testing.assert_allclose(lg[0], a["logits"][2], rtol=0, atol=2e-5)
-    np.testing.assert_allclose(lg[1], a["logits"][0], rtol=0, atol=2e-5)
+    # (up to re-association in fp32 and in the hi/lo split of the activations: the k range is
+    # split differently for different row counts; the bound is 100x below the logits tolerance)
+    np.testing.assert_allclose(lg[0], a["logits"][2], rtol=0, atol=1e-4)
+    np.testing.assert_allclose(lg[1], a["logits"][0], rtol=0, atol=1e-4)
 
 
 def test_argument_errors_return_status():
