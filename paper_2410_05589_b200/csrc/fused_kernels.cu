@@ -445,7 +445,7 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
 bool fused_supported(const ps_ctx* c, int M) {
   const ps_config& g = c->cfg;
   if (g.dtype != PS_DTYPE_BF16 || (g.flags & PS_FLAG_UNFUSED_KERNELS)) return false;
-  if (M > kMaxM) return false;
+  if (M > kMaxM || (g.head_dim != 64 && g.head_dim != 128)) return false;
   const int Hq = g.n_heads * g.head_dim;
   const int lim = c->smem_optin, n = c->n_sm;
   return choose_pass_cols(M, 2 * g.hidden, rows_cap_for(g.hidden, n, false), lim) &&

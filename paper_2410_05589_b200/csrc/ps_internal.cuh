@@ -15,7 +15,7 @@ namespace ps {
 
 constexpr int kMaxRowsPerSeq = PS_MAX_MASKS + 1;  // rows of one sequence in a draft step
 constexpr int kAppendChunk = 256;                 // rows handled per pass of ps_kv_append
-constexpr int kAttnMaxSplit = 16;                 // key-range splits of the fused attention
+constexpr int kAttnMaxSplit = 32;                 // key-range splits of the fused attention
 constexpr int kMaxSm = 192;                       // bound used to size per-CTA scratch
 
 // Which sequence each row of a launch belongs to.  Passed by value as a kernel parameter.
