@@ -47,7 +47,8 @@ typedef enum {
 enum { PS_DTYPE_F32 = 0, PS_DTYPE_BF16 = 1 };
 enum {
   PS_FLAG_FC_BIAS = 1,          /* ps_weights.b_fc is used */
-  PS_FLAG_UNFUSED_KERNELS = 2   /* force the unfused fp32-activation kernels (debugging aid) */
+  PS_FLAG_UNFUSED_KERNELS = 2,  /* force the unfused fp32-activation kernels (debugging aid) */
+  PS_FLAG_MMA_SYNC_GEMM = 4     /* fused path: mma.sync GEMM kernels instead of the tcgen05 ones */
 };
 enum { PS_MAX_BATCH = 128, PS_MAX_MASKS = 15, PS_MAX_TOP_N = 8 };
 enum { PS_STATIC_MAX_BATCH = 128, PS_STATIC_MAX_VOCAB = 262144 }; /* limits of ps_verify_static */

@@ -17,6 +17,7 @@
 #include <algorithm>
 #include <cfloat>
 
+#include "umma_gemm.cuh"
 #include "ws_gemm.cuh"
 
 namespace ps {
@@ -407,6 +408,11 @@ struct FusedScratch {
   unsigned* attn_tickets;   // [PS_MAX_BATCH][n_heads]
   float* ssq[3];            // partial sums of squares of x0, a and hdn rows: [kMaxSm][kMaxM] each
   Planes x0p, ap, hdnp, attnp, actp;
+  // tensor-core path
+  __nv_bfloat16* xin;       // [kMaxM][2H] gathered fc input (exact bf16: one plane)
+  float* partials;          // [kMaxSm][2][16][128] partial tiles of CTAs that share a tile
+  unsigned* tile_tickets;   // one per tile of the widest stage, zero between launches
+  int n_part_rows;          // rows of `parts` and of each ssq array
   size_t bytes;
 };
 
@@ -430,23 +436,640 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
   s.att_ml = (float*)take((size_t)kMaxM * g.n_heads * kAttnMaxSplit * 2 * 4);
   s.att_o = (float*)take((size_t)kMaxM * g.n_heads * kAttnMaxSplit * g.head_dim * 4);
   s.act = (float*)take((size_t)kMaxM * g.ffn * 4);
-  s.parts = (LmPart*)take((size_t)kMaxSm * kMaxM * sizeof(LmPart));
+  // per-CTA (mma.sync path) or per-tile (tensor-core path) summaries
+  const int tiles_v = (g.vocab + 127) / 128, tiles_h = (g.hidden + 127) / 128;
+  s.n_part_rows = std::max(kMaxSm, std::max(tiles_v, tiles_h));
+  s.parts = (LmPart*)take((size_t)s.n_part_rows * kMaxM * sizeof(LmPart));
   s.ticket = (unsigned*)take(256);
   s.attn_tickets = (unsigned*)take((size_t)PS_MAX_BATCH * g.n_heads * 4);
-  for (int i = 0; i < 3; ++i) s.ssq[i] = (float*)take((size_t)kMaxSm * kMaxM * 4);
+  for (int i = 0; i < 3; ++i) s.ssq[i] = (float*)take((size_t)s.n_part_rows * kMaxM * 4);
+  s.xin = (__nv_bfloat16*)take((size_t)kMaxM * 2 * g.hidden * 2);
+  s.partials = (float*)take((size_t)kMaxSm * 2 * 16 * 128 * 4);
+  const size_t max_tiles = std::max<size_t>({(size_t)tiles_v, (size_t)(g.ffn + 63) / 64,
+                                             (Hq + 127) / 128 + 2 * ((Hkv + 127) / 128), (size_t)tiles_h});
+  s.tile_tickets = (unsigned*)take(max_tiles * 4);
   s.x0p = planes(g.hidden); s.ap = planes(g.hidden); s.hdnp = planes(g.hidden);
   s.attnp = planes(Hq); s.actp = planes(g.ffn);
   s.bytes = off;
   return s;
 }
 
+
+// =============================================================================================
+// Tensor-core path (tcgen05 + tiled TMA), see umma_gemm.cuh
+// =============================================================================================
+struct UArgs {
+  int N, K, M;
+  int n_tiles, KB;         // tiles of 128 weight rows (64 features when zipped), k-blocks of 64
+  int zip;                 // 1: a tile is 64 rows of matrix 0 (gate) over 64 rows of matrix 1 (up)
+  int lo;                  // 0: the activation operand is exact bf16 (no lo plane)
+  int n_mats;              // concatenated matrices (q|k|v): tiles never straddle two of them
+  int mat_tiles[3], mat_rows[3], mat_off[3];
+  const float* ssq_in; int ssq_n; float eps;
+  float* out; int ldo;
+  const __nv_bfloat16* bias;
+  const float* res; int ldr;
+  float* ssq_out;          // [n_tiles][M]
+  __nv_bfloat16 *out_hi, *out_lo; int ld_plane;
+  const __nv_bfloat16* gain_next;
+  float* logits_out; LmPart* parts; unsigned* ticket;
+  int top_n; int* top_ids; float* top_logit; float* row_max; float* row_lse;
+  float* partials; unsigned* tile_tickets;
+  int* status;
+};
+
+// CTA that owns unit u when CTA c owns [U c / G, U (c+1) / G).
+__device__ __forceinline__ int unit_owner(long long u, long long U, int G) {
+  return (int)(((u + 1) * G - 1) / U);
+}
+
+// Feature of accumulator row r of tile t; valid = false for rows past the end of a matrix.
+__device__ __forceinline__ int tile_feature(const UArgs& a, int t, int r, bool& valid) {
+  if (a.zip) {
+    const int f = t * 64 + (r & 63);
+    valid = f < a.N;
+    return f;
+  }
+  int m = 0;
+  while (m + 1 < a.n_mats && t >= a.mat_tiles[m]) {
+    t -= a.mat_tiles[m];
+    ++m;
+  }
+  const int local = t * umma::kTile + r;
+  valid = local < a.mat_rows[m];
+  return a.mat_off[m] + local;
+}
+
+// Epilogue of one finished tile; called by the 128 epilogue threads with v[m] = the tile's sums
+// for accumulator row r (= 32 * q + lane) and activation row m.
+template <int EPI>
+__device__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane, float (&v)[16]) {
+  using namespace umma;
+  const int et = 32 * q + lane;   // == r
+  bool valid;
+  const int n = tile_feature(a, t, r, valid);
+  if (EPI == EPI_STORE) {
+    float sq[16];
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+      sq[m] = 0.f;
+      if (m < a.M && valid) {
+        float x = v[m] * ctl.scale[m];
+        if (a.bias) x += __bfloat162float(a.bias[n]);
+        if (a.res) x += a.res[(size_t)m * a.ldr + n];
+        a.out[(size_t)m * a.ldo + n] = x;
+        sq[m] = x * x;
+        if (a.out_hi) {
+          const float gv = a.gain_next ? x * __bfloat162float(a.gain_next[n]) : x;
+          split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, gv);
+        }
+      }
+    }
+    if (a.ssq_out) {
+#pragma unroll
+      for (int m = 0; m < 16; ++m) {
+        if (m < a.M) {
+          const float s = warp_sum(sq[m]);
+          if (lane == 0) ctl.red[q][m] = s;
+        }
+      }
+      epi_sync();
+      if (et < a.M) a.ssq_out[(size_t)t * a.M + et] = (ctl.red[0][et] + ctl.red[1][et]) + (ctl.red[2][et] + ctl.red[3][et]);
+      epi_sync();
+    }
+  } else if (EPI == EPI_SWIGLU) {
+    if (r >= 64) {
+#pragma unroll
+      for (int m = 0; m < 16; ++m)
+        if (m < a.M) ctl.xch[m * 64 + (r - 64)] = v[m] * ctl.scale[m];
+    }
+    epi_sync();
+    if (r < 64 && valid) {
+#pragma unroll
+      for (int m = 0; m < 16; ++m) {
+        if (m < a.M) {
+          const float gv = v[m] * ctl.scale[m], uv = ctl.xch[m * 64 + r];
+          const float act = gv / (1.f + __expf(-gv)) * uv;
+          if (a.out) a.out[(size_t)m * a.ldo + n] = act;
+          split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, act);
+        }
+      }
+    }
+    epi_sync();
+  } else {  // EPI_LMHEAD
+    float x[16], bmax[16];
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+      x[m] = v[m] * ctl.scale[m < a.M ? m : 0];
+      if (m < a.M && valid && a.logits_out) a.logits_out[(size_t)m * a.N + n] = x[m];
+    }
+    // block maximum per row
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+      if (m < a.M) {
+        float mx = valid ? x[m] : -FLT_MAX;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) ctl.red[q][m] = mx;
+      }
+    }
+    epi_sync();
+#pragma unroll
+    for (int m = 0; m < 16; ++m)
+      bmax[m] = m < a.M ? fmaxf(fmaxf(ctl.red[0][m], ctl.red[1][m]), fmaxf(ctl.red[2][m], ctl.red[3][m])) : 0.f;
+    float my_vmax = 0.f;   // thread et < M reports row et
+    if (et < a.M) my_vmax = fmaxf(fmaxf(ctl.red[0][et], ctl.red[1][et]), fmaxf(ctl.red[2][et], ctl.red[3][et]));
+    epi_sync();
+    // block sum of exponentials per row
+#pragma unroll
+    for (int m = 0; m < 16; ++m) {
+      if (m < a.M) {
+        const float s = warp_sum(valid ? __expf(x[m] - bmax[m]) : 0.f);
+        if (lane == 0) ctl.red[q][m] = s;
+      }
+    }
+    epi_sync();
+    if (et < a.M) {
+      LmPart* p = a.parts + (size_t)t * a.M + et;
+      p->vmax = my_vmax;
+      p->sumexp = (ctl.red[0][et] + ctl.red[1][et]) + (ctl.red[2][et] + ctl.red[3][et]);
+    }
+    epi_sync();
+    // top-n per row: repeated block arg-max over the values after the previous pick
+    float pv[16]; int pi[16];
+#pragma unroll
+    for (int m = 0; m < 16; ++m) { pv[m] = FLT_MAX; pi[m] = -1; }
+    for (int tn = 0; tn < a.top_n; ++tn) {
+#pragma unroll
+      for (int m = 0; m < 16; ++m) {
+        if (m < a.M) {
+          const bool after = valid && ((x[m] < pv[m]) || (x[m] == pv[m] && n > pi[m]));
+          float bv = after ? x[m] : -FLT_MAX;
+          int bi = after ? n : 0x7fffffff;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+          }
+          if (lane == 0) { ctl.red[q][m] = bv; ctl.redi[q][m] = bi; }
+        }
+      }
+      epi_sync();
+#pragma unroll
+      for (int m = 0; m < 16; ++m) {
+        if (m < a.M) {
+          float bv = ctl.red[0][m]; int bi = ctl.redi[0][m];
+#pragma unroll
+          for (int w = 1; w < 4; ++w) {
+            const float ov = ctl.red[w][m]; const int oi = ctl.redi[w][m];
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+          }
+          pv[m] = bv; pi[m] = bi;
+          if (et == m) {
+            LmPart* p = a.parts + (size_t)t * a.M + m;
+            p->top_v[tn] = bv; p->top_i[tn] = bi;
+          }
+        }
+      }
+      epi_sync();
+    }
+  }
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(umma::kThreads, 1)
+k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUtensorMap tA1,
+            const __grid_constant__ CUtensorMap tA2, const __grid_constant__ CUtensorMap tBh,
+            const __grid_constant__ CUtensorMap tBl, UArgs a) {
+  using namespace umma;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;             // shared-space address of stage 0
+  unsigned char* stages = smem_raw + (base - raw);
+  Ctl& ctl = *reinterpret_cast<Ctl*>(stages + kStages * kStageBytes);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i) { mbar_init(&ctl.full[i], 1); mbar_init(&ctl.empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], kEpiThreads); }
+    ctl.abort_flag = 0; ctl.is_last = 0; ctl.tile_last = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {   // tensor memory for two accumulators
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem = *(volatile uint32_t*)&ctl.tmem_base;
+
+  const long long U = (long long)a.n_tiles * a.KB;
+  const long long u0 = U * blockIdx.x / gridDim.x, u1 = U * (blockIdx.x + 1) / gridDim.x;
+  volatile int* abort_flag = &ctl.abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---- TMA producer
+      const uint32_t bytes = kABytes + kBBytes * (a.lo ? 2 : 1);
+      int i = 0;
+      for (long long u = u0; u < u1; ++u, ++i) {
+        const int stage = i % kStages;
+        if (!mbar_wait(&ctl.empty[stage], ((i / kStages) & 1) ^ 1, abort_flag)) break;
+        int t = (int)(u / a.KB);
+        const int x = (int)(u - (long long)t * a.KB) * kBK;
+        const uint32_t dst = base + stage * kStageBytes;
+        mbar_arrive_expect_tx(&ctl.full[stage], bytes);
+        if (a.zip) {
+          tma_load_2d(dst, &tA0, x, t * 64, &ctl.full[stage]);
+          tma_load_2d(dst + kABytes / 2, &tA1, x, t * 64, &ctl.full[stage]);
+        } else {
+          int m = 0;
+          while (m + 1 < a.n_mats && t >= a.mat_tiles[m]) { t -= a.mat_tiles[m]; ++m; }
+          const CUtensorMap* map = m == 0 ? &tA0 : (m == 1 ? &tA1 : &tA2);
+          tma_load_2d(dst, map, x, t * kTile, &ctl.full[stage]);
+        }
+        tma_load_2d(dst + kABytes, &tBh, x, 0, &ctl.full[stage]);
+        if (a.lo) tma_load_2d(dst + kABytes + kBBytes, &tBl, x, 0, &ctl.full[stage]);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---- MMA issuer
+      int i = 0, seg = 0;
+      long long u = u0;
+      bool alive = true;
+      while (u < u1 && alive) {
+        const long long t = u / a.KB;
+        const long long seg_end = min(u1, (t + 1) * a.KB);
+        const int buf = seg & 1;
+        if (!mbar_wait(&ctl.acc_empty[buf], ((seg >> 1) & 1) ^ 1, abort_flag)) break;
+        fence_after_sync();
+        const uint32_t d = tmem + buf * kN;
+        uint32_t acc = 0;
+        for (; u < seg_end; ++u, ++i) {
+          const int stage = i % kStages;
+          if (!mbar_wait(&ctl.full[stage], (i / kStages) & 1, abort_flag)) { alive = false; break; }
+          fence_after_sync();
+          const uint32_t sa = base + stage * kStageBytes;
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+            const uint64_t da = smem_desc(sa + k * 32);
+            mma_f16(d, da, smem_desc(sa + kABytes + k * 32), acc);
+            acc = 1;
+            if (a.lo) mma_f16(d, da, smem_desc(sa + kABytes + kBBytes + k * 32), 1);
+          }
+          mma_commit(&ctl.empty[stage]);
+        }
+        if (alive) mma_commit(&ctl.acc_full[buf]);
+        ++seg;
+      }
+    }
+  } else {
+    // ---- epilogue warps: accumulator row r = 32 q + lane
+    const int q = warp & 3, r = 32 * q + lane, et = r;
+    for (int m = warp - 2; m < a.M; m += 4) {   // RMSNorm row scales of the input
+      float sc = 1.f;
+      if (a.ssq_in) {
+        float ss = 0.f;
+        for (int c = lane; c < a.ssq_n; c += 32) ss += a.ssq_in[(size_t)c * a.M + m];
+        ss = warp_sum(ss);
+        sc = rsqrtf(ss / (float)a.K + a.eps);
+      }
+      if (lane == 0) ctl.scale[m] = sc;
+    }
+    epi_sync();
+    int seg = 0;
+    long long u = u0;
+    while (u < u1) {
+      const int t = (int)(u / a.KB);
+      const long long t_begin = (long long)t * a.KB, t_end = t_begin + a.KB;
+      const long long seg_end = min(u1, t_end);
+      const bool whole = (u == t_begin) && (seg_end == t_end);
+      const int buf = seg & 1;
+      // all four warps take the same decision although each thread waits for itself
+      if (epi_any(!mbar_wait(&ctl.acc_full[buf], (seg >> 1) & 1, abort_flag))) break;
+      fence_after_sync();
+      float v[16];
+      tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + buf * kN, v);
+      fence_before_sync();
+      mbar_arrive(&ctl.acc_empty[buf]);
+      if (whole) {
+        tile_epilogue<EPI>(a, ctl, t, r, q, lane, v);
+      } else {
+        // partial tile: slot 0 = this CTA's first segment, slot 1 = its last one
+        const int slot = (t == (int)(u0 / a.KB)) ? 0 : 1;
+        float* P = a.partials + ((size_t)blockIdx.x * 2 + slot) * 16 * 128;
+#pragma unroll
+        for (int m = 0; m < 16; ++m)
+          if (m < a.M) P[m * 128 + r] = v[m];
+        __threadfence();
+        epi_sync();
+        const int c_first = unit_owner(t_begin, U, gridDim.x), c_last = unit_owner(t_end - 1, U, gridDim.x);
+        if (et == 0) {
+          int n_contrib = 0;   // CTAs between the owners of the tile's ends that hold any unit
+          for (int c = c_first; c <= c_last; ++c) n_contrib += (U * c / gridDim.x) < (U * (c + 1) / gridDim.x);
+          const unsigned old = atomicAdd(&a.tile_tickets[t], 1u);
+          const int last = old == (unsigned)(n_contrib - 1);
+          if (last) a.tile_tickets[t] = 0u;
+          ctl.tile_last = last;
+        }
+        epi_sync();
+        const bool last = ctl.tile_last != 0;
+        epi_sync();   // everyone has read the flag before a later segment rewrites it
+        if (last) {
+          __threadfence();
+#pragma unroll
+          for (int m = 0; m < 16; ++m) v[m] = 0.f;
+          for (int c = c_first; c <= c_last; ++c) {   // fixed order: the sum does not depend on who is last
+            if (U * c / gridDim.x >= U * (c + 1) / gridDim.x) continue;   // a CTA without units
+            const int c_tile0 = (int)((U * c / gridDim.x) / a.KB);
+            const int sl = (c == c_first && c_tile0 != t) ? 1 : 0;
+            const float* Pc = a.partials + ((size_t)c * 2 + sl) * 16 * 128;
+#pragma unroll
+            for (int m = 0; m < 16; ++m)
+              if (m < a.M) v[m] += __ldcg(Pc + m * 128 + r);
+          }
+          tile_epilogue<EPI>(a, ctl, t, r, q, lane, v);
+        }
+      }
+      u = seg_end;
+      ++seg;
+    }
+    fence_before_sync();
+  }
+
+  __syncthreads();
+  if (EPI == EPI_LMHEAD) {
+    // the last CTA to finish merges the per-tile summaries (no CTA waits for another)
+    if (tid == 0) {
+      __threadfence();
+      const unsigned tk = atomicAdd(a.ticket, 1u);
+      ctl.is_last = (tk == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (ctl.is_last && warp >= 2 && !ctl.abort_flag) {
+      __threadfence();
+      const int G = a.n_tiles;
+      for (int m = warp - 2; m < a.M; m += 4) {
+        const LmPart* P = a.parts + m;
+        float mx = -FLT_MAX;
+        for (int c = lane; c < G; c += 32) mx = fmaxf(mx, P[(size_t)c * a.M].vmax);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float se = 0.f;
+        for (int c = lane; c < G; c += 32) se += P[(size_t)c * a.M].sumexp * __expf(P[(size_t)c * a.M].vmax - mx);
+        se = warp_sum(se);
+        if (lane == 0) {
+          if (a.row_max) a.row_max[m] = mx;
+          if (a.row_lse) a.row_lse[m] = mx + logf(se);
+        }
+        float pv = FLT_MAX; int pi = -1;
+        for (int tn = 0; tn < a.top_n; ++tn) {
+          float bv = -FLT_MAX; int bi = 0x7fffffff;
+          for (int e = lane; e < G * a.top_n; e += 32) {
+            const int c = e / a.top_n, k = e - c * a.top_n;
+            const float xv = P[(size_t)c * a.M].top_v[k]; const int id = P[(size_t)c * a.M].top_i[k];
+            if (id == 0x7fffffff) continue;
+            const bool after = (xv < pv) || (xv == pv && id > pi);
+            if (after && (xv > bv || (xv == bv && id < bi))) { bv = xv; bi = id; }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+          }
+          if (lane == 0) { a.top_ids[(size_t)m * a.top_n + tn] = bi; a.top_logit[(size_t)m * a.top_n + tn] = bv; }
+          pv = bv; pi = bi;
+        }
+      }
+    }
+    if (ctl.is_last && tid == 0) *a.ticket = 0u;
+    __syncthreads();
+  }
+  if (ctl.abort_flag) {
+    // let copies and MMAs that are still in flight finish before shared and tensor memory go
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    if (tid == 0) atomicOr(a.status, kStatTimeout);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    fence_after_sync();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+// Rows of the fc input: [embedding(token) ; hidden] for a sequence's first row, the learned
+// [MASK] embedding and feature rows after it (Sec. 4.1).  One block per row.
+__global__ void k_gather_x(const __nv_bfloat16* __restrict__ embed, const __nv_bfloat16* __restrict__ mask_embed,
+                           const __nv_bfloat16* __restrict__ mask_feat, const __nv_bfloat16* __restrict__ hidden,
+                           const int* __restrict__ tokens, int H, int V, int R, __nv_bfloat16* __restrict__ xin) {
+  const int m = blockIdx.x, b = m / R, j = m - b * R;
+  const __nv_bfloat16 *e, *f;
+  if (j == 0) {
+    const int tok = min(max(tokens[b], 0), V - 1);
+    e = embed + (size_t)tok * H;
+    f = hidden + (size_t)b * H;
+  } else {
+    e = mask_embed + (size_t)(j - 1) * H;
+    f = mask_feat + (size_t)(j - 1) * H;
+  }
+  uint4* dst = reinterpret_cast<uint4*>(xin + (size_t)m * 2 * H);
+  const int nv = H / 8;
+  for (int i = threadIdx.x; i < nv; i += blockDim.x) {
+    dst[i] = reinterpret_cast<const uint4*>(e)[i];
+    dst[nv + i] = reinterpret_cast<const uint4*>(f)[i];
+  }
+}
+
+// ---- host side: tensor maps ---------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return (EncodeTiledFn)p;
+  }();
+  return fn;
+}
+
+// bf16 matrix [rows][cols] row-major; boxes of box_rows x 64 columns, 128-byte swizzle, zeros
+// outside the matrix.
+bool make_map(CUtensorMap* m, const void* base, size_t rows, size_t cols, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)umma::kBK, (cuuint32_t)box_rows};
+  cuuint32_t es[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct UmmaMaps {
+  CUtensorMap w_fc, w_q, w_k, w_v, w_o, w_gate, w_up, w_down, w_lm;
+  CUtensorMap xin, x0_hi, x0_lo, attn_hi, attn_lo, a_hi, a_lo, act_hi, act_lo, hdn_hi, hdn_lo;
+};
+
+UmmaMaps* build_maps(const ps_ctx* c, const FusedScratch& f) {
+  const ps_config& g = c->cfg;
+  const ps_weights& w = c->w;
+  const size_t H = g.hidden, Hq = (size_t)g.n_heads * g.head_dim, Hkv = (size_t)g.n_kv_heads * g.head_dim,
+               F = g.ffn, V = g.vocab;
+  UmmaMaps* u = new UmmaMaps;
+  bool ok = make_map(&u->w_fc, w.w_fc, H, 2 * H, 128) && make_map(&u->w_q, w.w_q, Hq, H, 128) &&
+            make_map(&u->w_k, w.w_k, Hkv, H, 128) && make_map(&u->w_v, w.w_v, Hkv, H, 128) &&
+            make_map(&u->w_o, w.w_o, H, Hq, 128) && make_map(&u->w_gate, w.w_gate, F, H, 64) &&
+            make_map(&u->w_up, w.w_up, F, H, 64) && make_map(&u->w_down, w.w_down, H, F, 128) &&
+            make_map(&u->w_lm, w.w_lm, V, H, 128);
+  ok = ok && make_map(&u->xin, f.xin, kMaxM, 2 * H, 16) && make_map(&u->x0_hi, f.x0p.hi, kMaxM, H, 16) &&
+       make_map(&u->x0_lo, f.x0p.lo, kMaxM, H, 16) && make_map(&u->attn_hi, f.attnp.hi, kMaxM, Hq, 16) &&
+       make_map(&u->attn_lo, f.attnp.lo, kMaxM, Hq, 16) && make_map(&u->a_hi, f.ap.hi, kMaxM, H, 16) &&
+       make_map(&u->a_lo, f.ap.lo, kMaxM, H, 16) && make_map(&u->act_hi, f.actp.hi, kMaxM, F, 16) &&
+       make_map(&u->act_lo, f.actp.lo, kMaxM, F, 16) && make_map(&u->hdn_hi, f.hdnp.hi, kMaxM, H, 16) &&
+       make_map(&u->hdn_lo, f.hdnp.lo, kMaxM, H, 16);
+  if (!ok) {
+    delete u;
+    return nullptr;
+  }
+  return u;
+}
+
+template <int EPI>
+ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
+                      const CUtensorMap& bh, const CUtensorMap& bl, UArgs& a, const FusedScratch& f,
+                      cudaStream_t st) {
+  a.KB = (a.K + umma::kBK - 1) / umma::kBK;
+  if (a.zip) {
+    a.n_tiles = (a.N + 63) / 64;
+  } else {
+    a.n_tiles = 0;
+    int off = 0;
+    for (int m = 0; m < a.n_mats; ++m) {
+      a.mat_tiles[m] = (a.mat_rows[m] + umma::kTile - 1) / umma::kTile;
+      a.mat_off[m] = off;
+      off += a.mat_rows[m];
+      a.n_tiles += a.mat_tiles[m];
+    }
+  }
+  a.partials = f.partials; a.tile_tickets = f.tile_tickets; a.status = c->dev_status;
+  auto kern = k_umma_gemm<EPI>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, umma::kSmemBytes);
+  if (e != cudaSuccess) return cuda_check(c, e, "umma smem attribute");
+  kern<<<c->n_sm, umma::kThreads, umma::kSmemBytes, st>>>(a0, a1, a2, bh, bl, a);
+  c->launches++;
+  return cuda_check(c, cudaGetLastError(), "k_umma_gemm");
+}
+
+ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B, const void* hidden_last,
+                          const int* token_last, int top_n, int* top_ids, float* top_logit, float* row_max,
+                          float* row_lse, float* logits_out, float* feat_out, cudaStream_t st) {
+  const ps_config& g = c->cfg;
+  const ps_weights& w = c->w;
+  const int H = g.hidden, Hq = g.n_heads * g.head_dim, Hkv = g.n_kv_heads * g.head_dim, F = g.ffn,
+            V = g.vocab, R = g.k_masks + 1, M = B * R;
+  typedef const __nv_bfloat16* BP;
+  const FusedScratch f = carve_fused(g, (char*)c->fused_scratch);
+  const int tiles_h = (H + umma::kTile - 1) / umma::kTile;
+  ps_status s;
+  prof_mark(c, st, "begin");
+  k_gather_x<<<M, 256, 0, st>>>((BP)w.embed, (BP)w.mask_embed, (BP)w.mask_feat, (BP)hidden_last, token_last, H, V,
+                                R, f.xin);
+  c->launches++;
+  {  // S1 fc: x0 = W_fc [e ; f] (+ b)
+    UArgs a{};
+    a.N = H; a.K = 2 * H; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 0;
+    a.out = c->x0; a.ldo = H; a.bias = (g.flags & PS_FLAG_FC_BIAS) ? (BP)w.b_fc : nullptr;
+    a.ssq_out = f.ssq[0];
+    a.out_hi = f.x0p.hi; a.out_lo = f.x0p.lo; a.ld_plane = H; a.gain_next = (BP)w.g_in;
+    if ((s = launch_umma<EPI_STORE>(c, u.w_fc, u.w_fc, u.w_fc, u.xin, u.xin, a, f, st))) return s;
+  }
+  prof_mark(c, st, "fc_norm");
+  {  // S2 q|k|v = W rms(x0)
+    UArgs a{};
+    a.N = Hq + 2 * Hkv; a.K = H; a.M = M; a.n_mats = 3;
+    a.mat_rows[0] = Hq; a.mat_rows[1] = Hkv; a.mat_rows[2] = Hkv; a.lo = 1;
+    a.ssq_in = f.ssq[0]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
+    a.out = f.qkv; a.ldo = Hq + 2 * Hkv;
+    if ((s = launch_umma<EPI_STORE>(c, u.w_q, u.w_k, u.w_v, u.x0_hi, u.x0_lo, a, f, st))) return s;
+  }
+  prof_mark(c, st, "qkv_rope");
+  if ((s = launch_attn_split(c, sm, B, f.qkv, f.att_ml, f.att_o, f.attn_tickets, f.attnp.hi, f.attnp.lo, st)))
+    return s;
+  prof_mark(c, st, "attention");
+  {  // S4 a = x0 + W_o attn
+    UArgs a{};
+    a.N = H; a.K = Hq; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 1;
+    a.out = c->a; a.ldo = H; a.res = c->x0; a.ldr = H;
+    a.ssq_out = f.ssq[1];
+    a.out_hi = f.ap.hi; a.out_lo = f.ap.lo; a.ld_plane = H; a.gain_next = (BP)w.g_post;
+    if ((s = launch_umma<EPI_STORE>(c, u.w_o, u.w_o, u.w_o, u.attn_hi, u.attn_lo, a, f, st))) return s;
+  }
+  prof_mark(c, st, "o_proj");
+  {  // S5a act = silu(W_g rms(a)) * (W_u rms(a))
+    UArgs a{};
+    a.N = F; a.K = H; a.M = M; a.zip = 1; a.n_mats = 2; a.lo = 1;
+    a.ssq_in = f.ssq[1]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
+    a.out = f.act; a.ldo = F;
+    a.out_hi = f.actp.hi; a.out_lo = f.actp.lo; a.ld_plane = F;
+    if ((s = launch_umma<EPI_SWIGLU>(c, u.w_gate, u.w_up, u.w_up, u.a_hi, u.a_lo, a, f, st))) return s;
+  }
+  float* hdn = feat_out ? feat_out : c->hdn;
+  {  // S5b hdn = a + W_d act
+    UArgs a{};
+    a.N = H; a.K = F; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 1;
+    a.out = hdn; a.ldo = H; a.res = c->a; a.ldr = H;
+    a.ssq_out = f.ssq[2];
+    a.out_hi = f.hdnp.hi; a.out_lo = f.hdnp.lo; a.ld_plane = H; a.gain_next = (BP)w.g_final;
+    if ((s = launch_umma<EPI_STORE>(c, u.w_down, u.w_down, u.w_down, u.act_hi, u.act_lo, a, f, st))) return s;
+  }
+  prof_mark(c, st, "ffn");
+  {  // S6 logits = W_lm rms(hdn), softmax statistics and top-n without a second pass over logits
+    UArgs a{};
+    a.N = V; a.K = H; a.M = M; a.n_mats = 1; a.mat_rows[0] = V; a.lo = 1;
+    a.ssq_in = f.ssq[2]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
+    a.logits_out = logits_out; a.parts = f.parts; a.ticket = f.ticket;
+    a.top_n = top_n; a.top_ids = top_ids; a.top_logit = top_logit; a.row_max = row_max; a.row_lse = row_lse;
+    if ((s = launch_umma<EPI_LMHEAD>(c, u.w_lm, u.w_lm, u.w_lm, u.hdn_hi, u.hdn_lo, a, f, st))) return s;
+  }
+  prof_mark(c, st, "lm_head");
+  return PS_OK;
+}
+
 }  // namespace
 
-bool fused_supported(const ps_ctx* c, int M) {
+// Builds the tensor maps of the tensor-core path once; without them (an old driver, unaligned
+// weights, too little shared memory) the mma.sync kernels serve.
+static void ensure_maps(ps_ctx* c) {
+  const ps_config& g = c->cfg;
+  const ps_weights& w = c->w;
+  if ((g.flags & PS_FLAG_MMA_SYNC_GEMM) || c->umma_tried) return;
+  c->umma_tried = true;
+  const bool aligned = ((((uintptr_t)w.w_fc | (uintptr_t)w.w_q | (uintptr_t)w.w_k | (uintptr_t)w.w_v |
+                          (uintptr_t)w.w_o | (uintptr_t)w.w_gate | (uintptr_t)w.w_up | (uintptr_t)w.w_down |
+                          (uintptr_t)w.w_lm | (uintptr_t)w.embed | (uintptr_t)w.mask_embed |
+                          (uintptr_t)w.mask_feat) & 15u) == 0);
+  if (aligned && c->smem_optin >= umma::kSmemBytes)
+    c->umma_maps = build_maps(c, carve_fused(g, (char*)c->fused_scratch));
+}
+
+bool fused_supported(ps_ctx* c, int M) {
   const ps_config& g = c->cfg;
   if (g.dtype != PS_DTYPE_BF16 || (g.flags & PS_FLAG_UNFUSED_KERNELS)) return false;
   if (M > kMaxM || (g.head_dim != 64 && g.head_dim != 128)) return false;
   const int Hq = g.n_heads * g.head_dim;
+  if (g.hidden % 8 || Hq % 8 || g.ffn % 8) return false;   // 16-byte operand rows
+  ensure_maps(c);
+  if (c->umma_maps) return true;
   const int lim = c->smem_optin, n = c->n_sm;
   return choose_pass_cols(M, 2 * g.hidden, rows_cap_for(g.hidden, n, false), lim) &&
          choose_pass_cols(M, g.hidden, rows_cap_for(Hq + 2 * g.n_kv_heads * g.head_dim, n, false), lim) &&
@@ -457,6 +1080,11 @@ bool fused_supported(const ps_ctx* c, int M) {
 }
 
 size_t fused_scratch_bytes(const ps_config& g) { return carve_fused(g, nullptr).bytes; }
+
+void fused_release(ps_ctx* c) {
+  delete static_cast<UmmaMaps*>(c->umma_maps);
+  c->umma_maps = nullptr;
+}
 
 ps_status fused_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* bytes) {
   const ps_config& g = c->cfg;
@@ -480,6 +1108,9 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
             V = g.vocab, R = g.k_masks + 1, M = B * R;
   typedef const __nv_bfloat16* BP;
   const FusedScratch f = carve_fused(g, (char*)c->fused_scratch);
+  if (c->umma_maps && !(g.flags & PS_FLAG_MMA_SYNC_GEMM))
+    return umma_draft_step(c, *static_cast<const UmmaMaps*>(c->umma_maps), sm, B, hidden_last, token_last, top_n,
+                           top_ids, top_logit, row_max, row_lse, logits_out, feat_out, st);
   ps_status s;
   prof_mark(c, st, "begin");
   {  // S1 fc: x0 = W_fc [e ; f] (+ b)

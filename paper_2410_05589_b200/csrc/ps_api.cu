@@ -178,6 +178,7 @@ ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* w, void*
 void ps_destroy(ps_ctx* c) {
   if (!c) return;
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+  fused_release(c);
   delete c;
 }
 

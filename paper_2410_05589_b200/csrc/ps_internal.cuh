@@ -68,6 +68,8 @@ struct ps_ctx {
   float *x_in, *x0, *xn, *q, *kv_tmp, *attn, *a, *an, *gate, *up, *hdn, *hn, *logits;
   // staging for ps_round_host
   void* fused_scratch;      // buffers of the fused bf16 path (see fused_kernels.cu)
+  void* umma_maps = nullptr;   // tensor maps of the tensor-core GEMMs, built on first use
+  bool umma_tried = false;
   double* rope_inv_freq;    // [head_dim/2] base^(-2i/d), filled once at ps_init
   int n_sm;                 // multiprocessors of the context's device
   int smem_optin;           // opt-in shared memory per block
@@ -97,8 +99,9 @@ ps_status plain_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
                            float* row_max, float* row_lse, float* logits_out, float* feat_out,
                            cudaStream_t st);
 // ---- fused bf16 kernels for small M ---------------------------------------------------------
-bool fused_supported(const ps_ctx* c, int M);
+bool fused_supported(ps_ctx* c, int M);
 size_t fused_scratch_bytes(const ps_config& g);
+void fused_release(ps_ctx* c);   // frees what the fused path holds on the host
 ps_status fused_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* bytes);
 ps_status launch_rope_table(ps_ctx* c, cudaStream_t st);
 ps_status launch_attn_split(ps_ctx* c, const SeqMap& sm, int B, const float* qkv, float* att_ml,

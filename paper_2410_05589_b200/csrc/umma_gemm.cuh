@@ -1,0 +1,138 @@
+// Weight-streaming small-M GEMM on the 5th-generation tensor cores:
+//   Y[m][n] = sum_k A[m][k] * W[n][k],  M = B*(k+1) <= 16 rows, W row-major bf16, fp32 sums.
+//
+// The weights are the M side of tcgen05.mma (128 weight rows per instruction), the activation
+// rows its N side (N = 16), so one instruction retires a 128 x 16 weight block (4 KB) against
+// one activation plane; the accumulator (128 lanes x 16 columns of fp32) lives in tensor
+// memory.  Operands reach shared memory by tiled TMA loads (cp.async.bulk.tensor.2d) in the
+// 128-byte-swizzled K-major layout the instruction reads: per stage one 128-row x 64-column
+// box of weights (16 KB) and the matching 16 x 64 boxes of the activation planes.
+//
+// Work is cut into units of (128-row tile, 64-column k-block); CTA c of a one-CTA-per-SM grid
+// takes the contiguous unit range [U c / G, U (c+1) / G) in tile-major order, so the load is
+// balanced to one 16 KB unit whatever N and K are.  A tile whose k range is shared by several
+// CTAs is reduced through fp32 partials in global memory: every contributor writes its partial
+// and takes a ticket, the last one adds the partials in CTA order (the sum does not depend on
+// who was last) and runs the tile's epilogue.  No CTA waits for another.
+//
+// Warp roles: warp 0 issues the TMA loads, warp 1 allocates tensor memory and issues the MMAs
+// (one lane), warps 2..5 read accumulators back (tcgen05.ld) and run the epilogues; two
+// accumulator buffers let a tile's epilogue overlap the next tile's MMAs.
+//
+// Activations stay fp32-accurate although the tensor cores take bf16: every activation x is
+// given as two bf16 planes, hi = bf16(x) and lo = bf16(x - hi), and every weight block is
+// multiplied with both (x*w = hi*w + lo*w up to 2^-17).
+// Every wait is bounded: on expiry the kernel raises the device status word and returns.
+#pragma once
+#include <cuda.h>
+
+#include "ws_gemm.cuh"
+
+namespace ps {
+namespace umma {
+
+using ws::mbar_arrive;
+using ws::mbar_arrive_expect_tx;
+using ws::mbar_init;
+using ws::mbar_wait;
+using ws::smem_u32;
+
+constexpr int kTile = 128;                        // weight rows per tile (MMA M)
+constexpr int kBK = 64;                           // k columns per unit: one 128-byte swizzle span
+constexpr int kN = 16;                            // activation rows (MMA N)
+constexpr int kABytes = kTile * kBK * 2;          // 16 KB
+constexpr int kBBytes = kN * kBK * 2;             // 2 KB per plane
+constexpr int kStageBytes = kABytes + 2 * kBBytes;
+constexpr int kStages = 10;
+constexpr int kThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr int kTmemCols = 32;                     // two accumulators of kN columns
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 x bf16, both operands K-major,
+// N / 8 in bits [17,23), M / 16 in bits [24,29).
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kN >> 3) << 17) |
+                            ((uint32_t)(kTile >> 4) << 24);
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+// Shared-memory matrix descriptor, K-major, 128-byte swizzle: rows of 128 bytes, groups of 8
+// rows 1024 bytes apart (stride byte offset), descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Tiled load of one box at element coordinates (x = column, y = row); x * 2 bytes must be a
+// multiple of 16.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(kIdesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the barrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void fence_before_sync() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void fence_after_sync() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// 16 consecutive accumulator columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void epi_sync() {
+  asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+}
+
+// Barrier of the epilogue threads that also tells every one of them whether any passed true.
+__device__ __forceinline__ bool epi_any(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, 1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)pred), "n"(kEpiThreads)
+      : "memory");
+  return r != 0;
+}
+
+// ---- control block behind the stages ----------------------------------------------------------
+struct Ctl {
+  uint64_t full[kStages];     // a stage's boxes have landed
+  uint64_t empty[kStages];    // the MMAs that read a stage have completed
+  uint64_t acc_full[2];       // an accumulator holds a finished segment
+  uint64_t acc_empty[2];      // the epilogue warps have read it back
+  uint32_t tmem_base;
+  int abort_flag;
+  int is_last;
+  int tile_last;
+  float scale[kN];
+  float red[4][kN];           // one value per epilogue warp and activation row
+  int redi[4][kN];
+  float xch[kN * 64];         // gate/up exchange: [m][feature of the tile]
+};
+
+constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + 1024;   // + alignment slack
+
+}  // namespace umma
+}  // namespace ps
