@@ -674,55 +674,78 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   if (warp == 0) {
     if (lane == 0) {   // ---- TMA producer
       const uint32_t bytes = kABytes + kBBytes * (a.lo ? 2 : 1);
-      int i = 0;
-      for (long long u = u0; u < u1; ++u, ++i) {
-        const int stage = i % kStages;
-        if (!mbar_wait(&ctl.empty[stage], ((i / kStages) & 1) ^ 1, abort_flag)) break;
-        int t = (int)(u / a.KB);
-        const int x = (int)(u - (long long)t * a.KB) * kBK;
+      // (tile, k-block) of the running unit, and the tile's matrix and first row, kept
+      // incrementally: the loop has no division
+      int t = (int)(u0 / a.KB), kb = (int)(u0 - (long long)t * a.KB);
+      int mat = 0, row0 = 0;
+      if (a.zip) {
+        row0 = t * 64;
+      } else {
+        int tl = t;
+        while (mat + 1 < a.n_mats && tl >= a.mat_tiles[mat]) { tl -= a.mat_tiles[mat]; ++mat; }
+        row0 = tl * kTile;
+      }
+      const int n_units = (int)(u1 - u0);
+      int stage = 0;
+      uint32_t parity = 1;   // a fresh barrier passes a wait on parity 1
+      for (int i = 0; i < n_units; ++i) {
+        if (!mbar_wait(&ctl.empty[stage], parity, abort_flag)) break;
+        const int x = kb * kBK;
         const uint32_t dst = base + stage * kStageBytes;
         mbar_arrive_expect_tx(&ctl.full[stage], bytes);
         if (a.zip) {
-          tma_load_2d(dst, &tA0, x, t * 64, &ctl.full[stage]);
-          tma_load_2d(dst + kABytes / 2, &tA1, x, t * 64, &ctl.full[stage]);
+          tma_load_2d(dst, &tA0, x, row0, &ctl.full[stage]);
+          tma_load_2d(dst + kABytes / 2, &tA1, x, row0, &ctl.full[stage]);
         } else {
-          int m = 0;
-          while (m + 1 < a.n_mats && t >= a.mat_tiles[m]) { t -= a.mat_tiles[m]; ++m; }
-          const CUtensorMap* map = m == 0 ? &tA0 : (m == 1 ? &tA1 : &tA2);
-          tma_load_2d(dst, map, x, t * kTile, &ctl.full[stage]);
+          const CUtensorMap* map = mat == 0 ? &tA0 : (mat == 1 ? &tA1 : &tA2);
+          tma_load_2d(dst, map, x, row0, &ctl.full[stage]);
         }
         tma_load_2d(dst + kABytes, &tBh, x, 0, &ctl.full[stage]);
         if (a.lo) tma_load_2d(dst + kABytes + kBBytes, &tBl, x, 0, &ctl.full[stage]);
+        if (++stage == kStages) { stage = 0; parity ^= 1; }
+        if (++kb == a.KB) {   // next tile
+          kb = 0;
+          ++t;
+          if (a.zip) {
+            row0 += 64;
+          } else {
+            row0 += kTile;
+            if (row0 >= a.mat_rows[mat] && mat + 1 < a.n_mats) { ++mat; row0 = 0; }
+          }
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {   // ---- MMA issuer
-      int i = 0, seg = 0;
-      long long u = u0;
+      int seg = 0, stage = 0;
+      uint32_t parity = 0;
+      const int t0 = (int)(u0 / a.KB);
+      int left = (int)(u1 - u0);                              // units still to do
+      int in_tile = a.KB - (int)(u0 - (long long)t0 * a.KB);  // units to the end of the running tile
       bool alive = true;
-      while (u < u1 && alive) {
-        const long long t = u / a.KB;
-        const long long seg_end = min(u1, (t + 1) * a.KB);
+      const uint32_t id = a.lo ? idesc(2 * kN) : idesc(kN);   // hi and lo planes as one N = 32 operand
+      while (left > 0 && alive) {
+        const int n_seg = min(left, in_tile);
         const int buf = seg & 1;
         if (!mbar_wait(&ctl.acc_empty[buf], ((seg >> 1) & 1) ^ 1, abort_flag)) break;
         fence_after_sync();
-        const uint32_t d = tmem + buf * kN;
+        const uint32_t d = tmem + buf * kAccCols;
         uint32_t acc = 0;
-        for (; u < seg_end; ++u, ++i) {
-          const int stage = i % kStages;
-          if (!mbar_wait(&ctl.full[stage], (i / kStages) & 1, abort_flag)) { alive = false; break; }
+        for (int j = 0; j < n_seg; ++j) {
+          if (!mbar_wait(&ctl.full[stage], parity, abort_flag)) { alive = false; break; }
           fence_after_sync();
           const uint32_t sa = base + stage * kStageBytes;
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k) {
-            const uint64_t da = smem_desc(sa + k * 32);
-            mma_f16(d, da, smem_desc(sa + kABytes + k * 32), acc);
+            mma_f16(d, smem_desc(sa + k * 32), smem_desc(sa + kABytes + k * 32), id, acc);
             acc = 1;
-            if (a.lo) mma_f16(d, da, smem_desc(sa + kABytes + kBBytes + k * 32), 1);
           }
           mma_commit(&ctl.empty[stage]);
+          if (++stage == kStages) { stage = 0; parity ^= 1; }
         }
         if (alive) mma_commit(&ctl.acc_full[buf]);
+        left -= n_seg;
+        in_tile = a.KB;
         ++seg;
       }
     }
@@ -752,7 +775,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       if (epi_any(!mbar_wait(&ctl.acc_full[buf], (seg >> 1) & 1, abort_flag))) break;
       fence_after_sync();
       float v[16];
-      tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + buf * kN, v);
+      tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + buf * kAccCols, v);
+      if (a.lo) {
+        float vl[16];
+        tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + buf * kAccCols + kN, vl);
+#pragma unroll
+        for (int m = 0; m < 16; ++m) v[m] += vl[m];
+      }
       fence_before_sync();
       mbar_arrive(&ctl.acc_empty[buf]);
       if (whole) {
@@ -1188,3 +1217,4 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
 }
 
 }  // namespace ps
+

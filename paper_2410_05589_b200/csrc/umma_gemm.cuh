@@ -2,9 +2,11 @@
 //   Y[m][n] = sum_k A[m][k] * W[n][k],  M = B*(k+1) <= 16 rows, W row-major bf16, fp32 sums.
 //
 // The weights are the M side of tcgen05.mma (128 weight rows per instruction), the activation
-// rows its N side (N = 16), so one instruction retires a 128 x 16 weight block (4 KB) against
-// one activation plane; the accumulator (128 lanes x 16 columns of fp32) lives in tensor
-// memory.  Operands reach shared memory by tiled TMA loads (cp.async.bulk.tensor.2d) in the
+// rows its N side: the 16 rows of the hi plane and the 16 rows of the lo plane sit one after the
+// other in shared memory and form one N = 32 operand, so one instruction retires a 128 x 16
+// weight block (4 KB) against both planes (measured: the cost of these small MMAs is per
+// instruction, not per column).  The accumulator (128 lanes x 32 columns of fp32) lives in
+// tensor memory; the epilogue adds the two halves.  Operands reach shared memory by tiled TMA loads (cp.async.bulk.tensor.2d) in the
 // 128-byte-swizzled K-major layout the instruction reads: per stage one 128-row x 64-column
 // box of weights (16 KB) and the matching 16 x 64 boxes of the activation planes.
 //
@@ -46,11 +48,13 @@ constexpr int kStageBytes = kABytes + 2 * kBBytes;
 constexpr int kStages = 10;
 constexpr int kThreads = 192;
 constexpr int kEpiThreads = 128;
-constexpr int kTmemCols = 32;                     // two accumulators of kN columns
+constexpr int kAccCols = 2 * kN;                  // accumulator columns: hi products, lo products
+constexpr int kTmemCols = 2 * kAccCols;           // two accumulators
 // Instruction descriptor of kind::f16: fp32 accumulator, bf16 x bf16, both operands K-major,
 // N / 8 in bits [17,23), M / 16 in bits [24,29).
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kN >> 3) << 17) |
-                            ((uint32_t)(kTile >> 4) << 24);
+constexpr uint32_t idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+}
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 // Shared-memory matrix descriptor, K-major, 128-byte swizzle: rows of 128 bytes, groups of 8
@@ -67,12 +71,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
-__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc_,
+                                        uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(kIdesc), "r"(accumulate)
+      "l"(a_desc), "l"(b_desc), "r"(idesc_), "r"(accumulate)
       : "memory");
 }
 // Arrives on the barrier once every MMA issued so far by this thread has completed.
