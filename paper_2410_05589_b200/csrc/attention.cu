@@ -312,16 +312,20 @@ __global__ void __launch_bounds__(kAttnThreads, NB == 1 ? 3 : 2) k_attn_mma(
   // ---- the last split of this (sequence, head) to finish merges all of them and writes the
   // attention output as hi/lo bf16 planes [row][n_heads * D] (no block waits for another)
   __shared__ int s_last;
-  __threadfence();
   __syncthreads();
   if (tid == 0) {
+    // one thread publishes the block's partial (the barrier ordered the other threads' stores
+    // before this fence) and, if it came last, acquires the other blocks'
+    __threadfence();
     const unsigned tk = atomicAdd(&tickets[b * n_heads + h], 1u);
     s_last = (tk == (unsigned)n_split - 1u);
-    if (s_last) tickets[b * n_heads + h] = 0u;
+    if (s_last) {
+      tickets[b * n_heads + h] = 0u;
+      __threadfence();
+    }
   }
   __syncthreads();
   if (s_last) {
-    __threadfence();
     for (int idx = tid; idx < R * D; idx += kAttnThreads) {
       const int j = idx / D, d = idx - j * D;
       const size_t rec0 = ((size_t)(m0 + j) * n_heads + h) * n_split;

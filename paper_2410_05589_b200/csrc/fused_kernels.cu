@@ -479,9 +479,33 @@ struct UArgs {
 };
 
 // CTA that owns unit u when CTA c owns [U c / G, U (c+1) / G).
-__device__ __forceinline__ int unit_owner(long long u, long long U, int G) {
-  return (int)(((u + 1) * G - 1) / U);
+// (Unit counts are small enough for 32-bit arithmetic: the launcher checks U * (G + 1) < 2^31.)
+__device__ __forceinline__ int unit_owner(int u, int U, int G) {
+  return (int)(((unsigned)(u + 1) * (unsigned)G - 1u) / (unsigned)U);
 }
+__device__ __forceinline__ int unit_begin(int c, int U, int G) {
+  return (int)((unsigned)U * (unsigned)c / (unsigned)G);
+}
+
+// The tiles a CTA's unit range [u0, u1) touches, in the order the CTA works through them.  A
+// range that ends inside a tile starts with that tail: the tiles a CTA shares with its
+// neighbours are then reduced while the rest of its range still streams, and the last thing it
+// does is a tile of its own.
+struct Segs {
+  int u0, u1, KB, t0, n, tail_first;
+  __device__ Segs(int u0_, int u1_, int KB_) : u0(u0_), u1(u1_), KB(KB_) {
+    t0 = u0 / KB;
+    n = u1 > u0 ? (u1 - 1) / KB - t0 + 1 : 0;
+    tail_first = n > 1 && (u1 % KB) != 0;
+  }
+  // i-th segment in working order: units [b, e) of tile t
+  __device__ void get(int i, int& t, int& b, int& e) const {
+    const int k = tail_first ? (i == 0 ? n - 1 : i - 1) : i;
+    t = t0 + k;
+    b = max(u0, t * KB);
+    e = min(u1, (t + 1) * KB);
+  }
+};
 
 // Feature of accumulator row r of tile t; valid = false for rows past the end of a matrix.
 __device__ __forceinline__ int tile_feature(const UArgs& a, int t, int r, bool& valid) {
@@ -667,71 +691,58 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   fence_after_sync();
   const uint32_t tmem = *(volatile uint32_t*)&ctl.tmem_base;
 
-  const long long U = (long long)a.n_tiles * a.KB;
-  const long long u0 = U * blockIdx.x / gridDim.x, u1 = U * (blockIdx.x + 1) / gridDim.x;
+  const int G = gridDim.x, U = a.n_tiles * a.KB;
+  const int u0 = unit_begin(blockIdx.x, U, G), u1 = unit_begin(blockIdx.x + 1, U, G);
+  const Segs segs(u0, u1, a.KB);
   volatile int* abort_flag = &ctl.abort_flag;
 
   if (warp == 0) {
     if (lane == 0) {   // ---- TMA producer
       const uint32_t bytes = kABytes + kBBytes * (a.lo ? 2 : 1);
-      // (tile, k-block) of the running unit, and the tile's matrix and first row, kept
-      // incrementally: the loop has no division
-      int t = (int)(u0 / a.KB), kb = (int)(u0 - (long long)t * a.KB);
-      int mat = 0, row0 = 0;
-      if (a.zip) {
-        row0 = t * 64;
-      } else {
-        int tl = t;
-        while (mat + 1 < a.n_mats && tl >= a.mat_tiles[mat]) { tl -= a.mat_tiles[mat]; ++mat; }
-        row0 = tl * kTile;
-      }
-      const int n_units = (int)(u1 - u0);
       int stage = 0;
       uint32_t parity = 1;   // a fresh barrier passes a wait on parity 1
-      for (int i = 0; i < n_units; ++i) {
-        if (!mbar_wait(&ctl.empty[stage], parity, abort_flag)) break;
-        const int x = kb * kBK;
-        const uint32_t dst = base + stage * kStageBytes;
-        mbar_arrive_expect_tx(&ctl.full[stage], bytes);
-        if (a.zip) {
-          tma_load_2d(dst, &tA0, x, row0, &ctl.full[stage]);
-          tma_load_2d(dst + kABytes / 2, &tA1, x, row0, &ctl.full[stage]);
-        } else {
-          const CUtensorMap* map = mat == 0 ? &tA0 : (mat == 1 ? &tA1 : &tA2);
-          tma_load_2d(dst, map, x, row0, &ctl.full[stage]);
+      bool alive = true;
+      for (int si = 0; si < segs.n && alive; ++si) {
+        int t, b, e;
+        segs.get(si, t, b, e);
+        int mat = 0, row0 = t * 64;   // the tile's matrix and first row
+        if (!a.zip) {
+          int tl = t;
+          while (mat + 1 < a.n_mats && tl >= a.mat_tiles[mat]) { tl -= a.mat_tiles[mat]; ++mat; }
+          row0 = tl * kTile;
         }
-        tma_load_2d(dst + kABytes, &tBh, x, 0, &ctl.full[stage]);
-        if (a.lo) tma_load_2d(dst + kABytes + kBBytes, &tBl, x, 0, &ctl.full[stage]);
-        if (++stage == kStages) { stage = 0; parity ^= 1; }
-        if (++kb == a.KB) {   // next tile
-          kb = 0;
-          ++t;
+        const CUtensorMap* map = mat == 0 ? &tA0 : (mat == 1 ? &tA1 : &tA2);
+        for (int x = (b - t * a.KB) * kBK, x_end = (e - t * a.KB) * kBK; x < x_end; x += kBK) {
+          if (!mbar_wait(&ctl.empty[stage], parity, abort_flag)) { alive = false; break; }
+          const uint32_t dst = base + stage * kStageBytes;
+          mbar_arrive_expect_tx(&ctl.full[stage], bytes);
           if (a.zip) {
-            row0 += 64;
+            tma_load_2d(dst, &tA0, x, row0, &ctl.full[stage]);
+            tma_load_2d(dst + kABytes / 2, &tA1, x, row0, &ctl.full[stage]);
           } else {
-            row0 += kTile;
-            if (row0 >= a.mat_rows[mat] && mat + 1 < a.n_mats) { ++mat; row0 = 0; }
+            tma_load_2d(dst, map, x, row0, &ctl.full[stage]);
           }
+          tma_load_2d(dst + kABytes, &tBh, x, 0, &ctl.full[stage]);
+          if (a.lo) tma_load_2d(dst + kABytes + kBBytes, &tBl, x, 0, &ctl.full[stage]);
+          if (++stage == kStages) { stage = 0; parity ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {   // ---- MMA issuer
-      int seg = 0, stage = 0;
+      int stage = 0;
       uint32_t parity = 0;
-      const int t0 = (int)(u0 / a.KB);
-      int left = (int)(u1 - u0);                              // units still to do
-      int in_tile = a.KB - (int)(u0 - (long long)t0 * a.KB);  // units to the end of the running tile
       bool alive = true;
       const uint32_t id = a.lo ? idesc(2 * kN) : idesc(kN);   // hi and lo planes as one N = 32 operand
-      while (left > 0 && alive) {
-        const int n_seg = min(left, in_tile);
-        const int buf = seg & 1;
-        if (!mbar_wait(&ctl.acc_empty[buf], ((seg >> 1) & 1) ^ 1, abort_flag)) break;
+      for (int si = 0; si < segs.n && alive; ++si) {
+        int t, b, e;
+        segs.get(si, t, b, e);
+        const int buf = si & 1;
+        if (!mbar_wait(&ctl.acc_empty[buf], ((si >> 1) & 1) ^ 1, abort_flag)) break;
         fence_after_sync();
         const uint32_t d = tmem + buf * kAccCols;
         uint32_t acc = 0;
-        for (int j = 0; j < n_seg; ++j) {
+        for (int j = b; j < e; ++j) {
           if (!mbar_wait(&ctl.full[stage], parity, abort_flag)) { alive = false; break; }
           fence_after_sync();
           const uint32_t sa = base + stage * kStageBytes;
@@ -744,9 +755,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
           if (++stage == kStages) { stage = 0; parity ^= 1; }
         }
         if (alive) mma_commit(&ctl.acc_full[buf]);
-        left -= n_seg;
-        in_tile = a.KB;
-        ++seg;
       }
     }
   } else {
@@ -763,13 +771,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       if (lane == 0) ctl.scale[m] = sc;
     }
     epi_sync();
-    int seg = 0;
-    long long u = u0;
-    while (u < u1) {
-      const int t = (int)(u / a.KB);
-      const long long t_begin = (long long)t * a.KB, t_end = t_begin + a.KB;
-      const long long seg_end = min(u1, t_end);
-      const bool whole = (u == t_begin) && (seg_end == t_end);
+    for (int seg = 0; seg < segs.n; ++seg) {
+      int t, sb, se;
+      segs.get(seg, t, sb, se);
+      const int t_begin = t * a.KB, t_end = t_begin + a.KB;
+      const bool whole = se - sb == a.KB;
       const int buf = seg & 1;
       // all four warps take the same decision although each thread waits for itself
       if (epi_any(!mbar_wait(&ctl.acc_full[buf], (seg >> 1) & 1, abort_flag))) break;
@@ -788,32 +794,37 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         tile_epilogue<EPI>(a, ctl, t, r, q, lane, v);
       } else {
         // partial tile: slot 0 = this CTA's first segment, slot 1 = its last one
-        const int slot = (t == (int)(u0 / a.KB)) ? 0 : 1;
+        const int slot = (t == segs.t0) ? 0 : 1;
         float* P = a.partials + ((size_t)blockIdx.x * 2 + slot) * 16 * 128;
 #pragma unroll
         for (int m = 0; m < 16; ++m)
           if (m < a.M) P[m * 128 + r] = v[m];
-        __threadfence();
         epi_sync();
-        const int c_first = unit_owner(t_begin, U, gridDim.x), c_last = unit_owner(t_end - 1, U, gridDim.x);
+        const int c_first = unit_owner(t_begin, U, G), c_last = unit_owner(t_end - 1, U, G);
         if (et == 0) {
+          // one thread publishes the block's partial (the barrier above ordered the other
+          // threads' stores before this fence) and, if it came last, acquires the others'
           int n_contrib = 0;   // CTAs between the owners of the tile's ends that hold any unit
-          for (int c = c_first; c <= c_last; ++c) n_contrib += (U * c / gridDim.x) < (U * (c + 1) / gridDim.x);
+          for (int c = c_first; c <= c_last; ++c) n_contrib += unit_begin(c, U, G) < unit_begin(c + 1, U, G);
+          __threadfence();
           const unsigned old = atomicAdd(&a.tile_tickets[t], 1u);
           const int last = old == (unsigned)(n_contrib - 1);
-          if (last) a.tile_tickets[t] = 0u;
+          if (last) {
+            a.tile_tickets[t] = 0u;
+            __threadfence();
+          }
           ctl.tile_last = last;
         }
         epi_sync();
         const bool last = ctl.tile_last != 0;
         epi_sync();   // everyone has read the flag before a later segment rewrites it
         if (last) {
-          __threadfence();
 #pragma unroll
           for (int m = 0; m < 16; ++m) v[m] = 0.f;
           for (int c = c_first; c <= c_last; ++c) {   // fixed order: the sum does not depend on who is last
-            if (U * c / gridDim.x >= U * (c + 1) / gridDim.x) continue;   // a CTA without units
-            const int c_tile0 = (int)((U * c / gridDim.x) / a.KB);
+            const int cb = unit_begin(c, U, G);
+            if (cb >= unit_begin(c + 1, U, G)) continue;   // a CTA without units
+            const int c_tile0 = cb / a.KB;
             const int sl = (c == c_first && c_tile0 != t) ? 1 : 0;
             const float* Pc = a.partials + ((size_t)c * 2 + sl) * 16 * 128;
 #pragma unroll
@@ -823,8 +834,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
           tile_epilogue<EPI>(a, ctl, t, r, q, lane, v);
         }
       }
-      u = seg_end;
-      ++seg;
     }
     fence_before_sync();
   }
@@ -836,19 +845,19 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       __threadfence();
       const unsigned tk = atomicAdd(a.ticket, 1u);
       ctl.is_last = (tk == gridDim.x - 1);
+      if (ctl.is_last) __threadfence();
     }
     __syncthreads();
     if (ctl.is_last && warp >= 2 && !ctl.abort_flag) {
-      __threadfence();
-      const int G = a.n_tiles;
+      const int Gt = a.n_tiles;
       for (int m = warp - 2; m < a.M; m += 4) {
         const LmPart* P = a.parts + m;
         float mx = -FLT_MAX;
-        for (int c = lane; c < G; c += 32) mx = fmaxf(mx, P[(size_t)c * a.M].vmax);
+        for (int c = lane; c < Gt; c += 32) mx = fmaxf(mx, P[(size_t)c * a.M].vmax);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         float se = 0.f;
-        for (int c = lane; c < G; c += 32) se += P[(size_t)c * a.M].sumexp * __expf(P[(size_t)c * a.M].vmax - mx);
+        for (int c = lane; c < Gt; c += 32) se += P[(size_t)c * a.M].sumexp * __expf(P[(size_t)c * a.M].vmax - mx);
         se = warp_sum(se);
         if (lane == 0) {
           if (a.row_max) a.row_max[m] = mx;
@@ -857,7 +866,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         float pv = FLT_MAX; int pi = -1;
         for (int tn = 0; tn < a.top_n; ++tn) {
           float bv = -FLT_MAX; int bi = 0x7fffffff;
-          for (int e = lane; e < G * a.top_n; e += 32) {
+          for (int e = lane; e < Gt * a.top_n; e += 32) {
             const int c = e / a.top_n, k = e - c * a.top_n;
             const float xv = P[(size_t)c * a.M].top_v[k]; const int id = P[(size_t)c * a.M].top_i[k];
             if (id == 0x7fffffff) continue;
@@ -990,6 +999,7 @@ ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, c
       a.n_tiles += a.mat_tiles[m];
     }
   }
+  if ((long long)a.n_tiles * a.KB * (c->n_sm + 1) >= (1ll << 31)) return fail(c, PS_ERR_UNSUPPORTED, "too many GEMM units");
   a.partials = f.partials; a.tile_tickets = f.tile_tickets; a.status = c->dev_status;
   auto kern = k_umma_gemm<EPI>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, umma::kSmemBytes);
@@ -1217,4 +1227,5 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
 }
 
 }  // namespace ps
+
 
