@@ -111,7 +111,9 @@ __global__ void __launch_bounds__(kAttnThreads, NB == 1 ? 3 : 2) k_attn_mma(
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  if (t_begin < t_end) stage(t_begin, min(tile, t_end - t_begin));
+  pdl_launch_dependents();
+  if (t_begin < t_end) stage(t_begin, min(tile, t_end - t_begin));   // the cache is older than the launch before
+  pdl_wait();   // q, k and v of the new rows come from the kernel before this one
 
   // rotation table of the R new positions, then q: rotated, scaled, split into hi/lo planes
   for (int idx = tid; idx < R * HALF; idx += kAttnThreads) {
@@ -394,11 +396,11 @@ static ps_status launch_attn_t(ps_ctx* c, const SeqMap& sm, int B, int max_len, 
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
   if (e != cudaSuccess) return cuda_check(c, e, "attention smem attribute");
   typedef const __nv_bfloat16* BP;
-  kern<<<dim3(g.n_heads, n_split, B), kAttnThreads, bytes, st>>>(
-      sm, qkv, Hq + 2 * Hkv, Hq, Hkv, (BP)c->kcache, (BP)c->vcache, g.n_heads, g.n_kv_heads, g.max_ctx,
-      c->rope_inv_freq, n_split, tile, att_ml, att_o, tickets, out_hi, out_lo);
+  e = launch_after(kern, dim3(g.n_heads, n_split, B), dim3(kAttnThreads), bytes, st, !c->prof, sm, qkv,
+                   Hq + 2 * Hkv, Hq, Hkv, (BP)c->kcache, (BP)c->vcache, g.n_heads, g.n_kv_heads, g.max_ctx,
+                   (const double*)c->rope_inv_freq, n_split, tile, att_ml, att_o, tickets, out_hi, out_lo);
   c->launches++;
-  return cuda_check(c, cudaGetLastError(), "k_attn_mma");
+  return cuda_check(c, e, "k_attn_mma");
 }
 
 ps_status launch_attn_split(ps_ctx* c, const SeqMap& sm, int B, const float* qkv, float* att_ml,

@@ -507,6 +507,32 @@ struct Segs {
   }
 };
 
+// Walks a CTA's units in working order: the running tile t, its k-block kb, and the tile's
+// matrix and first row.
+struct UnitWalk {
+  int si, t, kb, kb_end, mat, row0;
+  __device__ void enter(const Segs& s, const UArgs& a) {
+    int b, e;
+    s.get(si, t, b, e);
+    kb = b - t * a.KB;
+    kb_end = e - t * a.KB;
+    mat = 0;
+    row0 = t * 64;
+    if (!a.zip) {
+      int tl = t;
+      while (mat + 1 < a.n_mats && tl >= a.mat_tiles[mat]) { tl -= a.mat_tiles[mat]; ++mat; }
+      row0 = tl * umma::kTile;
+    }
+  }
+  __device__ void start(const Segs& s, const UArgs& a) {
+    si = 0;
+    if (s.n > 0) enter(s, a);
+  }
+  __device__ void next(const Segs& s, const UArgs& a) {
+    if (++kb == kb_end && ++si < s.n) enter(s, a);
+  }
+};
+
 // Feature of accumulator row r of tile t; valid = false for rows past the end of a matrix.
 __device__ __forceinline__ int tile_feature(const UArgs& a, int t, int r, bool& valid) {
   if (a.zip) {
@@ -679,6 +705,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
     for (int i = 0; i < 2; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], kEpiThreads); }
     ctl.abort_flag = 0; ctl.is_last = 0; ctl.tile_last = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    pdl_launch_dependents();
   }
   if (warp == 1) {   // tensor memory for two accumulators
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
@@ -699,33 +726,41 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   if (warp == 0) {
     if (lane == 0) {   // ---- TMA producer
       const uint32_t bytes = kABytes + kBBytes * (a.lo ? 2 : 1);
+      // The weights do not depend on the kernel before this one, its activations do: the
+      // weight boxes of the first kStages units are requested first, then the thread waits for
+      // that kernel and adds their activation boxes.
+      const int n_units = u1 - u0, n_early = min(kStages, n_units);
+      UnitWalk w;
+      auto load_a = [&](const UnitWalk& uw, int st_i) {
+        const uint32_t dst = base + st_i * kStageBytes;
+        const int x = uw.kb * kBK;
+        mbar_arrive_expect_tx(&ctl.full[st_i], bytes);
+        if (a.zip) {
+          tma_load_2d(dst, &tA0, x, uw.row0, &ctl.full[st_i]);
+          tma_load_2d(dst + kABytes / 2, &tA1, x, uw.row0, &ctl.full[st_i]);
+        } else {
+          tma_load_2d(dst, uw.mat == 0 ? &tA0 : (uw.mat == 1 ? &tA1 : &tA2), x, uw.row0, &ctl.full[st_i]);
+        }
+      };
+      auto load_b = [&](const UnitWalk& uw, int st_i) {
+        const uint32_t dst = base + st_i * kStageBytes + kABytes;
+        const int x = uw.kb * kBK;
+        tma_load_2d(dst, &tBh, x, 0, &ctl.full[st_i]);
+        if (a.lo) tma_load_2d(dst + kBBytes, &tBl, x, 0, &ctl.full[st_i]);
+      };
+      w.start(segs, a);
+      for (int i = 0; i < n_early; ++i) { load_a(w, i); w.next(segs, a); }
+      pdl_wait();
+      w.start(segs, a);
+      for (int i = 0; i < n_early; ++i) { load_b(w, i); w.next(segs, a); }
       int stage = 0;
-      uint32_t parity = 1;   // a fresh barrier passes a wait on parity 1
-      bool alive = true;
-      for (int si = 0; si < segs.n && alive; ++si) {
-        int t, b, e;
-        segs.get(si, t, b, e);
-        int mat = 0, row0 = t * 64;   // the tile's matrix and first row
-        if (!a.zip) {
-          int tl = t;
-          while (mat + 1 < a.n_mats && tl >= a.mat_tiles[mat]) { tl -= a.mat_tiles[mat]; ++mat; }
-          row0 = tl * kTile;
-        }
-        const CUtensorMap* map = mat == 0 ? &tA0 : (mat == 1 ? &tA1 : &tA2);
-        for (int x = (b - t * a.KB) * kBK, x_end = (e - t * a.KB) * kBK; x < x_end; x += kBK) {
-          if (!mbar_wait(&ctl.empty[stage], parity, abort_flag)) { alive = false; break; }
-          const uint32_t dst = base + stage * kStageBytes;
-          mbar_arrive_expect_tx(&ctl.full[stage], bytes);
-          if (a.zip) {
-            tma_load_2d(dst, &tA0, x, row0, &ctl.full[stage]);
-            tma_load_2d(dst + kABytes / 2, &tA1, x, row0, &ctl.full[stage]);
-          } else {
-            tma_load_2d(dst, map, x, row0, &ctl.full[stage]);
-          }
-          tma_load_2d(dst + kABytes, &tBh, x, 0, &ctl.full[stage]);
-          if (a.lo) tma_load_2d(dst + kABytes + kBBytes, &tBl, x, 0, &ctl.full[stage]);
-          if (++stage == kStages) { stage = 0; parity ^= 1; }
-        }
+      uint32_t parity = 0;   // second use of a stage: its first release
+      for (int i = n_early; i < n_units; ++i) {
+        if (!mbar_wait(&ctl.empty[stage], parity, abort_flag)) break;
+        load_a(w, stage);
+        load_b(w, stage);
+        w.next(segs, a);
+        if (++stage == kStages) { stage = 0; parity ^= 1; }
       }
     }
   } else if (warp == 1) {
@@ -760,6 +795,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   } else {
     // ---- epilogue warps: accumulator row r = 32 q + lane
     const int q = warp & 3, r = 32 * q + lane, et = r;
+    pdl_wait();   // everything below reads or writes what the kernel before this one touches
     for (int m = warp - 2; m < a.M; m += 4) {   // RMSNorm row scales of the input
       float sc = 1.f;
       if (a.ssq_in) {
@@ -904,6 +940,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
 __global__ void k_gather_x(const __nv_bfloat16* __restrict__ embed, const __nv_bfloat16* __restrict__ mask_embed,
                            const __nv_bfloat16* __restrict__ mask_feat, const __nv_bfloat16* __restrict__ hidden,
                            const int* __restrict__ tokens, int H, int V, int R, __nv_bfloat16* __restrict__ xin) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int m = blockIdx.x, b = m / R, j = m - b * R;
   const __nv_bfloat16 *e, *f;
   if (j == 0) {
@@ -1004,9 +1042,9 @@ ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, c
   auto kern = k_umma_gemm<EPI>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, umma::kSmemBytes);
   if (e != cudaSuccess) return cuda_check(c, e, "umma smem attribute");
-  kern<<<c->n_sm, umma::kThreads, umma::kSmemBytes, st>>>(a0, a1, a2, bh, bl, a);
+  e = launch_after(kern, dim3(c->n_sm), dim3(umma::kThreads), umma::kSmemBytes, st, !c->prof, a0, a1, a2, bh, bl, a);
   c->launches++;
-  return cuda_check(c, cudaGetLastError(), "k_umma_gemm");
+  return cuda_check(c, e, "k_umma_gemm");
 }
 
 ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B, const void* hidden_last,
@@ -1021,9 +1059,10 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
   const int tiles_h = (H + umma::kTile - 1) / umma::kTile;
   ps_status s;
   prof_mark(c, st, "begin");
-  k_gather_x<<<M, 256, 0, st>>>((BP)w.embed, (BP)w.mask_embed, (BP)w.mask_feat, (BP)hidden_last, token_last, H, V,
-                                R, f.xin);
+  cudaError_t ge = launch_after(k_gather_x, dim3(M), dim3(256), 0, st, !c->prof, (BP)w.embed, (BP)w.mask_embed,
+                                (BP)w.mask_feat, (BP)hidden_last, token_last, H, V, R, f.xin);
   c->launches++;
+  if (ge != cudaSuccess) return cuda_check(c, ge, "k_gather_x");
   {  // S1 fc: x0 = W_fc [e ; f] (+ b)
     UArgs a{};
     a.N = H; a.K = 2 * H; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 0;

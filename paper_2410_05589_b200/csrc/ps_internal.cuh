@@ -41,6 +41,28 @@ __device__ __forceinline__ void seq_of_row(const SeqMap& s, int m, int& b, int& 
   j = g - s.row_off[lo];
 }
 
+// Programmatic dependent launch.  A kernel launched with `launch_after` (pdl = true) may start
+// while the kernel before it in the stream still runs; it must call pdl_wait() before it reads
+// or writes anything that kernel touches (a no-op for a plain launch), and calls
+// pdl_launch_dependents() early so that its own successor may be scheduled behind it.
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+cudaError_t launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                         Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // Device status word values (bit flags).
 constexpr int kStatNonfinite = 1;
 constexpr int kStatTimeout = 2;
