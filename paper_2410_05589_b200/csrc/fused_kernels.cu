@@ -30,8 +30,9 @@ enum Epi { EPI_STORE = 0, EPI_SWIGLU = 1, EPI_LMHEAD = 2 };
 constexpr int kMaxM = 16;
 constexpr int kTopMax = PS_MAX_TOP_N;
 
-struct LmPart {  // softmax / top-n summary of one CTA's vocabulary range for one row
+struct __align__(16) LmPart {  // softmax / top-n summary of one vocabulary range for one row
   float vmax, sumexp;
+  float v0; int i0;          // copy of top_v[0], top_i[0]: the first 16 bytes decide a top-1 merge
   float top_v[kTopMax];
   int top_i[kTopMax];
 };
@@ -458,6 +459,8 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
 // =============================================================================================
 // Tensor-core path (tcgen05 + tiled TMA), see umma_gemm.cuh
 // =============================================================================================
+__device__ unsigned long long g_tr[1024];
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); return g; }
 struct UArgs {
   int N, K, M;
   int n_tiles, KB;         // tiles of 128 weight rows (64 features when zipped), k-blocks of 64
@@ -550,140 +553,115 @@ __device__ __forceinline__ int tile_feature(const UArgs& a, int t, int r, bool& 
   return a.mat_off[m] + local;
 }
 
-// Epilogue of one finished tile; called by the 128 epilogue threads with v[m] = the tile's sums
-// for accumulator row r (= 32 * q + lane) and activation row m.
+// Epilogue of one finished tile; called by the 128 epilogue threads after each has put its
+// accumulator row r (= 32 * q + lane) into ctl.acc[m * 128 + r], m = activation row.  The loops
+// over m are rolled on purpose: this code runs once or twice per CTA, so what it costs is the
+// fetch of its instructions, not their execution.
 template <int EPI>
-__device__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane, float (&v)[16]) {
+__device__ __noinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane) {
   using namespace umma;
-  const int et = 32 * q + lane;   // == r
+  const int et = r;
   bool valid;
   const int n = tile_feature(a, t, r, valid);
+  const float* acc = ctl.acc + r;
   if (EPI == EPI_STORE) {
-    float sq[16];
-#pragma unroll
-    for (int m = 0; m < 16; ++m) {
-      sq[m] = 0.f;
-      if (m < a.M && valid) {
-        float x = v[m] * ctl.scale[m];
-        if (a.bias) x += __bfloat162float(a.bias[n]);
+    const float bias = (a.bias && valid) ? __bfloat162float(a.bias[n]) : 0.f;
+    const float gain = (a.gain_next && valid) ? __bfloat162float(a.gain_next[n]) : 1.f;
+#pragma unroll 1
+    for (int m = 0; m < a.M; ++m) {
+      float sq = 0.f;
+      if (valid) {
+        float x = acc[m * 128] * ctl.scale[m] + bias;
         if (a.res) x += a.res[(size_t)m * a.ldr + n];
         a.out[(size_t)m * a.ldo + n] = x;
-        sq[m] = x * x;
-        if (a.out_hi) {
-          const float gv = a.gain_next ? x * __bfloat162float(a.gain_next[n]) : x;
-          split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, gv);
-        }
+        sq = x * x;
+        if (a.out_hi)
+          split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, x * gain);
+      }
+      if (a.ssq_out) {
+        sq = warp_sum(sq);
+        if (lane == 0) ctl.red[q][m] = sq;
       }
     }
     if (a.ssq_out) {
-#pragma unroll
-      for (int m = 0; m < 16; ++m) {
-        if (m < a.M) {
-          const float s = warp_sum(sq[m]);
-          if (lane == 0) ctl.red[q][m] = s;
-        }
-      }
       epi_sync();
       if (et < a.M) a.ssq_out[(size_t)t * a.M + et] = (ctl.red[0][et] + ctl.red[1][et]) + (ctl.red[2][et] + ctl.red[3][et]);
       epi_sync();
     }
   } else if (EPI == EPI_SWIGLU) {
     if (r >= 64) {
-#pragma unroll
-      for (int m = 0; m < 16; ++m)
-        if (m < a.M) ctl.xch[m * 64 + (r - 64)] = v[m] * ctl.scale[m];
+#pragma unroll 1
+      for (int m = 0; m < a.M; ++m) ctl.xch[m * 64 + (r - 64)] = acc[m * 128] * ctl.scale[m];
     }
     epi_sync();
     if (r < 64 && valid) {
-#pragma unroll
-      for (int m = 0; m < 16; ++m) {
-        if (m < a.M) {
-          const float gv = v[m] * ctl.scale[m], uv = ctl.xch[m * 64 + r];
-          const float act = gv / (1.f + __expf(-gv)) * uv;
-          if (a.out) a.out[(size_t)m * a.ldo + n] = act;
-          split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, act);
-        }
+#pragma unroll 1
+      for (int m = 0; m < a.M; ++m) {
+        const float gv = acc[m * 128] * ctl.scale[m], uv = ctl.xch[m * 64 + r];
+        const float act = gv / (1.f + __expf(-gv)) * uv;
+        if (a.out) a.out[(size_t)m * a.ldo + n] = act;
+        split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, act);
       }
     }
     epi_sync();
-  } else {  // EPI_LMHEAD
-    float x[16], bmax[16];
+  } else {  // EPI_LMHEAD: logits, and the tile's softmax / top-n summary per row
+#pragma unroll 1
+    for (int m = 0; m < a.M; ++m) {
+      const float x = acc[m * 128] * ctl.scale[m];
+      if (valid && a.logits_out) a.logits_out[(size_t)m * a.N + n] = x;
+      float mx = valid ? x : -FLT_MAX;
 #pragma unroll
-    for (int m = 0; m < 16; ++m) {
-      x[m] = v[m] * ctl.scale[m < a.M ? m : 0];
-      if (m < a.M && valid && a.logits_out) a.logits_out[(size_t)m * a.N + n] = x[m];
-    }
-    // block maximum per row
-#pragma unroll
-    for (int m = 0; m < 16; ++m) {
-      if (m < a.M) {
-        float mx = valid ? x[m] : -FLT_MAX;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if (lane == 0) ctl.red[q][m] = mx;
-      }
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      if (lane == 0) ctl.red[q][m] = mx;
     }
     epi_sync();
-#pragma unroll
-    for (int m = 0; m < 16; ++m)
-      bmax[m] = m < a.M ? fmaxf(fmaxf(ctl.red[0][m], ctl.red[1][m]), fmaxf(ctl.red[2][m], ctl.red[3][m])) : 0.f;
-    float my_vmax = 0.f;   // thread et < M reports row et
-    if (et < a.M) my_vmax = fmaxf(fmaxf(ctl.red[0][et], ctl.red[1][et]), fmaxf(ctl.red[2][et], ctl.red[3][et]));
-    epi_sync();
-    // block sum of exponentials per row
-#pragma unroll
-    for (int m = 0; m < 16; ++m) {
-      if (m < a.M) {
-        const float s = warp_sum(valid ? __expf(x[m] - bmax[m]) : 0.f);
-        if (lane == 0) ctl.red[q][m] = s;
-      }
+#pragma unroll 1
+    for (int m = 0; m < a.M; ++m) {
+      const float bmax = fmaxf(fmaxf(ctl.red[0][m], ctl.red[1][m]), fmaxf(ctl.red[2][m], ctl.red[3][m]));
+      const float s = warp_sum(valid ? __expf(acc[m * 128] * ctl.scale[m] - bmax) : 0.f);
+      if (lane == 0) ctl.red2[q][m] = s;
     }
     epi_sync();
     if (et < a.M) {
       LmPart* p = a.parts + (size_t)t * a.M + et;
-      p->vmax = my_vmax;
-      p->sumexp = (ctl.red[0][et] + ctl.red[1][et]) + (ctl.red[2][et] + ctl.red[3][et]);
+      p->vmax = fmaxf(fmaxf(ctl.red[0][et], ctl.red[1][et]), fmaxf(ctl.red[2][et], ctl.red[3][et]));
+      p->sumexp = (ctl.red2[0][et] + ctl.red2[1][et]) + (ctl.red2[2][et] + ctl.red2[3][et]);
     }
-    epi_sync();
     // top-n per row: repeated block arg-max over the values after the previous pick
-    float pv[16]; int pi[16];
-#pragma unroll
-    for (int m = 0; m < 16; ++m) { pv[m] = FLT_MAX; pi[m] = -1; }
+#pragma unroll 1
     for (int tn = 0; tn < a.top_n; ++tn) {
+#pragma unroll 1
+      for (int m = 0; m < a.M; ++m) {
+        const float x = acc[m * 128] * ctl.scale[m];
+        const float pv = tn ? ctl.prev_v[m] : FLT_MAX;
+        const int pi = tn ? ctl.prev_i[m] : -1;
+        const bool after = valid && ((x < pv) || (x == pv && n > pi));
+        float bv = after ? x : -FLT_MAX;
+        int bi = after ? n : 0x7fffffff;
 #pragma unroll
-      for (int m = 0; m < 16; ++m) {
-        if (m < a.M) {
-          const bool after = valid && ((x[m] < pv[m]) || (x[m] == pv[m] && n > pi[m]));
-          float bv = after ? x[m] : -FLT_MAX;
-          int bi = after ? n : 0x7fffffff;
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-          }
-          if (lane == 0) { ctl.red[q][m] = bv; ctl.redi[q][m] = bi; }
+        for (int o = 16; o > 0; o >>= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+          if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
+        if (lane == 0) { ctl.cand_v[q][m] = bv; ctl.cand_i[q][m] = bi; }
       }
       epi_sync();
+      if (et < a.M) {
+        float bv = ctl.cand_v[0][et]; int bi = ctl.cand_i[0][et];
 #pragma unroll
-      for (int m = 0; m < 16; ++m) {
-        if (m < a.M) {
-          float bv = ctl.red[0][m]; int bi = ctl.redi[0][m];
-#pragma unroll
-          for (int w = 1; w < 4; ++w) {
-            const float ov = ctl.red[w][m]; const int oi = ctl.redi[w][m];
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-          }
-          pv[m] = bv; pi[m] = bi;
-          if (et == m) {
-            LmPart* p = a.parts + (size_t)t * a.M + m;
-            p->top_v[tn] = bv; p->top_i[tn] = bi;
-          }
+        for (int w = 1; w < 4; ++w) {
+          const float ov = ctl.cand_v[w][et]; const int oi = ctl.cand_i[w][et];
+          if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
+        ctl.prev_v[et] = bv; ctl.prev_i[et] = bi;
+        LmPart* p = a.parts + (size_t)t * a.M + et;
+        p->top_v[tn] = bv; p->top_i[tn] = bi;
+        if (tn == 0) { p->v0 = bv; p->i0 = bi; }
       }
       epi_sync();
     }
+    epi_sync();   // red / red2 are free again
   }
 }
 
@@ -718,6 +696,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   fence_after_sync();
   const uint32_t tmem = *(volatile uint32_t*)&ctl.tmem_base;
 
+  if (tid == 0) g_tr[blockIdx.x * 4] = gtime();
   const int G = gridDim.x, U = a.n_tiles * a.KB;
   const int u0 = unit_begin(blockIdx.x, U, G), u1 = unit_begin(blockIdx.x + 1, U, G);
   const Segs segs(u0, u1, a.KB);
@@ -827,7 +806,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       fence_before_sync();
       mbar_arrive(&ctl.acc_empty[buf]);
       if (whole) {
-        tile_epilogue<EPI>(a, ctl, t, r, q, lane, v);
+#pragma unroll
+        for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
+        tile_epilogue<EPI>(a, ctl, t, r, q, lane);
       } else {
         // partial tile: slot 0 = this CTA's first segment, slot 1 = its last one
         const int slot = (t == segs.t0) ? 0 : 1;
@@ -867,7 +848,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
             for (int m = 0; m < 16; ++m)
               if (m < a.M) v[m] += __ldcg(Pc + m * 128 + r);
           }
-          tile_epilogue<EPI>(a, ctl, t, r, q, lane, v);
+#pragma unroll
+          for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
+          tile_epilogue<EPI>(a, ctl, t, r, q, lane);
         }
       }
     }
@@ -875,6 +858,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   }
 
   __syncthreads();
+  if (tid == 0) g_tr[blockIdx.x * 4 + 1] = gtime();
   if (EPI == EPI_LMHEAD) {
     // the last CTA to finish merges the per-tile summaries (no CTA waits for another)
     if (tid == 0) {
@@ -884,30 +868,65 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       if (ctl.is_last) __threadfence();
     }
     __syncthreads();
-    if (ctl.is_last && warp >= 2 && !ctl.abort_flag) {
+    if (ctl.is_last && !ctl.abort_flag) {
+      // all six warps, one activation row each; the loops are unrolled so that the loads of
+      // eight tiles are in flight together (they come from L2, written by other SMs)
       const int Gt = a.n_tiles;
-      for (int m = warp - 2; m < a.M; m += 4) {
+      for (int m = warp; m < a.M; m += umma::kThreads / 32) {
         const LmPart* P = a.parts + m;
-        float mx = -FLT_MAX;
-        for (int c = lane; c < Gt; c += 32) mx = fmaxf(mx, P[(size_t)c * a.M].vmax);
+        // 256 tiles per round, 8 per lane, their loads issued together.  The first round also
+        // fetches every tile's best token: the row's arg-max needs nothing else.
+        float mx = -FLT_MAX, se = 0.f;
+        float bv0 = -FLT_MAX; int bi0 = 0x7fffffff;
+        for (int c0 = 0; c0 < Gt; c0 += 256) {
+          float vm[8], sx[8], tv[8]; int ti[8];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        float se = 0.f;
-        for (int c = lane; c < Gt; c += 32) se += P[(size_t)c * a.M].sumexp * __expf(P[(size_t)c * a.M].vmax - mx);
-        se = warp_sum(se);
+          for (int j = 0; j < 8; ++j) {
+            const int c = c0 + lane + 32 * j;
+            float4 hd = make_float4(-FLT_MAX, 0.f, -FLT_MAX, __int_as_float(0x7fffffff));
+            if (c < Gt) hd = __ldcg(reinterpret_cast<const float4*>(&P[(size_t)c * a.M]));
+            vm[j] = hd.x; sx[j] = hd.y; tv[j] = hd.z;
+            ti[j] = a.top_n > 0 ? __float_as_int(hd.w) : 0x7fffffff;
+          }
+          float nm = mx;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            nm = fmaxf(nm, vm[j]);
+            if (ti[j] != 0x7fffffff && (tv[j] > bv0 || (tv[j] == bv0 && ti[j] < bi0))) { bv0 = tv[j]; bi0 = ti[j]; }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) nm = fmaxf(nm, __shfl_xor_sync(0xffffffffu, nm, o));
+          float add = 0.f;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) add += sx[j] * __expf(vm[j] - nm);
+          se = se * __expf(mx - nm) + warp_sum(add);
+          mx = nm;
+        }
         if (lane == 0) {
           if (a.row_max) a.row_max[m] = mx;
           if (a.row_lse) a.row_lse[m] = mx + logf(se);
         }
         float pv = FLT_MAX; int pi = -1;
         for (int tn = 0; tn < a.top_n; ++tn) {
-          float bv = -FLT_MAX; int bi = 0x7fffffff;
-          for (int e = lane; e < Gt * a.top_n; e += 32) {
-            const int c = e / a.top_n, k = e - c * a.top_n;
-            const float xv = P[(size_t)c * a.M].top_v[k]; const int id = P[(size_t)c * a.M].top_i[k];
-            if (id == 0x7fffffff) continue;
-            const bool after = (xv < pv) || (xv == pv && id > pi);
-            if (after && (xv > bv || (xv == bv && id < bi))) { bv = xv; bi = id; }
+          float bv = bv0; int bi = bi0;
+          if (tn > 0) {   // deeper picks: a tile's list is sorted, any of its entries may be next
+            bv = -FLT_MAX; bi = 0x7fffffff;
+            for (int k = 0; k < a.top_n; ++k) {
+              for (int c0 = 0; c0 < Gt; c0 += 256) {
+                float xv[8]; int id[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const int c = c0 + lane + 32 * j;
+                  xv[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_v[k]) : 0.f;
+                  id[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_i[k]) : 0x7fffffff;
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const bool after = id[j] != 0x7fffffff && ((xv[j] < pv) || (xv[j] == pv && id[j] > pi));
+                  if (after && (xv[j] > bv || (xv[j] == bv && id[j] < bi))) { bv = xv[j]; bi = id[j]; }
+                }
+              }
+            }
           }
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
@@ -920,7 +939,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         }
       }
     }
-    if (ctl.is_last && tid == 0) *a.ticket = 0u;
+    if (ctl.is_last && tid == 0) { *a.ticket = 0u; g_tr[602] = gtime() - g_tr[blockIdx.x * 4 + 1]; }
     __syncthreads();
   }
   if (ctl.abort_flag) {
@@ -929,6 +948,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
     if (tid == 0) atomicOr(a.status, kStatTimeout);
     __syncthreads();
   }
+  if (tid == 0) g_tr[blockIdx.x * 4 + 2] = gtime();
   if (warp == 1) {
     fence_after_sync();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -1268,3 +1288,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
 }  // namespace ps
 
 
+
+extern "C" int ps_trace_read(unsigned long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, ps::g_tr, 8192);
+}

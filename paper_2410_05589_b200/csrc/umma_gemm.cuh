@@ -133,8 +133,13 @@ struct Ctl {
   int tile_last;
   float scale[kN];
   float red[4][kN];           // one value per epilogue warp and activation row
-  int redi[4][kN];
+  float red2[4][kN];
+  float cand_v[4][kN];        // top-n candidates per epilogue warp, and the row's previous pick
+  int cand_i[4][kN];
+  float prev_v[kN];
+  int prev_i[kN];
   float xch[kN * 64];         // gate/up exchange: [m][feature of the tile]
+  float acc[kN * 128];        // a tile's sums, [m][accumulator row]: each thread reads back its own
 };
 
 constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + 1024;   // + alignment slack
