@@ -459,8 +459,6 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
 // =============================================================================================
 // Tensor-core path (tcgen05 + tiled TMA), see umma_gemm.cuh
 // =============================================================================================
-__device__ unsigned long long g_tr[1024];
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); return g; }
 struct UArgs {
   int N, K, M;
   int n_tiles, KB;         // tiles of 128 weight rows (64 features when zipped), k-blocks of 64
@@ -558,7 +556,7 @@ __device__ __forceinline__ int tile_feature(const UArgs& a, int t, int r, bool& 
 // over m are rolled on purpose: this code runs once or twice per CTA, so what it costs is the
 // fetch of its instructions, not their execution.
 template <int EPI>
-__device__ __noinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane) {
+__device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane) {
   using namespace umma;
   const int et = r;
   bool valid;
@@ -696,7 +694,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   fence_after_sync();
   const uint32_t tmem = *(volatile uint32_t*)&ctl.tmem_base;
 
-  if (tid == 0) g_tr[blockIdx.x * 4] = gtime();
   const int G = gridDim.x, U = a.n_tiles * a.KB;
   const int u0 = unit_begin(blockIdx.x, U, G), u1 = unit_begin(blockIdx.x + 1, U, G);
   const Segs segs(u0, u1, a.KB);
@@ -761,10 +758,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
           fence_after_sync();
           const uint32_t sa = base + stage * kStageBytes;
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) {
-            mma_f16(d, smem_desc(sa + k * 32), smem_desc(sa + kABytes + k * 32), id, acc);
-            acc = 1;
-          }
+          for (int k = 0; k < kAccSplit; ++k)   // four accumulators: no MMA waits for the one before
+            mma_f16(d + k * 2 * kN, smem_desc(sa + k * 32), smem_desc(sa + kABytes + k * 32), id, acc);
+          acc = 1;
           mma_commit(&ctl.empty[stage]);
           if (++stage == kStages) { stage = 0; parity ^= 1; }
         }
@@ -796,19 +792,25 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       if (epi_any(!mbar_wait(&ctl.acc_full[buf], (seg >> 1) & 1, abort_flag))) break;
       fence_after_sync();
       float v[16];
-      tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + buf * kAccCols, v);
-      if (a.lo) {
-        float vl[16];
-        tmem_ld16(tmem + ((uint32_t)(32 * q) << 16) + buf * kAccCols + kN, vl);
+      {
+        const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + buf * kAccCols;
+        tmem_ld16(ta, v);
 #pragma unroll
-        for (int m = 0; m < 16; ++m) v[m] += vl[m];
+        for (int c = 1; c < 2 * kAccSplit; ++c) {   // 16-column chunks: k step c / 2, hi (even) or lo (odd)
+          if (a.lo || !(c & 1)) {
+            float vp[16];
+            tmem_ld16(ta + c * kN, vp);
+#pragma unroll
+            for (int m = 0; m < 16; ++m) v[m] += vp[m];
+          }
+        }
       }
       fence_before_sync();
       mbar_arrive(&ctl.acc_empty[buf]);
+      bool finish = whole;   // this CTA runs the tile's epilogue
       if (whole) {
 #pragma unroll
         for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
-        tile_epilogue<EPI>(a, ctl, t, r, q, lane);
       } else {
         // partial tile: slot 0 = this CTA's first segment, slot 1 = its last one
         const int slot = (t == segs.t0) ? 0 : 1;
@@ -820,45 +822,56 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         const int c_first = unit_owner(t_begin, U, G), c_last = unit_owner(t_end - 1, U, G);
         if (et == 0) {
           // one thread publishes the block's partial (the barrier above ordered the other
-          // threads' stores before this fence) and, if it came last, acquires the others'
+          // threads' stores before this release) and, if it came last, acquires the others'
           int n_contrib = 0;   // CTAs between the owners of the tile's ends that hold any unit
           for (int c = c_first; c <= c_last; ++c) n_contrib += unit_begin(c, U, G) < unit_begin(c + 1, U, G);
-          __threadfence();
-          const unsigned old = atomicAdd(&a.tile_tickets[t], 1u);
+          unsigned old;
+          asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(&a.tile_tickets[t]) : "memory");
           const int last = old == (unsigned)(n_contrib - 1);
-          if (last) {
-            a.tile_tickets[t] = 0u;
-            __threadfence();
-          }
+          if (last) a.tile_tickets[t] = 0u;
           ctl.tile_last = last;
         }
         epi_sync();
         const bool last = ctl.tile_last != 0;
         epi_sync();   // everyone has read the flag before a later segment rewrites it
         if (last) {
+          // sum of the partials in CTA order (it does not depend on who came last); the loads
+          // of up to eight contributors are issued together
+          for (int m = 0; m < a.M; ++m) ctl.acc[m * 128 + r] = 0.f;
+          for (int cb0 = c_first; cb0 <= c_last; cb0 += 8) {
+            int off[8];   // element offset of contributor cb0 + j's partial, -1: none
 #pragma unroll
-          for (int m = 0; m < 16; ++m) v[m] = 0.f;
-          for (int c = c_first; c <= c_last; ++c) {   // fixed order: the sum does not depend on who is last
-            const int cb = unit_begin(c, U, G);
-            if (cb >= unit_begin(c + 1, U, G)) continue;   // a CTA without units
-            const int c_tile0 = cb / a.KB;
-            const int sl = (c == c_first && c_tile0 != t) ? 1 : 0;
-            const float* Pc = a.partials + ((size_t)c * 2 + sl) * 16 * 128;
+            for (int j = 0; j < 8; ++j) {
+              const int c = cb0 + j;
+              off[j] = -1;
+              if (c <= c_last) {
+                const int cb = unit_begin(c, U, G);
+                if (cb < unit_begin(c + 1, U, G)) {   // else a CTA without units
+                  const int sl = (c == c_first && cb / a.KB != t) ? 1 : 0;
+                  off[j] = (c * 2 + sl) * 16 * 128 + r;
+                }
+              }
+            }
+#pragma unroll 1
+            for (int m = 0; m < a.M; ++m) {
+              float x[8];
 #pragma unroll
-            for (int m = 0; m < 16; ++m)
-              if (m < a.M) v[m] += __ldcg(Pc + m * 128 + r);
+              for (int j = 0; j < 8; ++j) x[j] = off[j] >= 0 ? __ldcg(a.partials + off[j] + m * 128) : 0.f;
+              float sum = ctl.acc[m * 128 + r];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) sum += x[j];
+              ctl.acc[m * 128 + r] = sum;
+            }
           }
-#pragma unroll
-          for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
-          tile_epilogue<EPI>(a, ctl, t, r, q, lane);
+          finish = true;
         }
       }
+      if (finish) tile_epilogue<EPI>(a, ctl, t, r, q, lane);
     }
     fence_before_sync();
   }
 
   __syncthreads();
-  if (tid == 0) g_tr[blockIdx.x * 4 + 1] = gtime();
   if (EPI == EPI_LMHEAD) {
     // the last CTA to finish merges the per-tile summaries (no CTA waits for another)
     if (tid == 0) {
@@ -939,7 +952,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         }
       }
     }
-    if (ctl.is_last && tid == 0) { *a.ticket = 0u; g_tr[602] = gtime() - g_tr[blockIdx.x * 4 + 1]; }
+    if (ctl.is_last && tid == 0) *a.ticket = 0u;
     __syncthreads();
   }
   if (ctl.abort_flag) {
@@ -948,7 +961,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
     if (tid == 0) atomicOr(a.status, kStatTimeout);
     __syncthreads();
   }
-  if (tid == 0) g_tr[blockIdx.x * 4 + 2] = gtime();
   if (warp == 1) {
     fence_after_sync();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -1289,6 +1301,3 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
 
 
 
-extern "C" int ps_trace_read(unsigned long long* host) {
-  return (int)cudaMemcpyFromSymbol(host, ps::g_tr, 8192);
-}

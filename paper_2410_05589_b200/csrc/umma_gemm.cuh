@@ -6,7 +6,9 @@
 // other in shared memory and form one N = 32 operand, so one instruction retires a 128 x 16
 // weight block (4 KB) against both planes (measured: the cost of these small MMAs is per
 // instruction, not per column).  The accumulator (128 lanes x 32 columns of fp32) lives in
-// tensor memory; the epilogue adds the two halves.  Operands reach shared memory by tiled TMA loads (cp.async.bulk.tensor.2d) in the
+// tensor memory.  MMAs that add into the same accumulator run one after the other at full
+// latency, so the four k steps of a unit go to four accumulators of their own; the epilogue
+// adds the four and their two halves.  Operands reach shared memory by tiled TMA loads (cp.async.bulk.tensor.2d) in the
 // 128-byte-swizzled K-major layout the instruction reads: per stage one 128-row x 64-column
 // box of weights (16 KB) and the matching 16 x 64 boxes of the activation planes.
 //
@@ -48,7 +50,8 @@ constexpr int kStageBytes = kABytes + 2 * kBBytes;
 constexpr int kStages = 10;
 constexpr int kThreads = 192;
 constexpr int kEpiThreads = 128;
-constexpr int kAccCols = 2 * kN;                  // accumulator columns: hi products, lo products
+constexpr int kAccSplit = kBK / 16;               // independent partial accumulators, one per k step of a unit
+constexpr int kAccCols = kAccSplit * 2 * kN;      // accumulator columns: per k step hi products, lo products
 constexpr int kTmemCols = 2 * kAccCols;           // two accumulators
 // Instruction descriptor of kind::f16: fp32 accumulator, bf16 x bf16, both operands K-major,
 // N / 8 in bits [17,23), M / 16 in bits [24,29).
