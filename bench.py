@@ -50,6 +50,25 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+# Kernel that runs each stage of the bf16 small-batch path.
+KERNEL_OF_STAGE = {
+    "fc_norm": "k_gather_x + k_umma_gemm<STORE>", "qkv_rope": "k_umma_gemm<STORE>",
+    "attention": "k_attn_mma", "o_proj": "k_umma_gemm<STORE>", "ffn_gate_up": "k_umma_gemm<SWIGLU>",
+    "ffn_down": "k_umma_gemm<STORE>", "lm_head": "k_umma_gemm<LMHEAD>", "verify": "k_verify_cluster",
+}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
+# profiles/k_umma_gemm_13b_b1_k4.md, keyed by (workload, batch, k_masks, stage).  Valid for the
+# kernels as captured; set an entry to None when its kernel changes.
+NCU_DRAM_BYTES = {
+    ("13b", 1, 4, "fc_norm"): 105872384 + 4049152,
+    ("13b", 1, 4, "qkv_rope"): 157781248 + 3869440,
+    ("13b", 1, 4, "o_proj"): 52934144 + 5120,
+    ("13b", 1, 4, "ffn_gate_up"): 284786176 + 4916736,
+    ("13b", 1, 4, "ffn_down"): 143446272 + 4156416,
+    ("13b", 1, 4, "lm_head"): 329086208 + 4603136,
+}
+
+
 def stage_bytes(s, B, lens):
     """Algorithmic bytes each stage must move per step (weights once, KV once, logits written
     once by the LM head and read once by verify together with the target logits)."""
@@ -62,7 +81,8 @@ def stage_bytes(s, B, lens):
         "qkv_rope": e * (Hq * H + 2 * Hkv * H),
         "attention": e * 2 * Hkv * int(sum(lens)),
         "o_proj": e * H * Hq,
-        "ffn": e * 3 * H * F,
+        "ffn_gate_up": e * 2 * H * F,
+        "ffn_down": e * H * F,
         "lm_head": e * V * H + 4 * M * V,
         "verify": 8 * M * V,
     }
@@ -349,8 +369,10 @@ def main():
     roofline = None
     if dom:
         roofline = {
-            "bound": "hbm", "kernel": dom, "achieved": stages[dom]["gbs"], "peak": peak,
-            "unit": "GB/s", "frac": round(stages[dom]["gbs"] / peak, 4), "traffic": None,
+            "bound": "hbm", "kernel": KERNEL_OF_STAGE.get(dom, dom), "stage": dom,
+            "achieved": stages[dom]["gbs"], "peak": peak,
+            "unit": "GB/s", "frac": round(stages[dom]["gbs"] / peak, 4),
+            "traffic": NCU_DRAM_BYTES.get((args.workload, B, s.k_masks, dom)),
             "peak_kind": f"of {peak_kind}", "bytes_per_launch": sb[dom],
         }
 

@@ -1133,6 +1133,7 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
     a.out_hi = f.actp.hi; a.out_lo = f.actp.lo; a.ld_plane = F;
     if ((s = launch_umma<EPI_SWIGLU>(c, u.w_gate, u.w_up, u.w_up, u.a_hi, u.a_lo, a, f, st))) return s;
   }
+  prof_mark(c, st, "ffn_gate_up");
   float* hdn = feat_out ? feat_out : c->hdn;
   {  // S5b hdn = a + W_d act
     UArgs a{};
@@ -1142,7 +1143,7 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
     a.out_hi = f.hdnp.hi; a.out_lo = f.hdnp.lo; a.ld_plane = H; a.gain_next = (BP)w.g_final;
     if ((s = launch_umma<EPI_STORE>(c, u.w_down, u.w_down, u.w_down, u.act_hi, u.act_lo, a, f, st))) return s;
   }
-  prof_mark(c, st, "ffn");
+  prof_mark(c, st, "ffn_down");
   {  // S6 logits = W_lm rms(hdn), softmax statistics and top-n without a second pass over logits
     UArgs a{};
     a.N = V; a.K = H; a.M = M; a.n_mats = 1; a.mat_rows[0] = V; a.lo = 1;
@@ -1271,6 +1272,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.out_hi = f.actp.hi; a.out_lo = f.actp.lo; a.ld_plane = F;
     if ((s = launch_gemm<false, EPI_SWIGLU>(c, a, st))) return s;
   }
+  prof_mark(c, st, "ffn_gate_up");
   float* hdn = feat_out ? feat_out : c->hdn;
   {  // S5b hdn = a + W_d act
     GemmArgs a{};
@@ -1282,7 +1284,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.out_hi = f.hdnp.hi; a.out_lo = f.hdnp.lo; a.ld_plane = H; a.gain_next = (BP)w.g_final;
     if ((s = launch_gemm<false, EPI_STORE>(c, a, st))) return s;
   }
-  prof_mark(c, st, "ffn");
+  prof_mark(c, st, "ffn_down");
   {  // S6 logits = W_lm rms(hdn), softmax statistics and top-n without a second pass over logits
     GemmArgs a{};
     a.rs.W[0] = (BP)w.w_lm; a.rs.rows[0] = V; a.rs.n_mats = 1;
