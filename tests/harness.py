@@ -21,11 +21,11 @@ class Pair:
     """Oracle + CUDA drafter with identical weights and identical caches."""
 
     def __init__(self, s, B, with_bias=False, context="append", lens=None, flags=0, oracle_seqs=None,
-                 extra_ctx=0):
+                 extra_ctx=0, weights=None):
         import paper_2410_05589_b200 as ps
 
         self.s, self.B = s, B
-        self.W = synth.weights(s, with_bias=with_bias)
+        self.W = synth.weights(s, with_bias=with_bias) if weights is None else weights
         self.lens = synth.ctx_lengths(s, B) if lens is None else np.asarray(lens, np.int32)
         max_ctx = int(self.lens.max()) + s.k_masks + 1 + extra_ctx
         self.oracle_seqs = list(range(B)) if oracle_seqs is None else list(oracle_seqs)

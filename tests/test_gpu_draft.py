@@ -153,3 +153,35 @@ def test_full_size_batch1(name):
     Kg, Vg = Kg.float().cpu().numpy(), Vg.float().cpu().numpy()
     assert (np.abs(Kg[L:] - Ko[L:]) <= 2.0 ** -7 * np.abs(Ko[L:]) + 1e-2).all()
     assert (np.abs(Vg[L:] - Vo[L:]) <= 2.0 ** -7 * np.abs(Vo[L:]) + 1e-2).all()
+
+
+_W13 = {}
+
+
+def _weights_13b_sweep():
+    if "w" not in _W13:
+        _W13["w"] = synth.weights(synth.CONFIGS["13b_sweep"])
+    return _W13["w"]
+
+
+@pytest.mark.parametrize("B,k", [(4, 8), (16, 2), (64, 4)])
+def test_13b_batch_sweep_sampled_sequences(B, k):
+    """Points of the 13B-shaped batch / mask-count sweep at full size (ragged contexts of 256 to
+    2048 positions, imported): every sequence runs on the GPU, the oracle recomputes three of
+    them (the shortest, the longest and the last) row by row."""
+    s = synth.CONFIGS["13b_sweep"].with_(batch=B, k_masks=k)
+    lens = synth.ctx_lengths(s, B)
+    seqs = sorted({int(np.argmin(lens)), int(np.argmax(lens)), B - 1})
+    p = Pair(s, B, context="import", oracle_seqs=seqs, weights=_weights_13b_sweep())
+    _compare_step(p, top_n=1)
+    assert p.g.poll() == 0
+
+
+def test_33b_batch16_k8_sampled_sequences():
+    """The 33B-class shape at B=16, k=8, contexts of 1024 to 4096 positions: the oracle
+    recomputes the sequence with the longest context."""
+    s = synth.CONFIGS["33b"]
+    lens = synth.ctx_lengths(s, s.batch)
+    p = Pair(s, s.batch, context="import", oracle_seqs=[int(np.argmax(lens))])
+    _compare_step(p, top_n=1)
+    assert p.g.poll() == 0
