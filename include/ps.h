@@ -168,7 +168,8 @@ ps_status ps_verify(ps_ctx* ctx, int B, int n_draft, int n_target, const int* dr
  * target_logits from host memory, runs ps_draft_step (arg-max drafts of all k+1 rows) and
  * ps_verify (n_draft = n_target = k+1) on `stream`, copies accept_len / out_tokens / n_out
  * back and waits for the stream.  All pointers except ctx are host memory; pinned memory
- * makes the copies asynchronous.
+ * makes the copies asynchronous.  The target logits travel on a stream of the context's own
+ * (created by the first call) while the draft step runs.
  *   hidden_last [B][H] config dtype, token_last [B], target_logits [B][k+1][V] float,
  *   accept_len [B], out_tokens [B][k+2], n_out [B]. */
 ps_status ps_round_host(ps_ctx* ctx, int B, const int* seq_slot, const void* hidden_last,

@@ -179,6 +179,10 @@ void ps_destroy(ps_ctx* c) {
   if (!c) return;
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   fused_release(c);
+  if (c->copy_stream) {
+    cudaEventDestroy(c->copy_done);
+    cudaStreamDestroy(c->copy_stream);
+  }
   delete c;
 }
 
@@ -365,12 +369,20 @@ ps_status ps_round_host(ps_ctx* c, int B, const int* seq_slot, const void* hidde
   const int R = g.k_masks + 1;
   const size_t eb = g.dtype == PS_DTYPE_F32 ? 4 : 2;
   cudaError_t e;
-  e = cudaMemcpyAsync(c->st_hidden, hidden_last, (size_t)B * g.hidden * eb, cudaMemcpyHostToDevice, st);
+  // The target logits are needed by the verify step only: they travel on a stream of their own
+  // while the draft step runs (the staging buffer is free: every round ends synchronised).
+  if (!c->copy_stream) {
+    e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->copy_done, cudaEventDisableTiming);
+    if (e != cudaSuccess) return cuda_check(c, e, "ps_round_host copy stream");
+  }
+  e = cudaMemcpyAsync(c->st_tlogits, target_logits, (size_t)B * R * g.vocab * 4, cudaMemcpyHostToDevice,
+                      c->copy_stream);
+  if (e == cudaSuccess) e = cudaEventRecord(c->copy_done, c->copy_stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(c->st_hidden, hidden_last, (size_t)B * g.hidden * eb, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(c->st_tok, token_last, (size_t)B * 4, cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess)
-    e = cudaMemcpyAsync(c->st_tlogits, target_logits, (size_t)B * R * g.vocab * 4,
-                        cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return cuda_check(c, e, "ps_round_host h2d");
   // top_n = 1: top_ids is then exactly the [B][k+1] chain of arg-max drafts.
   s = ps_draft_step(c, B, seq_slot, c->st_hidden, c->st_tok, 1, c->st_top, (float*)(c->st_top + (size_t)c->max_rows),
@@ -379,6 +391,8 @@ ps_status ps_round_host(ps_ctx* c, int B, const int* seq_slot, const void* hidde
   int* r_acc = c->st_res;
   int* r_n = c->st_res + B;
   int* r_out = c->st_res + 2 * B;
+  e = cudaStreamWaitEvent(st, c->copy_done, 0);
+  if (e != cudaSuccess) return cuda_check(c, e, "ps_round_host wait");
   s = ps_verify(c, B, R, R, c->st_top, c->st_dlogits, c->st_tlogits, temperature, seed, offset,
                 r_acc, r_out, r_n, st);
   if (s != PS_OK) return s;

@@ -95,6 +95,8 @@ struct ps_ctx {
   double* rope_inv_freq;    // [head_dim/2] base^(-2i/d), filled once at ps_init
   int n_sm;                 // multiprocessors of the context's device
   int smem_optin;           // opt-in shared memory per block
+  cudaStream_t copy_stream = nullptr;   // ps_round_host: carries the target logits beside the draft step
+  cudaEvent_t copy_done = nullptr;
   void* st_hidden; int* st_tok; float* st_tlogits; float* st_dlogits; int* st_top; int* st_res;
   std::vector<int> len;     // committed positions per slot (host is the source of truth)
   long long launches;
