@@ -12,4 +12,5 @@ from .ps_oracle import (  # noqa: F401
     row_stats,
     uniforms,
     verify,
+    verify_tree,
 )

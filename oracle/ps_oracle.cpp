@@ -13,6 +13,9 @@
 //                   Transformer layer with the target layer's hyper-parameters,
 //                   shared LM head), Algorithm 1 (the k+1 draft distributions)
 //   pso_verify      Eq. 1 and Algorithm 1 in its chain case (each node has one child)
+//   pso_verify_tree Algorithm 1 in full: a token tree, children tried in turn, the
+//                   target distribution replaced by its normalised residual after
+//                   every rejection
 //   pso_philox4x32  Salmon et al., "Parallel random numbers: as easy as 1, 2, 3"
 //                   (SC'11), Philox-4x32 with 10 rounds
 //
@@ -21,7 +24,9 @@
 // parameter count of Sec. 5.1, Philox known-answer vectors, closed forms of
 // Eq. 1 (acceptance probability = 1 - TV(p,q), emitted token ~ p), Monte-Carlo
 // losslessness on a 16-token vocabulary, and the special cases p = q, disjoint
-// supports and temperature 0.
+// supports and temperature 0.  The tree walk is pinned by its reduction to the chain
+// routine on chain-shaped trees, by Monte-Carlo losslessness with several children per
+// node drawn independently from q, and by the greedy longest-matching-path rule.
 // Parity unpinned: the numeric logits of a *trained* drafter and the paper's
 // acceptance lengths / speed-ups (they need weights and data the paper does not print).
 #include <cmath>
@@ -543,6 +548,104 @@ int pso_verify(int B, int n_draft, int n_target, int V, const int* draft_tokens,
     int n = a;
     if (emitted >= 0) out[n++] = emitted;
     n_out[b] = n;
+    if (nonfinite) nonfinite[b] = bad;
+  }
+  return 0;
+}
+
+// Algorithm 1 in full, for B independent sequences that share one tree shape.
+//   parent[n_nodes]: parent node of node i (< i), -1 for the children of the root.  The
+//   children of a node are tried in increasing node id (the Select order).  A child of the
+//   root has depth 0, a child of node i depth(i) + 1; all nodes of depth t were drafted
+//   from the same distribution q_t = softmax(draft_logits[b][t] / T) (the parallel drafter
+//   gives one distribution per depth).  tokens [B][n_nodes].  target_logits
+//   [B][n_nodes+1][V]: row 0 is the target distribution after the prefix, row 1+i the one
+//   after the path that ends in node i.  Decision row u (0 or 1+i) draws r for its j-th
+//   child from the Philox counter (u + (j << 16), b, offset), word 0, and its final sample
+//   from word 1 of the counter (u, b, offset): a chain-shaped tree then uses exactly the
+//   uniforms of pso_verify.
+// Outputs: accept_len[B] accepted nodes; path[B][max_depth] their ids (-1 unused);
+//   out_tokens[B][max_depth+1] their tokens followed by the token sampled at the node where
+//   the walk stopped (-1 unused); n_out[B] = accept_len + 1; margin_accept[B] = the smallest
+//   |r - min(1, p/q)| over the tests made; margin_cdf[B] as in pso_verify; nonfinite[B].
+int pso_verify_tree(int B, int n_nodes, int max_depth, int V, const int* parent, const int* tokens,
+                    const float* draft_logits, const float* target_logits, double temperature,
+                    uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
+                    int* path, double* margin_accept, double* margin_cdf, int* nonfinite) {
+  const double INF = std::numeric_limits<double>::infinity();
+  std::vector<int> depth(n_nodes);
+  for (int i = 0; i < n_nodes; ++i) {
+    if (parent[i] >= i || parent[i] < -1) return -1;
+    depth[i] = parent[i] < 0 ? 0 : depth[parent[i]] + 1;
+    if (depth[i] >= max_depth) return -1;
+  }
+  if (temperature != 0.0 && !draft_logits) return -1;
+#pragma omp parallel for schedule(dynamic, 16)
+  for (int b = 0; b < B; ++b) {
+    int* out = out_tokens + (size_t)b * (max_depth + 1);
+    int* pth = path + (size_t)b * max_depth;
+    for (int i = 0; i <= max_depth; ++i) out[i] = -1;
+    for (int i = 0; i < max_depth; ++i) pth[i] = -1;
+    double m_acc = INF, m_cdf = INF;
+    int bad = 0, a = 0, emitted = -1;
+    int u = 0;                                   // decision row: 0 = root, 1 + node id
+    std::vector<double> p(V), q(V);
+    for (;;) {
+      const float* t = target_logits + ((size_t)b * (n_nodes + 1) + u) * V;
+      std::vector<int> H;                        // children of u, in Select order
+      for (int i = 0; i < n_nodes; ++i)
+        if (parent[i] == u - 1) H.push_back(i);
+      const int d = u == 0 ? 0 : depth[u - 1] + 1;   // depth of the children
+      if (temperature == 0.0) {
+        int tstar = argmax_row(t, V), next = -1;
+        for (int c : H)
+          if (tokens[(size_t)b * n_nodes + c] == tstar) { next = c; break; }
+        if (next < 0) { emitted = tstar; break; }
+        out[a] = tstar; pth[a] = next; ++a; u = next + 1;
+        continue;
+      }
+      RowStat st = row_stat(t, V, temperature);
+      if (st.nonfinite) { bad = 1; emitted = argmax_row(t, V); break; }
+      for (int v = 0; v < V; ++v) p[v] = prob(t, v, temperature, st);
+      std::vector<double> p0 = p;
+      int next = -1;
+      if (!H.empty()) {
+        const float* dl = draft_logits + ((size_t)b * max_depth + d) * V;
+        RowStat sd = row_stat(dl, V, temperature);
+        if (sd.nonfinite) { bad = 1; emitted = argmax_row(t, V); break; }
+        for (int v = 0; v < V; ++v) q[v] = prob(dl, v, temperature, sd);
+        for (size_t j = 0; j < H.size(); ++j) {
+          const int x = tokens[(size_t)b * n_nodes + H[j]];
+          double r, unused;
+          pso_uniforms(seed, offset, b, u + (int)(j << 16), &r, &unused);
+          double ratio;
+          if (x < 0 || x >= V) ratio = 0.0;
+          else if (q[x] > 0.0) ratio = p[x] / q[x] < 1.0 ? p[x] / q[x] : 1.0;
+          else ratio = p[x] > 0.0 ? 1.0 : 0.0;
+          if (std::fabs(r - ratio) < m_acc) m_acc = std::fabs(r - ratio);
+          if (r < ratio) { next = H[j]; break; }
+          // rejected: p := norm((p - q)+)
+          double W = 0.0;
+          for (int v = 0; v < V; ++v) { p[v] = p[v] > q[v] ? p[v] - q[v] : 0.0; W += p[v]; }
+          if (W > 0.0) for (int v = 0; v < V; ++v) p[v] /= W;
+          else { p = p0; }   // nothing left of the residual: fall back to the node's own p
+        }
+      }
+      if (next >= 0) {
+        out[a] = tokens[(size_t)b * n_nodes + next]; pth[a] = next; ++a; u = next + 1;
+        continue;
+      }
+      double r_unused, u2, W = 0.0;
+      pso_uniforms(seed, offset, b, u, &r_unused, &u2);
+      for (int v = 0; v < V; ++v) W += p[v];
+      emitted = inverse_cdf(p, W, u2, &m_cdf);
+      break;
+    }
+    accept_len[b] = a;
+    out[a] = emitted;
+    n_out[b] = a + 1;
+    if (margin_accept) margin_accept[b] = m_acc;
+    if (margin_cdf) margin_cdf[b] = m_cdf;
     if (nonfinite) nonfinite[b] = bad;
   }
   return 0;

@@ -245,3 +245,42 @@ def verify(draft_tokens, draft_logits, target_logits, temperature: float, seed: 
         raise ValueError(f"oracle verify status {rc}")
     return dict(accept_len=accept_len, out_tokens=out_tokens, n_out=n_out,
                 margin_accept=margin_accept, margin_cdf=margin_cdf, nonfinite=nonfinite)
+
+
+def verify_tree(parent, tokens, draft_logits, target_logits, temperature: float, seed: int, offset: int,
+                max_depth: int | None = None):
+    """Algorithm 1 in full.  parent [n_nodes] (-1: child of the root; children are tried in
+    increasing node id), tokens [B][n_nodes], draft_logits [B][max_depth][V] (one row per tree
+    depth) or None at temperature 0, target_logits [B][n_nodes+1][V] (row 0: after the prefix,
+    row 1+i: after node i).  Returns a dict of numpy arrays."""
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    target_logits = np.ascontiguousarray(target_logits, dtype=np.float32)
+    B, n_nodes = tokens.shape
+    V = target_logits.shape[-1]
+    assert target_logits.shape == (B, n_nodes + 1, V) and parent.shape == (n_nodes,)
+    if draft_logits is not None:
+        draft_logits = np.ascontiguousarray(draft_logits, dtype=np.float32)
+        max_depth = draft_logits.shape[1] if max_depth is None else max_depth
+        assert draft_logits.shape == (B, max_depth, V)
+    assert max_depth is not None
+    accept_len = np.empty(B, np.int32)
+    out_tokens = np.empty((B, max_depth + 1), np.int32)
+    n_out = np.empty(B, np.int32)
+    path = np.empty((B, max_depth), np.int32)
+    margin_accept = np.empty(B, np.float64)
+    margin_cdf = np.empty(B, np.float64)
+    nonfinite = np.empty(B, np.int32)
+    lib = _load()
+    lib.pso_verify_tree.restype = C.c_int
+    lib.pso_verify_tree.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                    C.c_void_p, C.c_double, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p,
+                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    rc = lib.pso_verify_tree(B, n_nodes, max_depth, V, _ptr(parent), _ptr(tokens), _ptr(draft_logits),
+                             _ptr(target_logits), float(temperature), seed, offset, _ptr(accept_len),
+                             _ptr(out_tokens), _ptr(n_out), _ptr(path), _ptr(margin_accept), _ptr(margin_cdf),
+                             _ptr(nonfinite))
+    if rc != 0:
+        raise ValueError(f"oracle verify_tree status {rc}")
+    return dict(accept_len=accept_len, out_tokens=out_tokens, n_out=n_out, path=path,
+                margin_accept=margin_accept, margin_cdf=margin_cdf, nonfinite=nonfinite)
