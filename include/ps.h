@@ -51,6 +51,7 @@ enum {
   PS_FLAG_MMA_SYNC_GEMM = 4     /* fused path: mma.sync GEMM kernels instead of the tcgen05 ones */
 };
 enum { PS_MAX_BATCH = 128, PS_MAX_MASKS = 15, PS_MAX_TOP_N = 8 };
+enum { PS_MAX_TREE_NODES = 64 };  /* nodes of a token tree (ps_verify_tree) */
 enum { PS_STATIC_MAX_BATCH = 128, PS_STATIC_MAX_VOCAB = 262144 }; /* limits of ps_verify_static */
 
 typedef struct ps_config {
@@ -163,6 +164,36 @@ ps_status ps_verify(ps_ctx* ctx, int B, int n_draft, int n_target, const int* dr
                     const float* draft_logits, const float* target_logits, float temperature,
                     uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
                     void* stream);
+
+/* Lossless verification of a drafted token tree (Algorithm 1 in full; Sec. 3 "token tree
+ * verification").  The tree shape is shared by the batch: parent[i] is the parent of node i
+ * (a node before i) or -1 for a child of the root; the children of a node are tried in
+ * increasing node id (the algorithm's Select order).  A child of the root has depth 0; every
+ * node of depth t was drafted from q_t = softmax(draft_logits[b][t]/T), the parallel drafter's
+ * distribution for position t.  Decision row u = 0 is the root, u = 1+i the node i;
+ * p_u = softmax(target_logits[b][u]/T) is the target distribution after the path that ends
+ * there.  At row u the children are tried in turn: accept x iff r < min(1, p(x)/q(x)) and move
+ * to that child; otherwise p := max(0, p-q) normalised and the next child is tried.  When no
+ * child is left (or u is a leaf) one token is drawn from the current p and the walk stops.
+ * r of the j-th child of row u is word 0 of Philox-4x32-10 with key = seed and counter =
+ * (u + (j << 16), b, offset); the final draw uses word 1 of the counter (u, b, offset), so a
+ * chain-shaped tree reproduces ps_verify with n_target = n_draft + 1.  temperature 0 is
+ * greedy: the walk follows the first child that carries the arg-max of the target row.
+ *   parent        HOST [n_nodes] int32, 1 <= n_nodes <= PS_MAX_TREE_NODES
+ *   tokens        device [B][n_nodes] int32
+ *   draft_logits  device [B][D][V] float, D = 1 + the largest depth (may be NULL at T = 0)
+ *   target_logits device [B][n_nodes+1][V] float
+ *   accept_len    device [B] int32: accepted nodes
+ *   out_tokens    device [B][D+1] int32: their tokens, then the drawn token, then -1
+ *   n_out         device [B] int32 = accept_len + 1
+ *   path          device [B][D] int32: the accepted nodes' ids, then -1
+ * Needs vocab % 4 == 0, vocab <= 65536 and 16-byte aligned logits (PS_ERR_UNSUPPORTED
+ * otherwise).  Non-finite logits in an examined row: the walk stops there with the arg-max of
+ * that target row and ps_poll reports PS_ERR_NONFINITE. */
+ps_status ps_verify_tree(ps_ctx* ctx, int B, int n_nodes, const int* parent, const int* tokens,
+                         const float* draft_logits, const float* target_logits, float temperature,
+                         uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,
+                         int* n_out, int* path, void* stream);
 
 /* Host-buffer convenience for one draft+verify round: copies hidden_last / token_last /
  * target_logits from host memory, runs ps_draft_step (arg-max drafts of all k+1 rows) and

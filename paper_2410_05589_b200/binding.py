@@ -29,7 +29,7 @@ EXPORTS = (
     "ps_workspace_bytes", "ps_init", "ps_kv_append", "ps_draft_step", "ps_verify", "ps_round_host",
     "ps_kv_len", "ps_kv_reset", "ps_kv_export", "ps_kv_import", "ps_poll", "ps_launch_count",
     "ps_last_error", "ps_destroy", "ps_philox_fill", "ps_profile", "ps_profile_read",
-    "ps_verify_static", "ps_debug_buffer",
+    "ps_verify_static", "ps_debug_buffer", "ps_verify_tree",
 )
 
 
@@ -74,6 +74,8 @@ def load_library(path: str | None = None) -> C.CDLL:
                               C.c_uint64, vp, vp, vp, vp]
     lib.ps_round_host.argtypes = [vp, C.c_int, ip, vp, vp, vp, C.c_float, C.c_uint64, C.c_uint64,
                                   vp, vp, vp, vp]
+    lib.ps_verify_tree.argtypes = [vp, C.c_int, C.c_int, ip, vp, vp, vp, C.c_float, C.c_uint64, C.c_uint64,
+                                   vp, vp, vp, vp, vp]
     lib.ps_kv_len.argtypes = [vp, C.c_int, ip]
     lib.ps_kv_reset.argtypes = [vp, C.c_int]
     lib.ps_kv_export.argtypes = [vp, C.c_int, vp, vp, vp]
@@ -263,6 +265,31 @@ class Drafter:
             self.h, B, n_draft, n_target, _dptr(draft_tokens), _dptr(draft_logits),
             _dptr(target_logits), float(temperature), seed, offset, _dptr(o["accept_len"]),
             _dptr(o["out_tokens"]), _dptr(o["n_out"]), _stream(stream)))
+        return o
+
+    def verify_tree(self, parent, tokens: torch.Tensor, draft_logits, target_logits: torch.Tensor,
+                    temperature: float, seed: int, offset: int, out: dict | None = None, stream=None) -> dict:
+        """ps_verify_tree.  parent: host list [n_nodes]; tokens [B][n_nodes] int32; draft_logits
+        [B][D][V] float32 (D = 1 + largest depth) or None at temperature 0; target_logits
+        [B][n_nodes+1][V] float32."""
+        B, n_nodes = tokens.shape
+        assert len(parent) == n_nodes and target_logits.shape == (B, n_nodes + 1, self.cfg.vocab)
+        depth = []
+        for i, p in enumerate(parent):
+            depth.append(0 if p < 0 or p >= i else depth[p] + 1)   # a malformed tree is the library's to reject
+        D = max(depth) + 1
+        if draft_logits is not None:
+            assert draft_logits.shape == (B, D, self.cfg.vocab) and draft_logits.dtype == torch.float32
+        o = out if out is not None else {}
+        if "accept_len" not in o:
+            o["accept_len"] = torch.empty(B, dtype=torch.int32, device="cuda")
+            o["out_tokens"] = torch.empty((B, D + 1), dtype=torch.int32, device="cuda")
+            o["n_out"] = torch.empty(B, dtype=torch.int32, device="cuda")
+            o["path"] = torch.empty((B, D), dtype=torch.int32, device="cuda")
+        self._check(self.lib.ps_verify_tree(
+            self.h, B, n_nodes, _iarr(parent), _dptr(tokens), _dptr(draft_logits), _dptr(target_logits),
+            float(temperature), seed, offset, _dptr(o["accept_len"]), _dptr(o["out_tokens"]),
+            _dptr(o["n_out"]), _dptr(o["path"]), _stream(stream)))
         return o
 
     def round_host(self, seq_slot, hidden_last: torch.Tensor, token_last: torch.Tensor,

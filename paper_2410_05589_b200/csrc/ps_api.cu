@@ -70,6 +70,8 @@ size_t carve(const ps_config& g, ps_ctx* c, char* base) {
   void* status = take(256);
   void* tickets = take(sizeof(unsigned) * PS_MAX_BATCH);
   void* vrec = take(sizeof(VerifyRec) * PS_MAX_BATCH * (PS_MAX_MASKS + 2));
+  void* trec = take(sizeof(TreeRec) * PS_MAX_BATCH * (PS_MAX_TREE_NODES + 1));
+  void* ttick = take(sizeof(unsigned) * PS_MAX_BATCH);
   void* x_in = take(Mx * 2 * H * 4);
   void* x0 = take(Mx * H * 4);
   void* xn = take(Mx * H * 4);
@@ -94,6 +96,7 @@ size_t carve(const ps_config& g, ps_ctx* c, char* base) {
   if (c) {
     c->kcache = kc; c->vcache = vc; c->dev_status = (int*)status; c->tickets = (unsigned*)tickets;
     c->vrec = (VerifyRec*)vrec;
+    c->trec = (TreeRec*)trec; c->tree_tickets = (unsigned*)ttick;
     c->x_in = (float*)x_in; c->x0 = (float*)x0; c->xn = (float*)xn; c->q = (float*)q;
     c->kv_tmp = (float*)kv_tmp; c->attn = (float*)attn; c->a = (float*)a; c->an = (float*)an;
     c->gate = (float*)gate; c->up = (float*)up; c->hdn = (float*)hdn; c->hn = (float*)hn;
@@ -167,6 +170,7 @@ ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* w, void*
   if (e == cudaSuccess)
     e = cudaMemsetAsync(c->fused_scratch, 0, fused_scratch_bytes(*cfg), st);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * PS_MAX_BATCH, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->tree_tickets, 0, sizeof(unsigned) * PS_MAX_BATCH, st);
   if (e != cudaSuccess || launch_rope_table(c, st) != PS_OK) {
     delete c;
     return PS_ERR_CUDA;
@@ -353,6 +357,20 @@ ps_status ps_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draf
   return launch_verify(c, B, n_draft, n_target, draft_tokens, draft_logits, target_logits,
                        temperature, seed, offset, accept_len, out_tokens, n_out,
                        (cudaStream_t)stream);
+}
+
+ps_status ps_verify_tree(ps_ctx* c, int B, int n_nodes, const int* parent, const int* tokens,
+                         const float* draft_logits, const float* target_logits, float temperature,
+                         uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
+                         int* path, void* stream) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  if (B < 1 || B > PS_MAX_BATCH) return fail(c, PS_ERR_INVALID_ARG, "bad batch");
+  if (n_nodes < 1 || n_nodes > PS_MAX_TREE_NODES) return fail(c, PS_ERR_CAPACITY, "tree of 1..PS_MAX_TREE_NODES nodes");
+  if (!parent || !tokens || !target_logits || !accept_len || !out_tokens || !n_out || !path)
+    return fail(c, PS_ERR_INVALID_ARG, "null pointer");
+  if (!(temperature >= 0.f)) return fail(c, PS_ERR_INVALID_ARG, "temperature must be >= 0");
+  return launch_verify_tree(c, B, n_nodes, parent, tokens, draft_logits, target_logits, temperature, seed,
+                            offset, accept_len, out_tokens, n_out, path, nullptr, (cudaStream_t)stream);
 }
 
 ps_status ps_round_host(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,

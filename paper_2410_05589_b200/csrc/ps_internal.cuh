@@ -67,6 +67,12 @@ cudaError_t launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t s
 constexpr int kStatNonfinite = 1;
 constexpr int kStatTimeout = 2;
 
+struct TreeRec {    // one per (sequence, decision row) of the token-tree verification
+  int next;         // accepted child node, -1 if none
+  int token;        // token to emit if the walk stops here
+  int bad;          // a non-finite logit was met
+};
+
 struct VerifyRec {  // one per (sequence, position): result of the acceptance test
   int accept;       // bit 0: accepted; bit 1: a non-finite logit was met
   int token;        // token to emit if this position ends the chain
@@ -87,6 +93,8 @@ struct ps_ctx {
   int* dev_status;
   unsigned* tickets;        // [max_batch] arrival counters of the verify kernel (zero between calls)
   ps::VerifyRec* vrec;      // [max_batch][PS_MAX_MASKS+2]
+  ps::TreeRec* trec;        // [max_batch][PS_MAX_TREE_NODES+1]
+  unsigned* tree_tickets;   // [max_batch], zero between calls
   float *x_in, *x0, *xn, *q, *kv_tmp, *attn, *a, *an, *gate, *up, *hdn, *hn, *logits;
   // staging for ps_round_host
   void* fused_scratch;      // buffers of the fused bf16 path (see fused_kernels.cu)
@@ -139,6 +147,10 @@ ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* 
                         const float* draft_logits, const float* target_logits, float temperature,
                         uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,
                         int* n_out, cudaStream_t st);
+ps_status launch_verify_tree(ps_ctx* c, int B, int n_nodes, const int* parent, const int* tokens,
+                             const float* draft_logits, const float* target_logits, float temperature,
+                             uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
+                             int* path, int* max_depth_out, cudaStream_t st);
 ps_status launch_kv_copy(ps_ctx* c, int slot, int len, void* K, void* V, bool to_cache,
                          cudaStream_t st);
 }  // namespace ps

@@ -579,6 +579,322 @@ k_verify_cluster(VerifyArgs a) {
   cl.sync();   // no block leaves while another may still read its shared memory
 }
 
+
+// ---- token-tree verification (Algorithm 1 in full) -------------------------------------------
+// One cluster per (decision row, sequence): row u = 0 is the root, u = 1 + i the node i.  The
+// cluster holds the target row of u and the draft row of its children's depth in registers and
+// tries the children in turn.  After j rejections the target distribution of Algorithm 1 is
+// norm((p - c q)+) with c_0 = 0, c_{j+1} = c_j + Z(c_j), Z(c) = sum_v (p_v - c q_v)+ (the
+// repeated "subtract q, clip, renormalise" in closed form), so a rejection costs one reduction
+// over the cluster.  If no child is accepted (or u is a leaf) the cluster draws the token that
+// would be emitted at u.  The last cluster of a sequence to finish walks the tree from the root
+// along the accepted children.  Nothing spins.
+struct TreeTopo {
+  int n_nodes, max_depth;
+  unsigned char depth[PS_MAX_TREE_NODES];
+  unsigned char child_off[PS_MAX_TREE_NODES + 2];   // children of decision row u: child_idx[off[u] .. off[u+1])
+  unsigned char child_idx[PS_MAX_TREE_NODES];
+};
+
+struct TreeArgs {
+  int B, V;
+  TreeTopo topo;
+  const int* tokens;           // [B][n_nodes]
+  const float* draft_logits;   // [B][max_depth][V]
+  const float* target_logits;  // [B][n_nodes+1][V]
+  float temperature;
+  uint32_t key0, key1, off_lo, off_hi;
+  int* accept_len; int* out_tokens; int* n_out; int* path;
+  TreeRec* rec;                // [B][PS_MAX_TREE_NODES+1]
+  unsigned* tickets;           // [B], zero on entry and on exit
+  int* status;
+};
+
+// Sum over the cluster of one double per thread; every thread of every block gets the value.
+__device__ double cluster_sum(cooperative_groups::cluster_group& cl, CluPart& part, CluScratch& s, double v,
+                              int tid, int warp, int lane) {
+  v = warp_sum_d(v);
+  __syncthreads();
+  if (lane == 0) s.d[warp] = v;
+  __syncthreads();
+  if (tid == 0) {
+    double x1 = 0.0;
+    for (int w = 0; w < kCluWarps; ++w) x1 += s.d[w];
+    part.wsum = x1;
+  }
+  cl.sync();
+  double tot = 0.0;
+  for (int rr = 0; rr < kClu; ++rr) tot += cl.map_shared_rank(&part, rr)->wsum;
+  cl.sync();   // every block has read the partials before they are rewritten
+  return tot;
+}
+
+// Inverse-CDF draw by the cluster over per-thread weights w[] (thread owns tokens v0 + e): the
+// first token whose running sum exceeds u * total, found block -> warp -> lane -> token.
+// Returns the token to every thread of every block, -1 if the total weight is not positive.
+__device__ int cluster_draw(cooperative_groups::cluster_group& cl, CluPart& part, CluScratch& s,
+                            const float (&w)[kCluV4 * 4], int v0, double u, int rank, int tid, int warp,
+                            int lane) {
+  double mine = 0.0;
+  int lastp = -1;
+#pragma unroll
+  for (int e = 0; e < kCluV4 * 4; ++e) {
+    mine += (double)w[e];
+    if (w[e] > 0.f) lastp = v0 + e;
+  }
+  double incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const double up = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  lastp = __reduce_max_sync(0xffffffffu, lastp);
+  __syncthreads();
+  if (lane == 31) { s.d[warp] = incl; s.i[warp] = lastp; }
+  __syncthreads();
+  if (tid == 0) {
+    double x1 = 0.0;
+    int lp = -1;
+    for (int k = 0; k < kCluWarps; ++k) { x1 += s.d[k]; lp = max(lp, s.i[k]); }
+    part.wsum = x1; part.lastp = lp; part.pick = -1;
+  }
+  cl.sync();
+  double total = 0.0;
+  for (int rr = 0; rr < kClu; ++rr) total += cl.map_shared_rank(&part, rr)->wsum;
+  int sel = -1, token = -1;
+  if (total > 0.0) {
+    const double target = u * total;
+    double run = 0.0, base = 0.0;
+    for (int rr = 0; rr < kClu; ++rr) {
+      const double nx = run + cl.map_shared_rank(&part, rr)->wsum;
+      if (sel < 0 && nx > target) { sel = rr; base = run; }
+      run = nx;
+    }
+    if (sel == rank) {
+      double t2 = target - base, wrun = 0.0, wbase = 0.0;
+      int wsel = -1;
+      for (int k = 0; k < kCluWarps; ++k) {
+        const double nx = wrun + s.d[k];
+        if (wsel < 0 && nx > t2) { wsel = k; wbase = wrun; }
+        wrun = nx;
+      }
+      if (warp == wsel) {
+        const double t3 = t2 - wbase;
+        const unsigned over = __ballot_sync(0xffffffffu, incl > t3);
+        if (over) {
+          const int src = __ffs(over) - 1;
+          double excl = __shfl_up_sync(0xffffffffu, incl, 1);
+          if (lane == 0) excl = 0.0;
+          if (lane == src) {
+            const double t4 = t3 - excl;
+            double run4 = 0.0;
+            int pick = -1, lp = -1;
+#pragma unroll
+            for (int e = 0; e < kCluV4 * 4; ++e) {
+              if (w[e] > 0.f) lp = e;
+              run4 += (double)w[e];
+              if (pick < 0 && run4 > t4) pick = e;
+            }
+            if (pick < 0) pick = lp;
+            if (pick >= 0) part.pick = v0 + pick;
+          }
+        }
+      }
+    }
+  }
+  cl.sync();
+  if (total > 0.0) {
+    // rounding may leave no token chosen on the way down: take the last one with weight
+    token = sel >= 0 ? cl.map_shared_rank(&part, sel)->pick : -1;
+    if (token < 0)
+      for (int rr = 0; rr < kClu; ++rr) token = max(token, cl.map_shared_rank(&part, rr)->lastp);
+  }
+  cl.sync();   // all reads of the partials are done before they are rewritten
+  return token;
+}
+
+__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads) k_verify_tree(TreeArgs a) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cl = cg::this_cluster();
+  __shared__ CluPart part;
+  __shared__ CluScratch s;
+  const int rank = (int)cl.block_rank();
+  const int u = blockIdx.x / kClu, b = blockIdx.y, V = a.V, n_nodes = a.topo.n_nodes;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int kid0 = a.topo.child_off[u], n_kids = a.topo.child_off[u + 1] - kid0;
+  const int dq = u == 0 ? 0 : a.topo.depth[u - 1] + 1;   // depth of the children of u
+  const bool greedy = a.temperature == 0.f;
+  const float* trow = a.target_logits + ((size_t)b * (n_nodes + 1) + u) * V;
+  const float* drow = (!greedy && n_kids > 0) ? a.draft_logits + ((size_t)b * a.topo.max_depth + dq) * V : nullptr;
+  const int* toks = a.tokens + (size_t)b * n_nodes;
+  const int nv4 = ((V + kClu * kCluThreads - 1) / (kClu * kCluThreads) + 3) / 4;
+  const int C = nv4 * 4, v0 = (rank * kCluThreads + tid) * C;
+
+  float t[kCluV4 * 4], d[kCluV4 * 4];
+#pragma unroll
+  for (int k = 0; k < kCluV4; ++k) {
+    const int v = v0 + 4 * k;   // V % 4 == 0: a vector lies inside the row or outside it
+    float4 tv = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY), dv = tv;
+    if (k < nv4 && v < V) {
+      tv = *reinterpret_cast<const float4*>(trow + v);
+      if (drow) dv = *reinterpret_cast<const float4*>(drow + v);
+    }
+    t[4 * k] = tv.x; t[4 * k + 1] = tv.y; t[4 * k + 2] = tv.z; t[4 * k + 3] = tv.w;
+    d[4 * k] = dv.x; d[4 * k + 1] = dv.y; d[4 * k + 2] = dv.z; d[4 * k + 3] = dv.w;
+  }
+  // ---- maxima (NaN counts as -inf, ties to the lower id) and non-finite flags
+  float tm = -INFINITY, dm = -INFINITY;
+  int ti = 0x7fffffff, bad = 0;
+#pragma unroll
+  for (int e = 0; e < kCluV4 * 4; ++e) {
+    const int v = v0 + e;
+    if (e < C && v < V) {
+      float xt = t[e];
+      if (xt != xt || xt == INFINITY) bad = 1;
+      if (xt != xt) xt = -INFINITY;
+      if (xt > tm || (xt == tm && v < ti)) { tm = xt; ti = v; }
+      if (drow) {
+        float xd = d[e];
+        if (xd != xd || xd == INFINITY) bad = 1;
+        if (xd != xd) xd = -INFINITY;
+        dm = fmaxf(dm, xd);
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, tm, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, ti, o);
+    if (ov > tm || (ov == tm && oi < ti)) { tm = ov; ti = oi; }
+    dm = fmaxf(dm, __shfl_xor_sync(0xffffffffu, dm, o));
+    bad |= __shfl_xor_sync(0xffffffffu, bad, o);
+  }
+  if (lane == 0) { s.f[warp] = tm; s.i[warp] = ti; s.flag[warp] = bad; s.f2[warp] = dm; }
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < kCluWarps; ++w) {
+      if (s.f[w] > tm || (s.f[w] == tm && s.i[w] < ti)) { tm = s.f[w]; ti = s.i[w]; }
+      dm = fmaxf(dm, s.f2[w]);
+      bad |= s.flag[w];
+    }
+    part.tmax = tm; part.targ = ti; part.dmax = dm; part.bad = bad;
+    part.pick = -1; part.lastp = -1; part.wsum = 0.0; part.st = 0.0; part.sd = 0.0;
+  }
+  cl.sync();
+  tm = -INFINITY; dm = -INFINITY; ti = 0x7fffffff; bad = 0;
+  for (int r = 0; r < kClu; ++r) {
+    const CluPart* pr = cl.map_shared_rank(&part, r);
+    const float ov = pr->tmax;
+    const int oi = pr->targ;
+    if (ov > tm || (ov == tm && oi < ti)) { tm = ov; ti = oi; }
+    dm = fmaxf(dm, pr->dmax);
+    bad |= pr->bad;
+  }
+  cl.sync();   // the partials are free again
+  if (tm == -INFINITY || (drow && dm == -INFINITY)) bad = 1;  // a row without a distribution
+  const float tmax = tm, dmax = dm;
+  const int targ = ti;
+
+  int next = -1, token = -1;
+  if (greedy) {
+    for (int j = 0; j < n_kids && next < 0; ++j)
+      if (toks[a.topo.child_idx[kid0 + j]] == targ) next = a.topo.child_idx[kid0 + j];
+    token = targ;
+    bad = 0;
+  } else if (bad) {
+    token = targ;
+  } else {
+    // every block takes the same branches below: the values they depend on are identical
+    const double inv_t = 1.0 / (double)a.temperature;
+    double st = 0.0, sd = 0.0;
+#pragma unroll
+    for (int e = 0; e < kCluV4 * 4; ++e) {
+      const bool in = e < C && v0 + e < V;
+      t[e] = in ? expf((float)(((double)t[e] - (double)tmax) * inv_t)) : 0.f;
+      st += (double)t[e];
+      d[e] = (in && drow) ? expf((float)(((double)d[e] - (double)dmax) * inv_t)) : 0.f;
+      sd += (double)d[e];
+    }
+    st = cluster_sum(cl, part, s, st, tid, warp, lane);
+    sd = drow ? cluster_sum(cl, part, s, sd, tid, warp, lane) : 1.0;
+    const float inv_st = (float)(1.0 / st), inv_sd = (float)(1.0 / sd);
+    double c = 0.0, Zc = 1.0;   // the target distribution at u is now (p - c q)+ / Zc
+    for (int j = 0; j < n_kids; ++j) {
+      const int kid = a.topo.child_idx[kid0 + j];
+      const int x = toks[kid];
+      uint32_t ctr[4] = {(uint32_t)u + ((uint32_t)j << 16), (uint32_t)b, a.off_lo, a.off_hi};
+      philox4x32_10(a.key0, a.key1, ctr);
+      const double r = (double)(ctr[0] >> 8) * (1.0 / 16777216.0);
+      const bool in_range = x >= 0 && x < V;
+      const double logp = in_range ? ((double)trow[x] - (double)tmax) * inv_t - log(st) : -INFINITY;
+      const double logq = in_range ? ((double)drow[x] - (double)dmax) * inv_t - log(sd) : -INFINITY;
+      double ratio;
+      if (c == 0.0) {
+        const double diff = logp - logq;
+        ratio = (diff != diff) ? 0.0 : exp(fmin(diff, 0.0));
+      } else {
+        const double px = exp(logp), qx = exp(logq);
+        const double wx = fmax(px - c * qx, 0.0) / Zc;
+        ratio = qx > 0.0 ? fmin(wx / qx, 1.0) : (wx > 0.0 ? 1.0 : 0.0);
+      }
+      if (r < ratio) { next = kid; break; }
+      // rejected: the target distribution becomes norm((p - (c + Zc) q)+)
+      const double c_new = c + Zc;
+      const float cf = (float)c_new;
+      double mine = 0.0;
+#pragma unroll
+      for (int e = 0; e < kCluV4 * 4; ++e) mine += (double)fmaxf(t[e] * inv_st - cf * (d[e] * inv_sd), 0.f);
+      const double Z = cluster_sum(cl, part, s, mine, tid, warp, lane);
+      if (Z > 0.0) { c = c_new; Zc = Z; } else { c = 0.0; Zc = 1.0; }   // nothing left: back to p
+    }
+    if (next < 0) {
+      uint32_t ctr[4] = {(uint32_t)u, (uint32_t)b, a.off_lo, a.off_hi};
+      philox4x32_10(a.key0, a.key1, ctr);
+      const double u2 = (double)(ctr[1] >> 8) * (1.0 / 16777216.0);
+      const float cf = (float)c;
+      float w[kCluV4 * 4];
+#pragma unroll
+      for (int e = 0; e < kCluV4 * 4; ++e) w[e] = fmaxf(t[e] * inv_st - cf * (d[e] * inv_sd), 0.f);
+      token = cluster_draw(cl, part, s, w, v0, u2, rank, tid, warp, lane);
+      if (token < 0 && c != 0.0) {   // the residual vanished in fp32: draw from p
+#pragma unroll
+        for (int e = 0; e < kCluV4 * 4; ++e) w[e] = t[e] * inv_st;
+        token = cluster_draw(cl, part, s, w, v0, u2, rank, tid, warp, lane);
+      }
+      if (token < 0) token = targ;
+    }
+  }
+  if (rank == 0 && tid == 0) {
+    TreeRec* rec = a.rec + (size_t)b * (PS_MAX_TREE_NODES + 1);
+    rec[u].next = next; rec[u].token = token; rec[u].bad = bad;
+    __threadfence();
+    const unsigned tk = atomicAdd(&a.tickets[b], 1u);
+    if (tk == (unsigned)n_nodes) {   // the last of the n_nodes + 1 decision rows
+      __threadfence();
+      volatile TreeRec* R = rec;
+      int* out = a.out_tokens + (size_t)b * (a.topo.max_depth + 1);
+      int* pth = a.path + (size_t)b * a.topo.max_depth;
+      int uu = 0, len = 0, any_bad = 0;
+      for (;;) {
+        any_bad |= R[uu].bad;
+        const int nx = R[uu].next;
+        if (nx < 0 || len >= a.topo.max_depth) { out[len] = R[uu].token; break; }
+        out[len] = toks[nx];
+        pth[len] = nx;
+        ++len;
+        uu = nx + 1;
+      }
+      for (int j = len + 1; j <= a.topo.max_depth; ++j) out[j] = -1;
+      for (int j = len; j < a.topo.max_depth; ++j) pth[j] = -1;
+      a.accept_len[b] = len;
+      a.n_out[b] = len + 1;
+      if (any_bad) atomicOr(a.status, kStatNonfinite);
+      a.tickets[b] = 0u;
+    }
+  }
+  cl.sync();   // no block leaves while another may still read its shared memory
+}
+
 }  // namespace
 
 ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draft_tokens,
@@ -613,6 +929,45 @@ ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* 
   c->launches++;
   prof_mark(c, st, "verify");
   return cuda_check(c, cudaGetLastError(), "k_verify");
+}
+
+ps_status launch_verify_tree(ps_ctx* c, int B, int n_nodes, const int* parent, const int* tokens,
+                             const float* draft_logits, const float* target_logits, float temperature,
+                             uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
+                             int* path, int* max_depth_out, cudaStream_t st) {
+  TreeArgs a;
+  a.B = B; a.V = c->cfg.vocab;
+  TreeTopo& tp = a.topo;
+  tp.n_nodes = n_nodes;
+  tp.max_depth = 0;
+  for (int i = 0; i < n_nodes; ++i) {
+    if (parent[i] >= i || parent[i] < -1) return fail(c, PS_ERR_INVALID_ARG, "parent[i] must be -1 or a node before i");
+    tp.depth[i] = (unsigned char)(parent[i] < 0 ? 0 : tp.depth[parent[i]] + 1);
+    tp.max_depth = std::max(tp.max_depth, (int)tp.depth[i] + 1);
+  }
+  int off = 0;
+  for (int u = 0; u <= n_nodes; ++u) {   // children of decision row u in increasing node id
+    tp.child_off[u] = (unsigned char)off;
+    for (int i = 0; i < n_nodes; ++i)
+      if (parent[i] == u - 1) tp.child_idx[off++] = (unsigned char)i;
+  }
+  tp.child_off[n_nodes + 1] = (unsigned char)off;
+  if (max_depth_out) *max_depth_out = tp.max_depth;
+  if (temperature != 0.f && !draft_logits) return fail(c, PS_ERR_INVALID_ARG, "draft_logits needed at temperature > 0");
+  const bool aligned = (((uintptr_t)target_logits | (uintptr_t)draft_logits) & 15u) == 0;
+  if (a.V % 4 || a.V > kCluMaxVocab || !aligned)
+    return fail(c, PS_ERR_UNSUPPORTED, "ps_verify_tree needs vocab % 4 == 0, vocab <= 65536 and 16-byte aligned logits");
+  a.tokens = tokens; a.draft_logits = draft_logits; a.target_logits = target_logits;
+  a.temperature = temperature;
+  a.key0 = (uint32_t)seed; a.key1 = (uint32_t)(seed >> 32);
+  a.off_lo = (uint32_t)offset; a.off_hi = (uint32_t)(offset >> 32);
+  a.accept_len = accept_len; a.out_tokens = out_tokens; a.n_out = n_out; a.path = path;
+  a.rec = c->trec; a.tickets = c->tree_tickets; a.status = c->dev_status;
+  prof_mark(c, st, "begin");
+  k_verify_tree<<<dim3((n_nodes + 1) * kClu, B), kCluThreads, 0, st>>>(a);
+  c->launches++;
+  prof_mark(c, st, "verify_tree");
+  return cuda_check(c, cudaGetLastError(), "k_verify_tree");
 }
 
 }  // namespace ps
