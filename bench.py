@@ -88,6 +88,53 @@ def stage_bytes(s, B, lens):
     }
 
 
+# A 26-node draft tree of the shape tree drafters use (4 children of the root, depth 6).
+TREE26 = [-1, -1, -1, -1, 0, 0, 0, 1, 1, 2, 4, 4, 5, 7, 10, 10, 11, 12, 13, 14, 14, 16, 18, 19, 21, 22]
+
+
+def tree_verify_leg(g, ps, s, B, T, peak, n_buf=6, reps=60):
+    """ps_verify_tree alone on the 26-node tree: synthetic target rows per node, one draft row
+    per depth (noisy copies, so that paths of several nodes are accepted), node tokens drawn
+    from the draft rows.  Buffers rotate so that rows come from HBM, not from L2."""
+    import numpy as np
+    import torch
+
+    import synth
+    n = len(TREE26)
+    depth = []
+    for p in TREE26:
+        depth.append(0 if p < 0 else depth[p] + 1)
+    D, V = max(depth) + 1, s.vocab
+    sets = []
+    for i in range(n_buf):
+        tl = synth.gauss_logits(s.seed, ("tree_t", i), (B, n + 1, V))
+        dl = synth.noisy_draft_logits(s.seed, ("tree_d", i), np.repeat(tl[:, :1], D, axis=1), 0.6)
+        for j in range(n):
+            if depth[j] + 1 < D:
+                tl[:, 1 + j] = dl[:, depth[j] + 1] + 0.5 * tl[:, 1 + j]
+        toks = synth.sample_from_logits(s.seed, ("tree_x", i), dl[:, depth], temperature=max(T, 0.5))
+        sets.append((ps.to_device(toks.astype(np.int32)), ps.to_device(dl), ps.to_device(tl)))
+    out = {}
+    for i in range(5):
+        t_, d_, l_ = sets[i % n_buf]
+        g.verify_tree(TREE26, t_, d_, l_, T, 1, i, out=out)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        t_, d_, l_ = sets[i % n_buf]
+        g.verify_tree(TREE26, t_, d_, l_, T, 1, 100 + i, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / reps * 1e3
+    rows_with_children = len({p for p in TREE26})            # decision rows that read a draft row
+    nbytes = 4 * V * B * ((n + 1) + rows_with_children)
+    return {"us": round(us, 2), "nodes": n, "depth": D, "bytes": nbytes,
+            "gbs": round(nbytes / (us * 1e-6) / 1e9, 1), "frac_of_peak": round(nbytes / (us * 1e-6) / 1e9 / peak, 4),
+            "mean_accepted_nodes": float(out["accept_len"].float().mean().item()),
+            "note": "(n+1) target rows and one draft row per row with children, each read once"}
+
+
 def max_over_ranks(x: float, device="cuda") -> float:
     """Slowest rank's value (every rank gets it).  Replicas exchange nothing else."""
     import torch
@@ -376,6 +423,11 @@ def main():
             "peak_kind": f"of {peak_kind}", "bytes_per_launch": sb[dom],
         }
 
+    # ---- token-tree verification (Algorithm 1 in full), timed on its own ---------------------
+    tree = None
+    if V % 4 == 0 and V <= 65536 and s.dtype == 1:
+        tree = tree_verify_leg(g, ps, s, B, T, peak)
+
     # ---- end to end through the host-buffer entry point -----------------------------------
     hl_h = torch.from_numpy(hl_np.view(np.int16) if hl_np.dtype == np.uint16 else hl_np).pin_memory()
     tl_h = torch.from_numpy(tl_np).pin_memory()
@@ -420,7 +472,7 @@ def main():
             "hbm_frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
             "mean_tokens_per_round": n_accept,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "stages": stages, "cpu_baseline": cpu,
+            "roofline": roofline, "stages": stages, "tree_verify": tree, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
     if world > 1:

@@ -624,7 +624,7 @@ __device__ double cluster_sum(cooperative_groups::cluster_group& cl, CluPart& pa
   }
   cl.sync();
   double tot = 0.0;
-  for (int rr = 0; rr < kClu; ++rr) tot += cl.map_shared_rank(&part, rr)->wsum;
+  for (int rr = 0; rr < (int)cl.num_blocks(); ++rr) tot += cl.map_shared_rank(&part, rr)->wsum;
   cl.sync();   // every block has read the partials before they are rewritten
   return tot;
 }
@@ -660,12 +660,12 @@ __device__ int cluster_draw(cooperative_groups::cluster_group& cl, CluPart& part
   }
   cl.sync();
   double total = 0.0;
-  for (int rr = 0; rr < kClu; ++rr) total += cl.map_shared_rank(&part, rr)->wsum;
+  for (int rr = 0; rr < (int)cl.num_blocks(); ++rr) total += cl.map_shared_rank(&part, rr)->wsum;
   int sel = -1, token = -1;
   if (total > 0.0) {
     const double target = u * total;
     double run = 0.0, base = 0.0;
-    for (int rr = 0; rr < kClu; ++rr) {
+    for (int rr = 0; rr < (int)cl.num_blocks(); ++rr) {
       const double nx = run + cl.map_shared_rank(&part, rr)->wsum;
       if (sel < 0 && nx > target) { sel = rr; base = run; }
       run = nx;
@@ -707,19 +707,22 @@ __device__ int cluster_draw(cooperative_groups::cluster_group& cl, CluPart& part
     // rounding may leave no token chosen on the way down: take the last one with weight
     token = sel >= 0 ? cl.map_shared_rank(&part, sel)->pick : -1;
     if (token < 0)
-      for (int rr = 0; rr < kClu; ++rr) token = max(token, cl.map_shared_rank(&part, rr)->lastp);
+      for (int rr = 0; rr < (int)cl.num_blocks(); ++rr) token = max(token, cl.map_shared_rank(&part, rr)->lastp);
   }
   cl.sync();   // all reads of the partials are done before they are rewritten
   return token;
 }
 
-__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads) k_verify_tree(TreeArgs a) {
+// (The cluster size is a launch attribute: 8 blocks per row, or fewer when a large tree would
+// otherwise need a second wave of blocks.)
+__global__ void __launch_bounds__(kCluThreads) k_verify_tree(TreeArgs a) {
   namespace cg = cooperative_groups;
   cg::cluster_group cl = cg::this_cluster();
   __shared__ CluPart part;
   __shared__ CluScratch s;
   const int rank = (int)cl.block_rank();
-  const int u = blockIdx.x / kClu, b = blockIdx.y, V = a.V, n_nodes = a.topo.n_nodes;
+  const int nclu = (int)cl.num_blocks();
+  const int u = blockIdx.x / nclu, b = blockIdx.y, V = a.V, n_nodes = a.topo.n_nodes;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int kid0 = a.topo.child_off[u], n_kids = a.topo.child_off[u + 1] - kid0;
   const int dq = u == 0 ? 0 : a.topo.depth[u - 1] + 1;   // depth of the children of u
@@ -727,7 +730,7 @@ __global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads) k_ve
   const float* trow = a.target_logits + ((size_t)b * (n_nodes + 1) + u) * V;
   const float* drow = (!greedy && n_kids > 0) ? a.draft_logits + ((size_t)b * a.topo.max_depth + dq) * V : nullptr;
   const int* toks = a.tokens + (size_t)b * n_nodes;
-  const int nv4 = ((V + kClu * kCluThreads - 1) / (kClu * kCluThreads) + 3) / 4;
+  const int nv4 = ((V + nclu * kCluThreads - 1) / (nclu * kCluThreads) + 3) / 4;
   const int C = nv4 * 4, v0 = (rank * kCluThreads + tid) * C;
 
   float t[kCluV4 * 4], d[kCluV4 * 4];
@@ -782,7 +785,7 @@ __global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads) k_ve
   }
   cl.sync();
   tm = -INFINITY; dm = -INFINITY; ti = 0x7fffffff; bad = 0;
-  for (int r = 0; r < kClu; ++r) {
+  for (int r = 0; r < (int)cl.num_blocks(); ++r) {
     const CluPart* pr = cl.map_shared_rank(&part, r);
     const float ov = pr->tmax;
     const int oi = pr->targ;
@@ -964,10 +967,24 @@ ps_status launch_verify_tree(ps_ctx* c, int B, int n_nodes, const int* parent, c
   a.accept_len = accept_len; a.out_tokens = out_tokens; a.n_out = n_out; a.path = path;
   a.rec = c->trec; a.tickets = c->tree_tickets; a.status = c->dev_status;
   prof_mark(c, st, "begin");
-  k_verify_tree<<<dim3((n_nodes + 1) * kClu, B), kCluThreads, 0, st>>>(a);
+  // blocks per decision row: as many as fit in one wave of the device, at most 8, and enough for
+  // each thread to hold its share of a row (16 tokens)
+  int nclu = kClu;
+  while (nclu > 1 && (long)(n_nodes + 1) * B * nclu > c->n_sm && a.V <= (nclu / 2) * kCluThreads * 4 * kCluV4)
+    nclu /= 2;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((n_nodes + 1) * nclu, B);
+  cfg.blockDim = dim3(kCluThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = nclu; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, k_verify_tree, a);
   c->launches++;
   prof_mark(c, st, "verify_tree");
-  return cuda_check(c, cudaGetLastError(), "k_verify_tree");
+  return cuda_check(c, e, "k_verify_tree");
 }
 
 }  // namespace ps
