@@ -7,6 +7,7 @@ from .ps_oracle import (  # noqa: F401
     Oracle,
     OracleConfig,
     build_oracle,
+    gumbel_sample,
     num_threads,
     philox4x32,
     row_stats,

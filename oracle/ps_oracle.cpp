@@ -16,6 +16,8 @@
 //   pso_verify_tree Algorithm 1 in full: a token tree, children tried in turn, the
 //                   target distribution replaced by its normalised residual after
 //                   every rejection
+//   pso_gumbel_sample  Algorithm 1's "sampling from the parallel draft model": one token per
+//                   row drawn from softmax(logits/T) by the Gumbel-max rule with Philox uniforms
 //   pso_philox4x32  Salmon et al., "Parallel random numbers: as easy as 1, 2, 3"
 //                   (SC'11), Philox-4x32 with 10 rounds
 //
@@ -549,6 +551,33 @@ int pso_verify(int B, int n_draft, int n_target, int V, const int* draft_tokens,
     if (emitted >= 0) out[n++] = emitted;
     n_out[b] = n;
     if (nonfinite) nonfinite[b] = bad;
+  }
+  return 0;
+}
+
+// One token per row from softmax(logits[r] / T) by the Gumbel-max rule: the arg-max over v of
+// logits[r][v] / T + G, G = -ln(-ln u), u = ((w >> 8) + 0.5) / 2^24 with w = word 0 of
+// Philox-4x32-10, key = (seed_lo ^ 0x6D756247, seed_hi), counter = (v, row_id[r], offset).
+// Ties go to the lower id.  margin[r] = best perturbed value minus the runner-up.
+int pso_gumbel_sample(const double* logits, int n_rows, int V, double temperature, uint64_t seed,
+                      uint64_t offset, const int* row_id, int* tokens, double* margin) {
+  if (!(temperature > 0.0)) return -1;
+  uint32_t key[2] = {(uint32_t)seed ^ 0x6D756247u, (uint32_t)(seed >> 32)};
+  for (int r = 0; r < n_rows; ++r) {
+    const double* row = logits + (size_t)r * V;
+    double best = -std::numeric_limits<double>::infinity(), second = best;
+    int arg = -1;
+    for (int v = 0; v < V; ++v) {
+      uint32_t ctr[4] = {(uint32_t)v, (uint32_t)row_id[r], (uint32_t)offset, (uint32_t)(offset >> 32)};
+      uint32_t o[4];
+      philox4x32_10(key, ctr, o);
+      const double u = ((double)(o[0] >> 8) + 0.5) / 16777216.0;
+      const double y = row[v] / temperature - std::log(-std::log(u));
+      if (y > best) { second = best; best = y; arg = v; }
+      else if (y > second) second = y;
+    }
+    tokens[r] = arg;
+    if (margin) margin[r] = best - second;
   }
   return 0;
 }

@@ -284,3 +284,23 @@ def verify_tree(parent, tokens, draft_logits, target_logits, temperature: float,
         raise ValueError(f"oracle verify_tree status {rc}")
     return dict(accept_len=accept_len, out_tokens=out_tokens, n_out=n_out, path=path,
                 margin_accept=margin_accept, margin_cdf=margin_cdf, nonfinite=nonfinite)
+
+
+def gumbel_sample(logits, temperature: float, seed: int, offset: int, row_id):
+    """One token per row from softmax(logits / T) by the Gumbel-max rule with the Philox stream
+    of the draft sampler.  logits [rows][V] float64, row_id [rows] int (b | j << 8).
+    Returns (tokens, margin): margin = best perturbed value minus the runner-up."""
+    logits = np.ascontiguousarray(logits, dtype=np.float64)
+    row_id = np.ascontiguousarray(row_id, dtype=np.int32)
+    n, V = logits.shape
+    tokens = np.empty(n, np.int32)
+    margin = np.empty(n, np.float64)
+    lib = _load()
+    lib.pso_gumbel_sample.restype = C.c_int
+    lib.pso_gumbel_sample.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_double, C.c_uint64, C.c_uint64,
+                                      C.c_void_p, C.c_void_p, C.c_void_p]
+    rc = lib.pso_gumbel_sample(_ptr(logits), n, V, float(temperature), seed, offset, _ptr(row_id),
+                               _ptr(tokens), _ptr(margin))
+    if rc != 0:
+        raise ValueError(f"oracle gumbel_sample status {rc}")
+    return tokens, margin
