@@ -423,6 +423,28 @@ def main():
             "peak_kind": f"of {peak_kind}", "bytes_per_launch": sb[dom],
         }
 
+    # ---- the same step with the drafts sampled in the LM head (lossless at T > 0) -------------
+    sampled = None
+    if T > 0:
+        s_out = {}
+
+        def step_sampled(i):
+            o = g.draft_step_sampled(slots[i % n_sets], hl, tl, T, 1, i, top_n=1, want_logits=True, out=s_out)
+            g.verify(o["sampled"], o["logits"], tgt[i % len(tgt)], T, 1, i, out=v_out)
+
+        for i in range(5):
+            step_sampled(i)
+        torch.cuda.synchronize()
+        n_s = min(args.steps, 300)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for i in range(n_s):
+            step_sampled(i)
+        f1.record()
+        torch.cuda.synchronize()
+        sampled = {"ms_per_step": f0.elapsed_time(f1) / n_s, "steps": n_s,
+                   "note": "ps_draft_step_sampled (Gumbel-max in the LM-head epilogue) + ps_verify"}
+
     # ---- token-tree verification (Algorithm 1 in full), timed on its own ---------------------
     tree = None
     if V % 4 == 0 and V <= 65536 and s.dtype == 1:
@@ -472,7 +494,7 @@ def main():
             "hbm_frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
             "mean_tokens_per_round": n_accept,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "stages": stages, "tree_verify": tree, "cpu_baseline": cpu,
+            "roofline": roofline, "stages": stages, "sampled_drafts": sampled, "tree_verify": tree, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
     if world > 1:

@@ -142,6 +142,23 @@ ps_status ps_draft_step(ps_ctx* ctx, int B, const int* seq_slot, const void* hid
                         float* row_max, float* row_lse, float* logits_out, float* feat_out,
                         void* stream);
 
+/* ps_draft_step that also draws one token per row from softmax(logits / temperature)
+ * (Algorithm 1: the draft tree is built "by sampling from the parallel draft model"), inside
+ * the LM-head kernel, without a second pass over the logits.  The draw is the Gumbel-max rule:
+ * sampled = argmax_v (logit_v / T + G_v), G_v = -ln(-ln u_v), u_v = ((w >> 8) + 0.5) / 2^24
+ * with w = word 0 of Philox-4x32-10, key = (seed_lo ^ 0x6D756247, seed_hi), counter =
+ * (v, b | j << 8, offset) for row j of the b-th sequence of the call; ties go to the lower id.
+ * Passing these tokens and logits_out to ps_verify with the same temperature makes a round
+ * lossless end to end.  temperature > 0.
+ *   sampled_ids  device [B][k+1] int32
+ * Everything else as ps_draft_step.  On the mma.sync fall-back kernels (PS_FLAG_MMA_SYNC_GEMM)
+ * logits_out must be given (PS_ERR_UNSUPPORTED otherwise). */
+ps_status ps_draft_step_sampled(ps_ctx* ctx, int B, const int* seq_slot, const void* hidden_last,
+                                const int* token_last, float temperature, uint64_t seed,
+                                uint64_t offset, int* sampled_ids, int top_n, int* top_ids,
+                                float* top_logit, float* row_max, float* row_lse, float* logits_out,
+                                float* feat_out, void* stream);
+
 /* Lossless verification of a drafted chain (Eq. 1; Algorithm 1 with one child per node).
  * For position i = 0..n_draft-1 of sequence b, with p = softmax(target_logits[b][i]/T),
  * q = softmax(draft_logits[b][i]/T) and x = draft_tokens[b][i]: accept iff

@@ -29,7 +29,7 @@ EXPORTS = (
     "ps_workspace_bytes", "ps_init", "ps_kv_append", "ps_draft_step", "ps_verify", "ps_round_host",
     "ps_kv_len", "ps_kv_reset", "ps_kv_export", "ps_kv_import", "ps_poll", "ps_launch_count",
     "ps_last_error", "ps_destroy", "ps_philox_fill", "ps_profile", "ps_profile_read",
-    "ps_verify_static", "ps_debug_buffer", "ps_verify_tree",
+    "ps_verify_static", "ps_debug_buffer", "ps_verify_tree", "ps_draft_step_sampled",
 )
 
 
@@ -74,6 +74,8 @@ def load_library(path: str | None = None) -> C.CDLL:
                               C.c_uint64, vp, vp, vp, vp]
     lib.ps_round_host.argtypes = [vp, C.c_int, ip, vp, vp, vp, C.c_float, C.c_uint64, C.c_uint64,
                                   vp, vp, vp, vp]
+    lib.ps_draft_step_sampled.argtypes = [vp, C.c_int, ip, vp, vp, C.c_float, C.c_uint64, C.c_uint64, vp,
+                                          C.c_int, vp, vp, vp, vp, vp, vp, vp]
     lib.ps_verify_tree.argtypes = [vp, C.c_int, C.c_int, ip, vp, vp, vp, C.c_float, C.c_uint64, C.c_uint64,
                                    vp, vp, vp, vp, vp]
     lib.ps_kv_len.argtypes = [vp, C.c_int, ip]
@@ -248,6 +250,30 @@ class Drafter:
             self.h, B, _iarr(seq_slot), _dptr(hidden_last), _dptr(token_last), top_n,
             _dptr(o["top_ids"]), _dptr(o["top_logit"]), _dptr(o["row_max"]), _dptr(o["row_lse"]),
             _dptr(o.get("logits")), _dptr(o.get("feat")), _stream(stream)))
+        return o
+
+    def draft_step_sampled(self, seq_slot, hidden_last: torch.Tensor, token_last: torch.Tensor,
+                           temperature: float, seed: int, offset: int, top_n: int = 1,
+                           want_logits: bool = True, want_feat: bool = False, out: dict | None = None,
+                           stream=None) -> dict:
+        """ps_draft_step_sampled: ps_draft_step plus ``sampled`` [B][k+1] int32, one token per row
+        drawn from softmax(logits / temperature)."""
+        B, R, V, H = len(seq_slot), self.rows, self.cfg.vocab, self.cfg.hidden
+        o = out if out is not None else {}
+        dev = "cuda"
+        if "row_max" not in o:
+            o["top_ids"] = torch.empty((B, R, max(top_n, 1)), dtype=torch.int32, device=dev)
+            o["top_logit"] = torch.empty((B, R, max(top_n, 1)), dtype=torch.float32, device=dev)
+            o["row_max"] = torch.empty((B, R), dtype=torch.float32, device=dev)
+            o["row_lse"] = torch.empty((B, R), dtype=torch.float32, device=dev)
+            o["logits"] = torch.empty((B, R, V), dtype=torch.float32, device=dev) if want_logits else None
+            o["feat"] = torch.empty((B, R, H), dtype=torch.float32, device=dev) if want_feat else None
+        if "sampled" not in o:
+            o["sampled"] = torch.empty((B, R), dtype=torch.int32, device=dev)
+        self._check(self.lib.ps_draft_step_sampled(
+            self.h, B, _iarr(seq_slot), _dptr(hidden_last), _dptr(token_last), float(temperature), seed, offset,
+            _dptr(o["sampled"]), top_n, _dptr(o["top_ids"]), _dptr(o["top_logit"]), _dptr(o["row_max"]),
+            _dptr(o["row_lse"]), _dptr(o.get("logits")), _dptr(o.get("feat")), _stream(stream)))
         return o
 
     def verify(self, draft_tokens: torch.Tensor, draft_logits, target_logits: torch.Tensor,

@@ -35,6 +35,8 @@ struct __align__(16) LmPart {  // softmax / top-n summary of one vocabulary rang
   float v0; int i0;          // copy of top_v[0], top_i[0]: the first 16 bytes decide a top-1 merge
   float top_v[kTopMax];
   int top_i[kTopMax];
+  float sv; int si;          // draft sampling: best perturbed logit of the range and its token
+  int pad_[2];
 };
 
 struct GemmArgs {
@@ -476,6 +478,7 @@ struct UArgs {
   float* logits_out; LmPart* parts; unsigned* ticket;
   int top_n; int* top_ids; float* top_logit; float* row_max; float* row_lse;
   float* partials; unsigned* tile_tickets;
+  int sample; SampleArgs sa; int R;   // draft sampling in the LM head (sample != 0), rows per sequence
   int* status;
 };
 
@@ -659,7 +662,38 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
       }
       epi_sync();
     }
-    epi_sync();   // red / red2 are free again
+    if (a.sample) {   // Gumbel-max candidate of this vocabulary range per row
+#pragma unroll 1
+      for (int m = 0; m < a.M; ++m) {
+        const int sb = m / a.R;
+        const uint32_t row_id = (uint32_t)sb | ((uint32_t)(m - sb * a.R) << 8);
+        float bv = -FLT_MAX;
+        int bi = 0x7fffffff;
+        if (valid) {
+          bv = acc[m * 128] * ctl.scale[m] * a.sa.inv_temp + gumbel_noise(a.sa, (uint32_t)n, row_id);
+          bi = n;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+          if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == 0) { ctl.cand_v[q][m] = bv; ctl.cand_i[q][m] = bi; }
+      }
+      epi_sync();
+      if (et < a.M) {
+        float bv = ctl.cand_v[0][et]; int bi = ctl.cand_i[0][et];
+#pragma unroll
+        for (int w = 1; w < 4; ++w) {
+          const float ov = ctl.cand_v[w][et]; const int oi = ctl.cand_i[w][et];
+          if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        LmPart* p = a.parts + (size_t)t * a.M + et;
+        p->sv = bv; p->si = bi;
+      }
+    }
+    epi_sync();   // red / red2 / cand are free again
   }
 }
 
@@ -950,6 +984,28 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
           if (lane == 0) { a.top_ids[(size_t)m * a.top_n + tn] = bi; a.top_logit[(size_t)m * a.top_n + tn] = bv; }
           pv = bv; pi = bi;
         }
+        if (a.sample) {   // the row's sampled token: arg-max of the ranges' perturbed maxima
+          float bv = -FLT_MAX; int bi = 0x7fffffff;
+          for (int c0 = 0; c0 < Gt; c0 += 256) {
+            float xv[8]; int id[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int c = c0 + lane + 32 * j;
+              xv[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].sv) : -FLT_MAX;
+              id[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].si) : 0x7fffffff;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (xv[j] > bv || (xv[j] == bv && id[j] < bi)) { bv = xv[j]; bi = id[j]; }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+          }
+          if (lane == 0) a.sa.sampled[m] = bi;
+        }
       }
     }
     if (ctl.is_last && tid == 0) *a.ticket = 0u;
@@ -1081,7 +1137,8 @@ ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, c
 
 ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B, const void* hidden_last,
                           const int* token_last, int top_n, int* top_ids, float* top_logit, float* row_max,
-                          float* row_lse, float* logits_out, float* feat_out, cudaStream_t st) {
+                          float* row_lse, float* logits_out, float* feat_out, const SampleArgs* sa,
+                          cudaStream_t st) {
   const ps_config& g = c->cfg;
   const ps_weights& w = c->w;
   const int H = g.hidden, Hq = g.n_heads * g.head_dim, Hkv = g.n_kv_heads * g.head_dim, F = g.ffn,
@@ -1150,6 +1207,8 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
     a.ssq_in = f.ssq[2]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
     a.logits_out = logits_out; a.parts = f.parts; a.ticket = f.ticket;
     a.top_n = top_n; a.top_ids = top_ids; a.top_logit = top_logit; a.row_max = row_max; a.row_lse = row_lse;
+    a.R = R;
+    if (sa) { a.sample = 1; a.sa = *sa; }
     if ((s = launch_umma<EPI_LMHEAD>(c, u.w_lm, u.w_lm, u.w_lm, u.hdn_hi, u.hdn_lo, a, f, st))) return s;
   }
   prof_mark(c, st, "lm_head");
@@ -1212,16 +1271,18 @@ ps_status fused_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* by
 ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last,
                            const int* token_last, int top_n, int* top_ids, float* top_logit,
                            float* row_max, float* row_lse, float* logits_out, float* feat_out,
-                           cudaStream_t st) {
+                           const SampleArgs* sa, cudaStream_t st) {
   const ps_config& g = c->cfg;
   const ps_weights& w = c->w;
   const int H = g.hidden, Hq = g.n_heads * g.head_dim, Hkv = g.n_kv_heads * g.head_dim, F = g.ffn,
             V = g.vocab, R = g.k_masks + 1, M = B * R;
   typedef const __nv_bfloat16* BP;
   const FusedScratch f = carve_fused(g, (char*)c->fused_scratch);
+  if (sa && !c->umma_maps && !logits_out)
+    return fail(c, PS_ERR_UNSUPPORTED, "draft sampling on the mma.sync kernels needs logits_out");
   if (c->umma_maps && !(g.flags & PS_FLAG_MMA_SYNC_GEMM))
     return umma_draft_step(c, *static_cast<const UmmaMaps*>(c->umma_maps), sm, B, hidden_last, token_last, top_n,
-                           top_ids, top_logit, row_max, row_lse, logits_out, feat_out, st);
+                           top_ids, top_logit, row_max, row_lse, logits_out, feat_out, sa, st);
   ps_status s;
   prof_mark(c, st, "begin");
   {  // S1 fc: x0 = W_fc [e ; f] (+ b)
@@ -1295,6 +1356,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.top_n = top_n; a.top_ids = top_ids; a.top_logit = top_logit; a.row_max = row_max; a.row_lse = row_lse;
     if ((s = launch_gemm<false, EPI_LMHEAD>(c, a, st))) return s;
   }
+  if (sa && (s = launch_gumbel_argmax(c, logits_out, M, V, R, *sa, st))) return s;
   prof_mark(c, st, "lm_head");
   return PS_OK;
 }

@@ -312,6 +312,35 @@ __global__ void __launch_bounds__(256) k_row_stats(const float* logits, int V, i
   }
 }
 
+// Gumbel-max token of each row of stored logits (draft sampling on the paths that keep logits
+// in memory).  One block per row.
+__global__ void __launch_bounds__(256) k_gumbel_argmax(const float* logits, int V, int R, SampleArgs sa) {
+  __shared__ float s_v[8];
+  __shared__ int s_i[8];
+  const int m = blockIdx.x, b = m / R, j = m - b * R;
+  const uint32_t row_id = (uint32_t)b | ((uint32_t)j << 8);
+  const float* row = logits + (size_t)m * V;
+  float bv = -FLT_MAX;
+  int bi = 0x7fffffff;
+  for (int v = threadIdx.x; v < V; v += blockDim.x) {
+    const float y = row[v] * sa.inv_temp + gumbel_noise(sa, (uint32_t)v, row_id);
+    if (y > bv || (y == bv && v < bi)) { bv = y; bi = v; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+  }
+  if ((threadIdx.x & 31) == 0) { s_v[threadIdx.x >> 5] = bv; s_i[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w)
+      if (s_v[w] > bv || (s_v[w] == bv && s_i[w] < bi)) { bv = s_v[w]; bi = s_i[w]; }
+    sa.sampled[m] = bi;
+  }
+}
+
 template <typename WT>
 __global__ void k_kv_copy(WT* kcache, WT* vcache, WT* K, WT* V, int slot, int len, int n_kv_heads,
                           int d, int max_ctx, int to_cache) {
@@ -373,7 +402,7 @@ template <typename WT>
 ps_status draft_impl(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last,
                      const int* token_last, int top_n, int* top_ids, float* top_logit,
                      float* row_max, float* row_lse, float* logits_out, float* feat_out,
-                     cudaStream_t st) {
+                     const SampleArgs* sa, cudaStream_t st) {
   const ps_config& g = c->cfg;
   const ps_weights& w = c->w;
   int H = g.hidden, Hq = g.n_heads * g.head_dim, F = g.ffn, V = g.vocab;
@@ -409,6 +438,7 @@ ps_status draft_impl(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last
     k_row_stats<<<M, 256, 0, st>>>(logits, V, top_n, top_ids, top_logit, row_max, row_lse);
     c->launches++;
   }
+  if (sa && (s = launch_gumbel_argmax(c, logits, M, V, g.k_masks + 1, *sa, st))) return s;
   prof_mark(c, st, "lm_head");
   return cuda_check(c, cudaGetLastError(), "draft_step");
 }
@@ -425,12 +455,19 @@ ps_status plain_kv_append(ps_ctx* c, const SeqMap& sm, int rows, const void* hid
 ps_status plain_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last,
                            const int* token_last, int top_n, int* top_ids, float* top_logit,
                            float* row_max, float* row_lse, float* logits_out, float* feat_out,
-                           cudaStream_t st) {
+                           const SampleArgs* sa, cudaStream_t st) {
   return c->cfg.dtype == PS_DTYPE_F32
              ? draft_impl<float>(c, sm, B, hidden_last, token_last, top_n, top_ids, top_logit,
-                                 row_max, row_lse, logits_out, feat_out, st)
+                                 row_max, row_lse, logits_out, feat_out, sa, st)
              : draft_impl<__nv_bfloat16>(c, sm, B, hidden_last, token_last, top_n, top_ids,
-                                         top_logit, row_max, row_lse, logits_out, feat_out, st);
+                                         top_logit, row_max, row_lse, logits_out, feat_out, sa, st);
+}
+
+ps_status launch_gumbel_argmax(ps_ctx* c, const float* logits, int M, int V, int R, const SampleArgs& sa,
+                               cudaStream_t st) {
+  k_gumbel_argmax<<<M, 256, 0, st>>>(logits, V, R, sa);
+  c->launches++;
+  return cuda_check(c, cudaGetLastError(), "k_gumbel_argmax");
 }
 
 ps_status launch_kv_copy(ps_ctx* c, int slot, int len, void* K, void* V, bool to_cache,

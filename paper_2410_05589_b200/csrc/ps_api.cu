@@ -313,10 +313,10 @@ ps_status ps_kv_append(ps_ctx* c, int B, const int* seq_slot, const int* n_new,
   return PS_OK;
 }
 
-ps_status ps_draft_step(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,
-                        const int* token_last, int top_n, int* top_ids, float* top_logit,
-                        float* row_max, float* row_lse, float* logits_out, float* feat_out,
-                        void* stream) {
+static ps_status draft_common(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,
+                              const int* token_last, int top_n, int* top_ids, float* top_logit,
+                              float* row_max, float* row_lse, float* logits_out, float* feat_out,
+                              const SampleArgs* sa, void* stream) {
   if (!c) return PS_ERR_INVALID_ARG;
   ps_status s = check_slots(c, B, seq_slot);
   if (s != PS_OK) return s;
@@ -337,9 +337,34 @@ ps_status ps_draft_step(ps_ctx* c, int B, const int* seq_slot, const void* hidde
   sm.row_off[B] = B * R;
   if (fused_supported(c, B * R))
     return fused_draft_step(c, sm, B, hidden_last, token_last, top_n, top_ids, top_logit, row_max,
-                            row_lse, logits_out, feat_out, (cudaStream_t)stream);
+                            row_lse, logits_out, feat_out, sa, (cudaStream_t)stream);
   return plain_draft_step(c, sm, B, hidden_last, token_last, top_n, top_ids, top_logit, row_max,
-                          row_lse, logits_out, feat_out, (cudaStream_t)stream);
+                          row_lse, logits_out, feat_out, sa, (cudaStream_t)stream);
+}
+
+ps_status ps_draft_step(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,
+                        const int* token_last, int top_n, int* top_ids, float* top_logit,
+                        float* row_max, float* row_lse, float* logits_out, float* feat_out,
+                        void* stream) {
+  return draft_common(c, B, seq_slot, hidden_last, token_last, top_n, top_ids, top_logit, row_max, row_lse,
+                      logits_out, feat_out, nullptr, stream);
+}
+
+ps_status ps_draft_step_sampled(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,
+                                const int* token_last, float temperature, uint64_t seed, uint64_t offset,
+                                int* sampled_ids, int top_n, int* top_ids, float* top_logit,
+                                float* row_max, float* row_lse, float* logits_out, float* feat_out,
+                                void* stream) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  if (!sampled_ids) return fail(c, PS_ERR_INVALID_ARG, "null sampled_ids");
+  if (!(temperature > 0.f)) return fail(c, PS_ERR_INVALID_ARG, "temperature must be > 0 (use the arg-max of ps_draft_step at 0)");
+  SampleArgs sa;
+  sa.inv_temp = 1.f / temperature;
+  sa.key0 = (uint32_t)seed ^ 0x6D756247u; sa.key1 = (uint32_t)(seed >> 32);
+  sa.off_lo = (uint32_t)offset; sa.off_hi = (uint32_t)(offset >> 32);
+  sa.sampled = sampled_ids;
+  return draft_common(c, B, seq_slot, hidden_last, token_last, top_n, top_ids, top_logit, row_max, row_lse,
+                      logits_out, feat_out, &sa, stream);
 }
 
 ps_status ps_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draft_tokens,

@@ -63,6 +63,35 @@ cudaError_t launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
+// Philox-4x32 with 10 rounds (Salmon et al., SC'11): counter (c0..c3), key (k0, k1).
+__device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t (&c)[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0 = __umulhi(0xD2511F53u, c[0]), lo0 = 0xD2511F53u * c[0];
+    uint32_t hi1 = __umulhi(0xCD9E8D57u, c[2]), lo1 = 0xCD9E8D57u * c[2];
+    uint32_t n0 = hi1 ^ c[1] ^ k0, n2 = hi0 ^ c[3] ^ k1;
+    c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+}
+
+// Draft sampling (Algorithm 1: the tree is drafted by sampling from the parallel drafter): the
+// token of a row is the arg-max over v of logit_v / T + G(v, row), G = -ln(-ln u) (the
+// Gumbel-max rule), u = ((w >> 8) + 0.5) / 2^24 with w = word 0 of Philox, key = (seed_lo ^
+// 0x6D756247, seed_hi), counter = (v, row_id, offset); row_id = b | j << 8.
+struct SampleArgs {
+  float inv_temp;
+  uint32_t key0, key1, off_lo, off_hi;
+  int* sampled;   // [B][k+1]
+};
+__device__ __forceinline__ float gumbel_noise(const SampleArgs& sa, uint32_t v, uint32_t row_id) {
+  uint32_t c[4] = {v, row_id, sa.off_lo, sa.off_hi};
+  philox4x32_10(sa.key0, sa.key1, c);
+  const double u = ((double)(c[0] >> 8) + 0.5) * (1.0 / 16777216.0);
+  return (float)(-log(-log(u)));   // in double: u may sit within 2^-25 of 1
+}
+
 // Device status word values (bit flags).
 constexpr int kStatNonfinite = 1;
 constexpr int kStatTimeout = 2;
@@ -129,7 +158,10 @@ ps_status plain_kv_append(ps_ctx* c, const SeqMap& sm, int rows, const void* hid
 ps_status plain_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last,
                            const int* token_last, int top_n, int* top_ids, float* top_logit,
                            float* row_max, float* row_lse, float* logits_out, float* feat_out,
-                           cudaStream_t st);
+                           const SampleArgs* sa, cudaStream_t st);
+// One block per row of stored logits [M][V]: the Gumbel-max token of the row (R rows per sequence).
+ps_status launch_gumbel_argmax(ps_ctx* c, const float* logits, int M, int V, int R, const SampleArgs& sa,
+                               cudaStream_t st);
 // ---- fused bf16 kernels for small M ---------------------------------------------------------
 bool fused_supported(ps_ctx* c, int M);
 size_t fused_scratch_bytes(const ps_config& g);
@@ -142,7 +174,7 @@ ps_status launch_attn_split(ps_ctx* c, const SeqMap& sm, int B, const float* qkv
 ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last,
                            const int* token_last, int top_n, int* top_ids, float* top_logit,
                            float* row_max, float* row_lse, float* logits_out, float* feat_out,
-                           cudaStream_t st);
+                           const SampleArgs* sa, cudaStream_t st);
 ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draft_tokens,
                         const float* draft_logits, const float* target_logits, float temperature,
                         uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,

@@ -20,19 +20,6 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kSeg = 128;  // elements per warp-wide segment of the inverse-CDF search
 
-// Philox-4x32 with 10 rounds (Salmon et al., SC'11): counter (c0..c3), key (k0,k1).
-__device__ __forceinline__ void philox4x32_10(uint32_t k0, uint32_t k1, uint32_t (&c)[4]) {
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    uint32_t hi0 = __umulhi(0xD2511F53u, c[0]), lo0 = 0xD2511F53u * c[0];
-    uint32_t hi1 = __umulhi(0xCD9E8D57u, c[2]), lo1 = 0xCD9E8D57u * c[2];
-    uint32_t n0 = hi1 ^ c[1] ^ k0, n2 = hi0 ^ c[3] ^ k1;
-    c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
-  }
-}
-
 __global__ void k_philox_fill(uint32_t k0, uint32_t k1, const uint32_t* ctr, uint32_t* out, int n) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
