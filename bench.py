@@ -34,7 +34,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="13b", choices=["13b", "7b", "33b", "tiny", "mini"])
+    ap.add_argument("--workload", default="13b", choices=["13b", "7b", "33b", "llama3_8b", "tiny", "mini"])
     ap.add_argument("--temperature", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
@@ -447,7 +447,7 @@ def main():
 
     # ---- token-tree verification (Algorithm 1 in full), timed on its own ---------------------
     tree = None
-    if V % 4 == 0 and V <= 65536 and s.dtype == 1:
+    if V % 4 == 0 and V <= 131072 and s.dtype == 1:
         tree = tree_verify_leg(g, ps, s, B, T, peak)
 
     # ---- end to end through the host-buffer entry point -----------------------------------

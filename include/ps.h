@@ -204,7 +204,7 @@ ps_status ps_verify(ps_ctx* ctx, int B, int n_draft, int n_target, const int* dr
  *   out_tokens    device [B][D+1] int32: their tokens, then the drawn token, then -1
  *   n_out         device [B] int32 = accept_len + 1
  *   path          device [B][D] int32: the accepted nodes' ids, then -1
- * Needs vocab % 4 == 0, vocab <= 65536 and 16-byte aligned logits (PS_ERR_UNSUPPORTED
+ * Needs vocab % 4 == 0, vocab <= 131072 and 16-byte aligned logits (PS_ERR_UNSUPPORTED
  * otherwise).  Non-finite logits in an examined row: the walk stops there with the arg-max of
  * that target row and ps_poll reports PS_ERR_NONFINITE. */
 ps_status ps_verify_tree(ps_ctx* ctx, int B, int n_nodes, const int* parent, const int* tokens,

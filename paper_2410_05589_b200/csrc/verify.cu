@@ -320,7 +320,8 @@ constexpr int kClu = 8;
 constexpr int kCluThreads = 512;
 constexpr int kCluWarps = kCluThreads / 32;
 constexpr int kCluV4 = 4;  // float4 per thread and row: up to kClu * kCluThreads * 16 tokens
-constexpr int kCluMaxVocab = kClu * kCluThreads * 4 * kCluV4;
+constexpr int kCluMaxVocab = kClu * kCluThreads * 4 * kCluV4;        // with the portable cluster size
+constexpr int kCluMaxVocab16 = 16 * kCluThreads * 4 * kCluV4;         // with 16 blocks (opt-in size)
 
 struct CluPart {       // one per block, read by the whole cluster
   float tmax, dmax;
@@ -336,14 +337,15 @@ struct CluScratch {
   double d[kCluWarps], d2[kCluWarps];
 };
 
-__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads)
-k_verify_cluster(VerifyArgs a) {
+// (The cluster size is a launch attribute: 8 blocks, 16 for vocabularies beyond 65536.)
+__global__ void __launch_bounds__(kCluThreads) k_verify_cluster(VerifyArgs a) {
   namespace cg = cooperative_groups;
   cg::cluster_group cl = cg::this_cluster();
   __shared__ CluPart part;
   __shared__ CluScratch s;
   const int rank = (int)cl.block_rank();
-  const int i = blockIdx.x / kClu, b = blockIdx.y, V = a.V;
+  const int nclu = (int)cl.num_blocks();
+  const int i = blockIdx.x / nclu, b = blockIdx.y, V = a.V;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool bonus = i >= a.n_draft;
   const float* trow = a.target_logits + ((size_t)b * a.n_target + i) * V;
@@ -351,7 +353,7 @@ k_verify_cluster(VerifyArgs a) {
   const float* drow = (!bonus && !greedy && a.draft_logits)
                           ? a.draft_logits + ((size_t)b * a.n_draft + i) * V : nullptr;
   const int x = bonus ? -1 : a.draft_tokens[(size_t)b * a.n_draft + i];
-  const int nv4 = ((V + kClu * kCluThreads - 1) / (kClu * kCluThreads) + 3) / 4;
+  const int nv4 = ((V + nclu * kCluThreads - 1) / (nclu * kCluThreads) + 3) / 4;
   const int C = nv4 * 4, v0 = (rank * kCluThreads + tid) * C;
 
   float t[kCluV4 * 4], d[kCluV4 * 4];
@@ -407,7 +409,7 @@ k_verify_cluster(VerifyArgs a) {
   }
   cl.sync();
   tm = -INFINITY; dm = -INFINITY; ti = 0x7fffffff; bad = 0;
-  for (int r = 0; r < kClu; ++r) {
+  for (int r = 0; r < nclu; ++r) {
     const CluPart* pr = cl.map_shared_rank(&part, r);
     const float ov = pr->tmax;
     const int oi = pr->targ;
@@ -451,7 +453,7 @@ k_verify_cluster(VerifyArgs a) {
     }
     cl.sync();
     st = 0.0; sd = 0.0;
-    for (int r = 0; r < kClu; ++r) {
+    for (int r = 0; r < nclu; ++r) {
       const CluPart* pr = cl.map_shared_rank(&part, r);
       st += pr->st; sd += pr->sd;
     }
@@ -507,12 +509,12 @@ k_verify_cluster(VerifyArgs a) {
         cl.sync();
         // level 1: the block whose running sum first exceeds the target
         double total = 0.0;
-        for (int rr = 0; rr < kClu; ++rr) total += cl.map_shared_rank(&part, rr)->wsum;
+        for (int rr = 0; rr < nclu; ++rr) total += cl.map_shared_rank(&part, rr)->wsum;
         int sel = -1;
         if (total > 0.0) {
           const double target = u2 * total;
           double run = 0.0, base = 0.0;
-          for (int rr = 0; rr < kClu; ++rr) {
+          for (int rr = 0; rr < nclu; ++rr) {
             const double nx = run + cl.map_shared_rank(&part, rr)->wsum;
             if (sel < 0 && nx > target) { sel = rr; base = run; }
             run = nx;
@@ -555,7 +557,7 @@ k_verify_cluster(VerifyArgs a) {
           // rounding may leave no token chosen on the way down: take the last one with weight
           token = sel >= 0 ? cl.map_shared_rank(&part, sel)->pick : -1;
           if (token < 0)
-            for (int rr = 0; rr < kClu; ++rr) token = max(token, cl.map_shared_rank(&part, rr)->lastp);
+            for (int rr = 0; rr < nclu; ++rr) token = max(token, cl.map_shared_rank(&part, rr)->lastp);
         }
         cl.sync();   // all reads of this attempt's partials are done before they are rewritten
       }
@@ -887,6 +889,46 @@ __global__ void __launch_bounds__(kCluThreads) k_verify_tree(TreeArgs a) {
 
 }  // namespace
 
+// Launch with a cluster of nclu blocks along x (a launch attribute, not a compile-time one).
+template <class Args>
+cudaError_t launch_cluster(void (*kern)(Args), dim3 grid, int nclu, cudaStream_t st, const Args& a) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kCluThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = nclu; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+// Whether the device can co-schedule nclu blocks of this kernel as one cluster (sizes above 8
+// are an opt-in of the kernel).  Asked once per size.
+template <class Args>
+bool cluster_size_ok(void (*kern)(Args), int nclu) {
+  static int ok[17] = {0};   // 0 unknown, 1 yes, -1 no
+  if (nclu <= 8) return true;
+  if (ok[nclu] == 0) {
+    ok[nclu] = -1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(nclu);
+      cfg.blockDim = dim3(kCluThreads);
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = nclu; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      cfg.attrs = at;
+      cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0) ok[nclu] = 1;
+    }
+    (void)cudaGetLastError();
+  }
+  return ok[nclu] > 0;
+}
+
 ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draft_tokens,
                         const float* draft_logits, const float* target_logits, float temperature,
                         uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,
@@ -900,13 +942,14 @@ ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* 
   a.accept_len = accept_len; a.out_tokens = out_tokens; a.n_out = n_out;
   a.rec = c->vrec; a.tickets = c->tickets; a.status = c->dev_status;
   const bool aligned = (((uintptr_t)target_logits | (uintptr_t)draft_logits) & 15u) == 0;
-  if (a.V % 4 == 0 && a.V <= kCluMaxVocab && aligned) {
+  const int nclu = a.V <= kCluMaxVocab ? kClu : 16;
+  if (a.V % 4 == 0 && a.V <= kCluMaxVocab16 && aligned && cluster_size_ok(k_verify_cluster, nclu)) {
     prof_mark(c, st, "begin");
     // (a plain launch: joining the dependent-launch chain here was measured to cost 7 us a step)
-    k_verify_cluster<<<dim3(n_target * kClu, B), kCluThreads, 0, st>>>(a);
+    cudaError_t e = launch_cluster(k_verify_cluster, dim3(n_target * nclu, B), nclu, st, a);
     c->launches++;
     prof_mark(c, st, "verify");
-    return cuda_check(c, cudaGetLastError(), "k_verify_cluster");
+    return cuda_check(c, e, "k_verify_cluster");
   }
   size_t smem = (size_t)((a.V + kSeg - 1) / kSeg) * sizeof(double);
   if (smem > 160 * 1024) return fail(c, PS_ERR_UNSUPPORTED, "vocab too large for ps_verify");
@@ -945,8 +988,8 @@ ps_status launch_verify_tree(ps_ctx* c, int B, int n_nodes, const int* parent, c
   if (max_depth_out) *max_depth_out = tp.max_depth;
   if (temperature != 0.f && !draft_logits) return fail(c, PS_ERR_INVALID_ARG, "draft_logits needed at temperature > 0");
   const bool aligned = (((uintptr_t)target_logits | (uintptr_t)draft_logits) & 15u) == 0;
-  if (a.V % 4 || a.V > kCluMaxVocab || !aligned)
-    return fail(c, PS_ERR_UNSUPPORTED, "ps_verify_tree needs vocab % 4 == 0, vocab <= 65536 and 16-byte aligned logits");
+  if (a.V % 4 || a.V > kCluMaxVocab16 || !aligned)
+    return fail(c, PS_ERR_UNSUPPORTED, "ps_verify_tree needs vocab % 4 == 0, vocab <= 131072 and 16-byte aligned logits");
   a.tokens = tokens; a.draft_logits = draft_logits; a.target_logits = target_logits;
   a.temperature = temperature;
   a.key0 = (uint32_t)seed; a.key1 = (uint32_t)(seed >> 32);
@@ -954,21 +997,14 @@ ps_status launch_verify_tree(ps_ctx* c, int B, int n_nodes, const int* parent, c
   a.accept_len = accept_len; a.out_tokens = out_tokens; a.n_out = n_out; a.path = path;
   a.rec = c->trec; a.tickets = c->tree_tickets; a.status = c->dev_status;
   prof_mark(c, st, "begin");
-  // blocks per decision row: as many as fit in one wave of the device, at most 8, and enough for
-  // each thread to hold its share of a row (16 tokens)
-  int nclu = kClu;
+  // blocks per decision row: 8 (16 for vocabularies beyond 65536), fewer when the tree would
+  // otherwise need a second wave of blocks and a thread can still hold its share of a row
+  int nclu = a.V <= kCluMaxVocab ? kClu : 16;
+  if (!cluster_size_ok(k_verify_tree, nclu))
+    return fail(c, PS_ERR_UNSUPPORTED, "this device cannot run the 16-block clusters a vocabulary beyond 65536 needs");
   while (nclu > 1 && (long)(n_nodes + 1) * B * nclu > c->n_sm && a.V <= (nclu / 2) * kCluThreads * 4 * kCluV4)
     nclu /= 2;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((n_nodes + 1) * nclu, B);
-  cfg.blockDim = dim3(kCluThreads);
-  cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = nclu; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  cfg.attrs = at;
-  cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, k_verify_tree, a);
+  cudaError_t e = launch_cluster(k_verify_tree, dim3((n_nodes + 1) * nclu, B), nclu, st, a);
   c->launches++;
   prof_mark(c, st, "verify_tree");
   return cuda_check(c, e, "k_verify_tree");

@@ -59,6 +59,10 @@ CONFIGS = {
     "13b_sweep": ModelShape("13b_sweep", 1, 5120, 40, 40, 128, 13824, 32000, 8, 64, 256, 2048, 4000, 1.0, "zipf"),
     # 33B-class
     "33b": ModelShape("33b", 1, 6656, 52, 52, 128, 17920, 32000, 8, 16, 1024, 4096, 5000, 1.0, "zipf"),
+    # Llama-3-8B-shaped: grouped-query attention (8 KV heads) and a 128k vocabulary, where the
+    # LM head is two thirds of the bytes (Sec. 2 names the 128,000+ vocabularies of Llama-3)
+    "llama3_8b": ModelShape("llama3_8b", 1, 4096, 32, 8, 128, 14336, 128256, 4, 1, 1024, 1024, 6000, 1.0,
+                            "zipf", rope_base=500000.0),
     # small bf16 shape for element-by-element parity in seconds (several tiles, ragged tails)
     "mini": ModelShape("mini", 1, 768, 6, 6, 128, 2072, 5000, 4, 3, 37, 203, 7000, 1.0, "zipf"),
     # small fp32 shape with odd sizes

@@ -136,9 +136,10 @@ def test_argument_errors_return_status():
                    k_masks=1, max_batch=1, max_ctx=8, weights={})
 
 
-@pytest.mark.parametrize("name", ["7b", "13b"])
+@pytest.mark.parametrize("name", ["7b", "13b", "llama3_8b"])
 def test_full_size_batch1(name):
-    """The 7B- and 13B-shaped batch-1 workloads at full size; context built by ps_kv_append on
+    """The 7B-, 13B- and Llama-3-8B-shaped (grouped-query attention, 128k vocabulary) batch-1
+    workloads at full size; context built by ps_kv_append on
     the GPU and imported into the oracle (appends are checked above), oracle rows one by one."""
     s = synth.CONFIGS[name]
     p = Pair(s, 1, context="import", extra_ctx=8)

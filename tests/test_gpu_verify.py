@@ -73,11 +73,12 @@ def test_device_philox_equals_oracle_words():
 
 
 @pytest.mark.parametrize("V,n_draft,bonus", [(1000, 5, 0), (1000, 4, 1), (5003, 3, 1), (130, 1, 0),
-                                            (32000, 4, 1), (65536, 2, 1), (8, 1, 1), (65540, 1, 1)])
+                                            (32000, 4, 1), (65536, 2, 1), (8, 1, 1), (65540, 1, 1), (128256, 2, 1),
+                                            (131070, 1, 1)])
 @pytest.mark.parametrize("T", [1.0, 0.6])
 def test_stochastic_verify_matches_oracle(V, n_draft, bonus, T):
-    # vocabularies that are a multiple of 4 up to 65536 take the cluster kernel, the rest the
-    # one-block-per-row kernel
+    # vocabularies that are a multiple of 4 take the cluster kernel (8 blocks per row up to 65536,
+    # 16 up to 131072), the rest the one-block-per-row kernel
     B = 96 if V < 20000 else 24
     g = _ctx(V)
     tl = synth.gauss_logits(1, ("t", V), (B, n_draft + bonus, V))

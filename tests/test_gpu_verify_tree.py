@@ -65,16 +65,17 @@ def _assert_same(got, want):
     assert excused <= max(1, B // 100), excused
 
 
-@pytest.mark.parametrize("V", [1000, 32000])
+@pytest.mark.parametrize("V", [1000, 32000, 128256])
 @pytest.mark.parametrize("T", [1.0, 0.6])
 def test_tree_verify_matches_oracle(V, T):
-    B = 64 if V < 20000 else 16
+    B = 64 if V < 20000 else (16 if V < 100000 else 4)
     g = _ctx(V)
     toks, dl, tl = _case(TREE26, B, V, seed=2, T=T)
     got, want = _run_both(g, TREE26, toks, dl, tl, T, seed=1, offset=3)
     _assert_same(got, want)
-    assert want["accept_len"].max() >= 2 and want["accept_len"].min() == 0   # deep and empty paths
-    assert (want["path"][:, 0] > 0).any()                                   # a later sibling was taken
+    if B >= 16:
+        assert want["accept_len"].max() >= 2 and want["accept_len"].min() == 0   # deep and empty paths
+        assert (want["path"][:, 0] > 0).any()                                   # a later sibling was taken
     # second call, new offset: the scratch (tickets) was left clean by the first
     got, want = _run_both(g, TREE26, toks, dl, tl, T, seed=1, offset=4)
     _assert_same(got, want)
