@@ -48,7 +48,10 @@ enum { PS_DTYPE_F32 = 0, PS_DTYPE_BF16 = 1 };
 enum {
   PS_FLAG_FC_BIAS = 1,          /* ps_weights.b_fc is used */
   PS_FLAG_UNFUSED_KERNELS = 2,  /* force the unfused fp32-activation kernels (debugging aid) */
-  PS_FLAG_MMA_SYNC_GEMM = 4     /* fused path: mma.sync GEMM kernels instead of the tcgen05 ones */
+  PS_FLAG_MMA_SYNC_GEMM = 4,    /* fused path: mma.sync GEMM kernels instead of the tcgen05 ones */
+  PS_FLAG_NO_FC = 8             /* embedding-only input (the Medusa integration, Sec. 4.2): x0 is the token /
+                                   [MASK] embedding, there is no fc layer and no target feature; w_fc,
+                                   mask_feat and every `hidden` argument are ignored and may be NULL */
 };
 enum { PS_MAX_BATCH = 128, PS_MAX_MASKS = 15, PS_MAX_TOP_N = 8 };
 enum { PS_MAX_TREE_NODES = 64 };  /* nodes of a token tree (ps_verify_tree) */

@@ -49,6 +49,7 @@ struct Config {
   int max_batch, max_ctx;
   double rope_base, rms_eps;
   int has_fc_bias;
+  int no_fc;  // embedding-only input (the Medusa integration of Sec. 4.2): x0 = the embedding half
 };
 
 struct Weights {
@@ -135,8 +136,11 @@ void rope(double* v, int d, long long pos, double base) {
 // fc over [embedding ; feature] followed by the pre-attention norm.
 void fuse_and_norm(const Ctx& C, const double* x_in, double* x0, double* xn) {
   const Config& c = C.c;
-  matvec(C.w.w_fc, c.has_fc_bias ? C.w.b_fc : nullptr, c.dtype, c.hidden, 2 * (size_t)c.hidden,
-         x_in, x0);
+  if (c.no_fc)
+    for (int i = 0; i < c.hidden; ++i) x0[i] = x_in[i];
+  else
+    matvec(C.w.w_fc, c.has_fc_bias ? C.w.b_fc : nullptr, c.dtype, c.hidden, 2 * (size_t)c.hidden,
+           x_in, x0);
   rmsnorm(x0, C.w.g_in, c.dtype, c.hidden, c.rms_eps, xn);
 }
 

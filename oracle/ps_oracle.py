@@ -40,7 +40,7 @@ class _Config(C.Structure):
         ("dtype", C.c_int), ("hidden", C.c_int), ("n_heads", C.c_int), ("n_kv_heads", C.c_int),
         ("head_dim", C.c_int), ("ffn", C.c_int), ("vocab", C.c_int), ("k_masks", C.c_int),
         ("max_batch", C.c_int), ("max_ctx", C.c_int), ("rope_base", C.c_double),
-        ("rms_eps", C.c_double), ("has_fc_bias", C.c_int),
+        ("rms_eps", C.c_double), ("has_fc_bias", C.c_int), ("no_fc", C.c_int),
     ]
 
 
@@ -100,6 +100,7 @@ class OracleConfig:
     max_ctx: int
     rope_base: float = 10000.0
     rms_eps: float = 1e-5
+    no_fc: bool = False   # embedding-only input: no fc layer, no target feature
 
 
 class Oracle:
@@ -123,7 +124,7 @@ class Oracle:
         c = _Config(
             cfg.dtype, cfg.hidden, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
             cfg.k_masks, cfg.max_batch, cfg.max_ctx, cfg.rope_base, cfg.rms_eps,
-            1 if weights.get("b_fc") is not None else 0,
+            1 if weights.get("b_fc") is not None else 0, 1 if cfg.no_fc else 0,
         )
         self._h = lib.pso_create(C.byref(c), C.byref(w))
 

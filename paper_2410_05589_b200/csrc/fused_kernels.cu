@@ -1048,6 +1048,37 @@ __global__ void k_gather_x(const __nv_bfloat16* __restrict__ embed, const __nv_b
   }
 }
 
+// Embedding-only input (PS_FLAG_NO_FC): x0 = embedding(token) for a sequence's first row, the
+// learned [MASK] embeddings after it; also the planes of x0 * g_in and each row's sum of
+// squares (one partial per row).  One block per row.
+__global__ void __launch_bounds__(256) k_embed_x0(const __nv_bfloat16* __restrict__ embed,
+                                                  const __nv_bfloat16* __restrict__ mask_embed,
+                                                  const int* __restrict__ tokens, const __nv_bfloat16* __restrict__ g_in,
+                                                  int H, int V, int R, float* __restrict__ x0,
+                                                  __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                  float* __restrict__ ssq) {
+  __shared__ float s_part[8];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int m = blockIdx.x, b = m / R, j = m - b * R;
+  const __nv_bfloat16* e = j == 0 ? embed + (size_t)min(max(tokens[b], 0), V - 1) * H : mask_embed + (size_t)(j - 1) * H;
+  float ss = 0.f;
+  for (int n = threadIdx.x; n < H; n += blockDim.x) {
+    const float x = __bfloat162float(e[n]);
+    x0[(size_t)m * H + n] = x;
+    split_store(hi + (size_t)m * H + n, lo + (size_t)m * H + n, x * __bfloat162float(g_in[n]));
+    ss += x * x;
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+    for (int w = 0; w < 8; ++w) tot += s_part[w];
+    ssq[m] = tot;
+  }
+}
+
 // ---- host side: tensor maps ---------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1090,7 +1121,10 @@ UmmaMaps* build_maps(const ps_ctx* c, const FusedScratch& f) {
   const size_t H = g.hidden, Hq = (size_t)g.n_heads * g.head_dim, Hkv = (size_t)g.n_kv_heads * g.head_dim,
                F = g.ffn, V = g.vocab;
   UmmaMaps* u = new UmmaMaps;
-  bool ok = make_map(&u->w_fc, w.w_fc, H, 2 * H, 128) && make_map(&u->w_q, w.w_q, Hq, H, 128) &&
+  // (an embedding-only drafter has no fc matrix: its map is never used, w_q stands in)
+  const bool no_fc = (g.flags & PS_FLAG_NO_FC) != 0;
+  bool ok = (no_fc ? make_map(&u->w_fc, w.w_q, Hq, H, 128) : make_map(&u->w_fc, w.w_fc, H, 2 * H, 128)) &&
+            make_map(&u->w_q, w.w_q, Hq, H, 128) &&
             make_map(&u->w_k, w.w_k, Hkv, H, 128) && make_map(&u->w_v, w.w_v, Hkv, H, 128) &&
             make_map(&u->w_o, w.w_o, H, Hq, 128) && make_map(&u->w_gate, w.w_gate, F, H, 64) &&
             make_map(&u->w_up, w.w_up, F, H, 64) && make_map(&u->w_down, w.w_down, H, F, 128) &&
@@ -1148,24 +1182,32 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
   const int tiles_h = (H + umma::kTile - 1) / umma::kTile;
   ps_status s;
   prof_mark(c, st, "begin");
-  cudaError_t ge = launch_after(k_gather_x, dim3(M), dim3(256), 0, st, !c->prof, (BP)w.embed, (BP)w.mask_embed,
-                                (BP)w.mask_feat, (BP)hidden_last, token_last, H, V, R, f.xin);
-  c->launches++;
-  if (ge != cudaSuccess) return cuda_check(c, ge, "k_gather_x");
-  {  // S1 fc: x0 = W_fc [e ; f] (+ b)
-    UArgs a{};
-    a.N = H; a.K = 2 * H; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 0;
-    a.out = c->x0; a.ldo = H; a.bias = (g.flags & PS_FLAG_FC_BIAS) ? (BP)w.b_fc : nullptr;
-    a.ssq_out = f.ssq[0];
-    a.out_hi = f.x0p.hi; a.out_lo = f.x0p.lo; a.ld_plane = H; a.gain_next = (BP)w.g_in;
-    if ((s = launch_umma<EPI_STORE>(c, u.w_fc, u.w_fc, u.w_fc, u.xin, u.xin, a, f, st))) return s;
+  const bool no_fc = (g.flags & PS_FLAG_NO_FC) != 0;
+  if (no_fc) {   // embedding-only input: x0 and its planes come straight from the embedding rows
+    cudaError_t ee = launch_after(k_embed_x0, dim3(M), dim3(256), 0, st, !c->prof, (BP)w.embed, (BP)w.mask_embed,
+                                  token_last, (BP)w.g_in, H, V, R, c->x0, f.x0p.hi, f.x0p.lo, f.ssq[0]);
+    c->launches++;
+    if (ee != cudaSuccess) return cuda_check(c, ee, "k_embed_x0");
+  } else {
+    cudaError_t ge = launch_after(k_gather_x, dim3(M), dim3(256), 0, st, !c->prof, (BP)w.embed, (BP)w.mask_embed,
+                                  (BP)w.mask_feat, (BP)hidden_last, token_last, H, V, R, f.xin);
+    c->launches++;
+    if (ge != cudaSuccess) return cuda_check(c, ge, "k_gather_x");
+    {  // S1 fc: x0 = W_fc [e ; f] (+ b)
+      UArgs a{};
+      a.N = H; a.K = 2 * H; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 0;
+      a.out = c->x0; a.ldo = H; a.bias = (g.flags & PS_FLAG_FC_BIAS) ? (BP)w.b_fc : nullptr;
+      a.ssq_out = f.ssq[0];
+      a.out_hi = f.x0p.hi; a.out_lo = f.x0p.lo; a.ld_plane = H; a.gain_next = (BP)w.g_in;
+      if ((s = launch_umma<EPI_STORE>(c, u.w_fc, u.w_fc, u.w_fc, u.xin, u.xin, a, f, st))) return s;
+    }
   }
   prof_mark(c, st, "fc_norm");
   {  // S2 q|k|v = W rms(x0)
     UArgs a{};
     a.N = Hq + 2 * Hkv; a.K = H; a.M = M; a.n_mats = 3;
     a.mat_rows[0] = Hq; a.mat_rows[1] = Hkv; a.mat_rows[2] = Hkv; a.lo = 1;
-    a.ssq_in = f.ssq[0]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
+    a.ssq_in = f.ssq[0]; a.ssq_n = no_fc ? 1 : tiles_h; a.eps = g.rms_eps;
     a.out = f.qkv; a.ldo = Hq + 2 * Hkv;
     if ((s = launch_umma<EPI_STORE>(c, u.w_q, u.w_k, u.w_v, u.x0_hi, u.x0_lo, a, f, st))) return s;
   }
@@ -1285,7 +1327,12 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
                            top_ids, top_logit, row_max, row_lse, logits_out, feat_out, sa, st);
   ps_status s;
   prof_mark(c, st, "begin");
-  {  // S1 fc: x0 = W_fc [e ; f] (+ b)
+  const bool no_fc = (g.flags & PS_FLAG_NO_FC) != 0;
+  if (no_fc) {   // embedding-only input: x0 and its planes come straight from the embedding rows
+    k_embed_x0<<<M, 256, 0, st>>>((BP)w.embed, (BP)w.mask_embed, token_last, (BP)w.g_in, H, V, R, c->x0,
+                                  f.x0p.hi, f.x0p.lo, f.ssq[0]);
+    c->launches++;
+  } else {  // S1 fc: x0 = W_fc [e ; f] (+ b)
     GemmArgs a{};
     a.rs.W[0] = (BP)w.w_fc; a.rs.rows[0] = H; a.rs.n_mats = 1;
     a.N = H; a.K = 2 * H; a.M = M;
@@ -1303,7 +1350,7 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
     a.rs.rows[0] = Hq; a.rs.rows[1] = Hkv; a.rs.rows[2] = Hkv; a.rs.n_mats = 3;
     a.N = Hq + 2 * Hkv; a.K = H; a.M = M;
     a.in_hi = f.x0p.hi; a.in_lo = f.x0p.lo; a.ld_in = H;
-    a.ssq_in = f.ssq[0]; a.ssq_n = c->n_sm; a.eps = g.rms_eps;
+    a.ssq_in = f.ssq[0]; a.ssq_n = no_fc ? 1 : c->n_sm; a.eps = g.rms_eps;
     a.out = f.qkv; a.ldo = Hq + 2 * Hkv;
     if ((s = launch_gemm<false, EPI_STORE>(c, a, st))) return s;
   }

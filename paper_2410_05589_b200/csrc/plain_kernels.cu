@@ -61,7 +61,7 @@ __global__ void k_gather(SeqMap sm, int all_real, const WT* embed, const WT* mas
   float* out = x_in + (size_t)m * 2 * H;
   for (int i = threadIdx.x; i < H; i += blockDim.x) {
     out[i] = to_f32(e[i]);
-    out[H + i] = to_f32(f[i]);
+    out[H + i] = hidden ? to_f32(f[i]) : 0.f;   // embedding-only input: no feature half
   }
 }
 
@@ -377,12 +377,19 @@ ps_status fc_norm_kv(ps_ctx* c, const SeqMap& sm, int rows, int all_real, const 
   int H = g.hidden, Hq = g.n_heads * g.head_dim, Hkv = g.n_kv_heads * g.head_dim;
   prof_mark(c, st, "begin");
   k_gather<WT><<<rows, 256, 0, st>>>(sm, all_real, (const WT*)w.embed, (const WT*)w.mask_embed,
-                                     (const WT*)w.mask_feat, (const WT*)hidden, tokens, H, g.vocab,
+                                     (const WT*)w.mask_feat,
+                                     (g.flags & PS_FLAG_NO_FC) ? nullptr : (const WT*)hidden, tokens, H, g.vocab,
                                      c->x_in);
   c->launches++;
   ps_status s;
   const void* bias = (g.flags & PS_FLAG_FC_BIAS) ? w.b_fc : nullptr;
-  if ((s = linear<WT>(c, c->x_in, 2 * H, w.w_fc, bias, nullptr, 0, c->x0, H, rows, H, 2 * H, st))) return s;
+  if (g.flags & PS_FLAG_NO_FC) {   // x0 = the embedding half of x_in
+    cudaError_t e = cudaMemcpy2DAsync(c->x0, (size_t)H * 4, c->x_in, (size_t)2 * H * 4, (size_t)H * 4, rows,
+                                      cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) return cuda_check(c, e, "x0 copy");
+  } else if ((s = linear<WT>(c, c->x_in, 2 * H, w.w_fc, bias, nullptr, 0, c->x0, H, rows, H, 2 * H, st))) {
+    return s;
+  }
   k_rmsnorm<WT><<<rows, 256, 0, st>>>(c->x0, (const WT*)w.g_in, H, g.rms_eps, c->xn);
   c->launches++;
   prof_mark(c, st, "fc_norm");

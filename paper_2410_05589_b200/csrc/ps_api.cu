@@ -141,11 +141,13 @@ ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* w, void*
   if (s != PS_OK) return s;
   if (((uintptr_t)workspace & 255) != 0) return PS_ERR_INVALID_ARG;
   if (workspace_bytes < carve(*cfg, nullptr, nullptr)) return PS_ERR_CAPACITY;
-  const void* need[] = {w->embed, w->w_fc, w->g_in, w->w_q, w->w_k, w->w_v, w->w_o, w->g_post,
+  const bool no_fc = (cfg->flags & PS_FLAG_NO_FC) != 0;
+  const void* need[] = {w->embed, no_fc ? w->embed : w->w_fc, w->g_in, w->w_q, w->w_k, w->w_v, w->w_o, w->g_post,
                         w->w_gate, w->w_up, w->w_down, w->g_final, w->w_lm};
   for (const void* p : need)
     if (!p) return PS_ERR_INVALID_ARG;
-  if (cfg->k_masks > 0 && (!w->mask_embed || !w->mask_feat)) return PS_ERR_INVALID_ARG;
+  if (cfg->k_masks > 0 && (!w->mask_embed || (!w->mask_feat && !no_fc))) return PS_ERR_INVALID_ARG;
+  if (no_fc && (cfg->flags & PS_FLAG_FC_BIAS)) return PS_ERR_INVALID_ARG;
   if ((cfg->flags & PS_FLAG_FC_BIAS) && !w->b_fc) return PS_ERR_INVALID_ARG;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PS_ERR_CUDA;
@@ -293,7 +295,8 @@ ps_status ps_kv_append(ps_ctx* c, int B, const int* seq_slot, const int* n_new,
   }
   int total = row_offset[B];
   if (total == 0) return PS_OK;
-  if (!hidden || !tokens) return fail(c, PS_ERR_INVALID_ARG, "null hidden / tokens");
+  if ((!hidden && !(c->cfg.flags & PS_FLAG_NO_FC)) || !tokens)
+    return fail(c, PS_ERR_INVALID_ARG, "null hidden / tokens");
   SeqMap sm;
   std::memset(&sm, 0, sizeof(sm));
   sm.B = B;
@@ -320,7 +323,8 @@ static ps_status draft_common(ps_ctx* c, int B, const int* seq_slot, const void*
   if (!c) return PS_ERR_INVALID_ARG;
   ps_status s = check_slots(c, B, seq_slot);
   if (s != PS_OK) return s;
-  if (!hidden_last || !token_last) return fail(c, PS_ERR_INVALID_ARG, "null hidden / token");
+  if ((!hidden_last && !(c->cfg.flags & PS_FLAG_NO_FC)) || !token_last)
+    return fail(c, PS_ERR_INVALID_ARG, "null hidden / token");
   if (top_n < 0 || top_n > PS_MAX_TOP_N || top_n > c->cfg.vocab)
     return fail(c, PS_ERR_INVALID_ARG, "top_n out of range");
   if (top_n > 0 && (!top_ids || !top_logit)) return fail(c, PS_ERR_INVALID_ARG, "null top-n output");

@@ -8,9 +8,9 @@ import synth
 from oracle import Oracle, OracleConfig
 
 
-def oracle_for(s, W, max_batch, max_ctx):
+def oracle_for(s, W, max_batch, max_ctx, no_fc=False):
     return Oracle(OracleConfig(s.dtype, s.hidden, s.n_heads, s.n_kv_heads, s.head_dim, s.ffn,
-                               s.vocab, s.k_masks, max_batch, max_ctx, s.rope_base, s.rms_eps), W)
+                               s.vocab, s.k_masks, max_batch, max_ctx, s.rope_base, s.rms_eps, no_fc), W)
 
 
 def as_f64(a, dtype):
@@ -29,7 +29,7 @@ class Pair:
         self.lens = synth.ctx_lengths(s, B) if lens is None else np.asarray(lens, np.int32)
         max_ctx = int(self.lens.max()) + s.k_masks + 1 + extra_ctx
         self.oracle_seqs = list(range(B)) if oracle_seqs is None else list(oracle_seqs)
-        self.o = oracle_for(s, self.W, B, max_ctx)
+        self.o = oracle_for(s, self.W, B, max_ctx, no_fc=bool(flags & 8))   # 8 = PS_FLAG_NO_FC
         self.g = ps.drafter_from_shape(s, self.W, max_batch=B, max_ctx=max_ctx, flags=flags)
         self.to_device = ps.to_device
         hid, tok = [], []

@@ -186,3 +186,18 @@ def test_33b_batch16_k8_sampled_sequences():
     p = Pair(s, s.batch, context="import", oracle_seqs=[int(np.argmax(lens))])
     _compare_step(p, top_n=1)
     assert p.g.poll() == 0
+
+
+@pytest.mark.parametrize("name,B", [("mini", 3), ("mini", 1), ("tiny", 1)])
+def test_embedding_only_drafter(name, B):
+    """PS_FLAG_NO_FC: the drafter of the Medusa integration (Sec. 4.2), no fc and no target
+    feature; contexts built by ps_kv_append, the tensor-core path (mini) and the plain one."""
+    s = synth.CONFIGS[name]
+    p = Pair(s, B, flags=8)
+    _compare_step(p, top_n=2)
+    # the feature argument is not read: NULL is accepted
+    out = p.g.draft_step(list(range(B)), None, p.to_device(p.token_last), top_n=2)
+    torch.cuda.synchronize()
+    ref = p.gpu_step(top_n=2)
+    assert np.array_equal(out["logits"].cpu().numpy(), ref["logits"])
+    assert p.g.poll() == 0

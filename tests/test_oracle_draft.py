@@ -243,3 +243,25 @@ def test_row_stats():
     assert np.array_equal(ids, order)
     assert ids[1, 0] == 7 and ids[1, 1] == 9
     np.testing.assert_array_equal(vals, np.take_along_axis(x, order, 1))
+
+
+def test_embedding_only_input_is_the_identity_fc(oracle_mod):
+    """The embedding-only drafter of the Medusa integration (Sec. 4.2: shared embedding and LM
+    head, no target feature) is the pinned layer with fc = [I 0]: same logits, bit for bit."""
+    from oracle import Oracle, OracleConfig
+    s = synth.CONFIGS["mini32"].with_(k_masks=3)
+    W = synth.weights(s)
+    H = s.hidden
+    W_id = dict(W)
+    W_id["w_fc"] = np.concatenate([np.eye(H, dtype=np.float32), np.zeros((H, H), np.float32)], 1)
+    cfg = lambda no_fc: OracleConfig(s.dtype, s.hidden, s.n_heads, s.n_kv_heads, s.head_dim, s.ffn, s.vocab,
+                                     s.k_masks, 1, 64, s.rope_base, s.rms_eps, no_fc)
+    a, b = Oracle(cfg(True), W), Oracle(cfg(False), W_id)
+    h, t = synth.hidden_states(s, "c", 20), synth.token_ids(s, "c", 20)
+    assert a.kv_append(0, h, t) == 0 and b.kv_append(0, h, t) == 0
+    hl, tl = synth.hidden_states(s, "l", 1), synth.token_ids(s, "l", 1)
+    ra, rb = a.draft_step(0, hl, int(tl[0])), b.draft_step(0, hl, int(tl[0]))
+    assert np.array_equal(ra["logits"], rb["logits"]) and np.array_equal(ra["feat"], rb["feat"])
+    # and the target feature really is ignored
+    rc = a.draft_step(0, hl * 3 + 1, int(tl[0]))
+    assert np.array_equal(ra["logits"], rc["logits"])
