@@ -12,6 +12,8 @@
 //                   decoded in one pass), Sec. 4.3 / Sec. 5.1 "Models" (one
 //                   Transformer layer with the target layer's hyper-parameters,
 //                   shared LM head), Algorithm 1 (the k+1 draft distributions)
+//   pso_group_forward  Sec. 4.1 "Group-wise Parallel Training" (Fig. 3): the training layout of
+//                   parallel groups with its attention mask and position indices, forward only
 //   pso_verify      Eq. 1 and Algorithm 1 in its chain case (each node has one child)
 //   pso_verify_tree Algorithm 1 in full: a token tree, children tried in turn, the
 //                   target distribution replaced by its normalised residual after
@@ -416,6 +418,98 @@ int pso_draft_step(void* ctx, int slot, const void* hidden_last, int token_last,
     cp(taps->x_in, x_in); cp(taps->x0, x0); cp(taps->xn, xn); cp(taps->q, q);
     cp(taps->k_new, kn); cp(taps->v_new, vn); cp(taps->attn, attn); cp(taps->a, a);
     cp(taps->an, an); cp(taps->act, act); cp(taps->hdn, hdn); cp(taps->hn, hn);
+  }
+  return 0;
+}
+
+// Sec. 4.1 "Group-wise Parallel Training" (Fig. 3), forward only.  The source sequence is n
+// parallel groups; group t is the real pair (tokens[t], hidden[t]) followed by the k [MASK]
+// positions.  Row (t, j) has position index L + t + j (L = committed length of the slot: the
+// cached prefix) and attends to the cached positions, to the REAL rows of the groups 0..t and
+// to the [MASK] rows 1..j of its own group: never to a [MASK] row of another group.
+//   logits [n][k+1][V], feat [n][k+1][H].  Leaves the cache as it was.
+int pso_group_forward(void* ctx, int slot, int n, const void* hidden, const int* tokens, double* logits,
+                      double* feat) {
+  Ctx* C = (Ctx*)ctx;
+  const Config& c = C->c;
+  const int R = c.k_masks + 1, L = C->len[slot];
+  if (n < 1 || L + n + c.k_masks > c.max_ctx) return -3;
+  ensure_slab(C, slot);
+  const size_t H = c.hidden, d = c.head_dim, Hq = (size_t)c.n_heads * d, Hkv = (size_t)c.n_kv_heads * d;
+  const size_t F = c.ffn, V = c.vocab, M = (size_t)n * R;
+  const int group = c.n_heads / c.n_kv_heads;
+  std::vector<double> x_in(2 * H), x0(M * H), xn(H), q(M * Hq), kn(M * Hkv), vn(M * Hkv), attn(M * Hq);
+  for (int t = 0; t < n; ++t) {
+    for (int j = 0; j < R; ++j) {
+      const size_t r = (size_t)t * R + j;
+      if (j == 0) {
+        fill_real_input(*C, tokens[t], hidden, (size_t)t, x_in.data());
+      } else {
+        for (size_t i = 0; i < H; ++i) {
+          x_in[i] = widen(C->w.mask_embed, (size_t)(j - 1) * H + i, c.dtype);
+          x_in[H + i] = widen(C->w.mask_feat, (size_t)(j - 1) * H + i, c.dtype);
+        }
+      }
+      fuse_and_norm(*C, x_in.data(), &x0[r * H], xn.data());
+      matvec(C->w.w_q, nullptr, c.dtype, Hq, H, xn.data(), &q[r * Hq]);
+      for (int h = 0; h < c.n_heads; ++h) rope(&q[r * Hq + h * d], (int)d, L + t + j, c.rope_base);
+      project_kv(*C, xn.data(), L + t + j, &kn[r * Hkv], &vn[r * Hkv]);
+    }
+  }
+  const double scale = 1.0 / std::sqrt((double)d);
+  for (int t = 0; t < n; ++t) {
+    for (int j = 0; j < R; ++j) {
+      const size_t r = (size_t)t * R + j;
+      // the keys row (t, j) may see, as (source, index): cache rows, real rows, own [MASK] rows
+      std::vector<const double*> K, Vv;
+      for (int h = 0; h < c.n_heads; ++h) {
+        const int hk = h / group;
+        K.clear(); Vv.clear();
+        for (int p = 0; p < L; ++p) {
+          K.push_back(&C->K[slot][(size_t)p * Hkv + hk * d]);
+          Vv.push_back(&C->V[slot][(size_t)p * Hkv + hk * d]);
+        }
+        for (int g = 0; g <= t; ++g) {
+          K.push_back(&kn[((size_t)g * R) * Hkv + hk * d]);
+          Vv.push_back(&vn[((size_t)g * R) * Hkv + hk * d]);
+        }
+        for (int jj = 1; jj <= j; ++jj) {
+          K.push_back(&kn[((size_t)t * R + jj) * Hkv + hk * d]);
+          Vv.push_back(&vn[((size_t)t * R + jj) * Hkv + hk * d]);
+        }
+        const double* qv = &q[r * Hq + h * d];
+        std::vector<double> sc(K.size());
+        double smax = -std::numeric_limits<double>::infinity();
+        for (size_t u = 0; u < K.size(); ++u) {
+          double dot = 0.0;
+          for (size_t i = 0; i < d; ++i) dot += qv[i] * K[u][i];
+          sc[u] = dot * scale;
+          if (sc[u] > smax) smax = sc[u];
+        }
+        double denom = 0.0;
+        for (size_t u = 0; u < K.size(); ++u) { sc[u] = std::exp(sc[u] - smax); denom += sc[u]; }
+        double* o = &attn[r * Hq + h * d];
+        for (size_t i = 0; i < d; ++i) o[i] = 0.0;
+        for (size_t u = 0; u < K.size(); ++u) {
+          const double pw = sc[u] / denom;
+          for (size_t i = 0; i < d; ++i) o[i] += pw * Vv[u][i];
+        }
+      }
+    }
+  }
+  std::vector<double> a(H), an(H), gate(F), up(F), act(F), hdn(H), hn(H), tmp(H);
+  for (size_t r = 0; r < M; ++r) {
+    matvec(C->w.w_o, nullptr, c.dtype, H, Hq, &attn[r * Hq], tmp.data());
+    for (size_t i = 0; i < H; ++i) a[i] = x0[r * H + i] + tmp[i];
+    rmsnorm(a.data(), C->w.g_post, c.dtype, H, c.rms_eps, an.data());
+    matvec(C->w.w_gate, nullptr, c.dtype, F, H, an.data(), gate.data());
+    matvec(C->w.w_up, nullptr, c.dtype, F, H, an.data(), up.data());
+    for (size_t i = 0; i < F; ++i) act[i] = gate[i] / (1.0 + std::exp(-gate[i])) * up[i];
+    matvec(C->w.w_down, nullptr, c.dtype, H, F, act.data(), tmp.data());
+    for (size_t i = 0; i < H; ++i) hdn[i] = a[i] + tmp[i];
+    if (feat) std::memcpy(feat + r * H, hdn.data(), H * sizeof(double));
+    rmsnorm(hdn.data(), C->w.g_final, c.dtype, H, c.rms_eps, hn.data());
+    if (logits) matvec(C->w.w_lm, nullptr, c.dtype, V, H, hn.data(), &logits[r * V]);
   }
   return 0;
 }

@@ -189,6 +189,25 @@ class Oracle:
         out["feat"] = feat
         return out
 
+    def group_forward(self, slot: int, hidden: np.ndarray, tokens: np.ndarray):
+        """Group-wise parallel training layout, forward only (Sec. 4.1, Fig. 3): n groups of one
+        real pair + k [MASK] rows.  Returns dict(logits [n][k+1][V], feat [n][k+1][H])."""
+        cfg = self.cfg
+        hidden = np.ascontiguousarray(hidden)
+        tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+        assert hidden.dtype == self._np_dtype and hidden.shape == (len(tokens), cfg.hidden)
+        n, R = len(tokens), cfg.k_masks + 1
+        logits = np.empty((n, R, cfg.vocab), np.float64)
+        feat = np.empty((n, R, cfg.hidden), np.float64)
+        lib = _load()
+        lib.pso_group_forward.restype = C.c_int
+        lib.pso_group_forward.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p]
+        rc = lib.pso_group_forward(self._h, slot, n, _ptr(hidden), _ptr(tokens), _ptr(logits), _ptr(feat))
+        if rc != 0:
+            raise RuntimeError(f"oracle group_forward status {rc}")
+        return dict(logits=logits, feat=feat)
+
 
 def num_threads() -> int:
     """OpenMP threads the oracle's row loops run on."""

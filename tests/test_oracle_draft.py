@@ -265,3 +265,35 @@ def test_embedding_only_input_is_the_identity_fc(oracle_mod):
     # and the target feature really is ignored
     rc = a.draft_step(0, hl * 3 + 1, int(tl[0]))
     assert np.array_equal(ra["logits"], rc["logits"])
+
+
+def test_group_wise_training_forward_equals_inference_at_every_prefix(oracle_mod):
+    """Sec. 4.1 "Group-wise Parallel Training": the parallel-group layout with its mask and
+    position indices makes the drafter behave in training as in inference: group t of the one
+    batched forward equals the inference draft step taken after t real tokens."""
+    from oracle import Oracle, OracleConfig
+    s = synth.CONFIGS["mini32"].with_(k_masks=3)
+    W = synth.weights(s)
+    cfg = OracleConfig(s.dtype, s.hidden, s.n_heads, s.n_kv_heads, s.head_dim, s.ffn, s.vocab, s.k_masks,
+                       1, 64, s.rope_base, s.rms_eps)
+    n, L0 = 9, 6
+    hp, tp = synth.hidden_states(s, "pre", L0), synth.token_ids(s, "pre", L0)
+    h, t = synth.hidden_states(s, "grp", n), synth.token_ids(s, "grp", n)
+    a = Oracle(cfg, W)
+    assert a.kv_append(0, hp, tp) == 0
+    got = a.group_forward(0, h, t)
+    assert a.kv_len(0) == L0                      # forward only: the cache is as it was
+    b = Oracle(cfg, W)
+    assert b.kv_append(0, hp, tp) == 0
+    for g in range(n):
+        want = b.draft_step(0, h[g:g + 1], int(t[g]))
+        np.testing.assert_allclose(got["logits"][g], want["logits"], rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(got["feat"][g], want["feat"], rtol=1e-12, atol=1e-12)
+        assert b.kv_append(0, h[g:g + 1], t[g:g + 1]) == 0
+    # a [MASK] row of another group is never seen: changing group 2's learned rows' inputs
+    # (here: its real pair) leaves the [MASK] rows of group 1 untouched but moves group 3
+    h2 = h.copy()
+    h2[2] = synth.hidden_states(s, "other", 1)[0]
+    got2 = a.group_forward(0, h2, t)
+    assert np.array_equal(got2["logits"][:2], got["logits"][:2])
+    assert not np.allclose(got2["logits"][3], got["logits"][3])
