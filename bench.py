@@ -355,7 +355,8 @@ def main():
     # rotate over enough distinct KV sets that consecutive steps never find their KV in L2
     n_sets = 1 if kv_bytes_seq * B > 2 * L2_BYTES else max(2, min(16, -(-2 * L2_BYTES // max(1, kv_bytes_seq * B))))
     n_sets = min(n_sets, 128 // B)
-    g = ps.drafter_from_shape(s, W, max_batch=B * n_sets, max_ctx=int(lens.max()) + R)
+    max_ctx_bench = int(lens.max()) + R + 64        # + room for the groups of the training-layout leg
+    g = ps.drafter_from_shape(s, W, max_batch=B * n_sets, max_ctx=max_ctx_bench)
     del W
     for i in range(n_sets):
         for b in range(B):
@@ -445,6 +446,24 @@ def main():
         sampled = {"ms_per_step": f0.elapsed_time(f1) / n_s, "steps": n_s,
                    "note": "ps_draft_step_sampled (Gumbel-max in the LM-head epilogue) + ps_verify"}
 
+    # ---- group-wise training layout, forward only (Sec. 4.1): groups on the last KV set ---------
+    group = None
+    if int(lens.max()) + 64 + s.k_masks <= max_ctx_bench:
+        n_g = 64
+        gh = ps.to_device(synth.hidden_states(s, "grp", n_g))
+        gt = ps.to_device(synth.token_ids(s, "grp", n_g))
+        for i in range(2):
+            g.group_forward(int(slots[0][0]), gh, gt, top_n=1, want_logits=False)
+        torch.cuda.synchronize()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record()
+        for i in range(5):
+            g.group_forward(int(slots[0][0]), gh, gt, top_n=1, want_logits=False)
+        h1.record()
+        torch.cuda.synchronize()
+        group = {"ms_per_call": h0.elapsed_time(h1) / 5, "groups": n_g, "rows": n_g * R,
+                 "note": "ps_group_forward; more than 16 rows per launch run on the plain (untuned) kernels"}
+
     # ---- token-tree verification (Algorithm 1 in full), timed on its own ---------------------
     tree = None
     if V % 4 == 0 and V <= 131072 and s.dtype == 1:
@@ -494,7 +513,7 @@ def main():
             "hbm_frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
             "mean_tokens_per_round": n_accept,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "stages": stages, "sampled_drafts": sampled, "tree_verify": tree, "cpu_baseline": cpu,
+            "roofline": roofline, "stages": stages, "sampled_drafts": sampled, "group_forward": group, "tree_verify": tree, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
     if world > 1:

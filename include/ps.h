@@ -162,6 +162,20 @@ ps_status ps_draft_step_sampled(ps_ctx* ctx, int B, const int* seq_slot, const v
                                 float* top_logit, float* row_max, float* row_lse, float* logits_out,
                                 float* feat_out, void* stream);
 
+/* Group-wise parallel training layout, forward only (Sec. 4.1 "Group-wise Parallel Training",
+ * Fig. 3).  The n_groups real pairs (tokens[t], hidden[t]) that follow the slot's committed
+ * context each head a parallel group of k+1 rows: the pair and the k [MASK] positions.  Row j
+ * of group t has position index len + t + j and attends to the committed context, to the real
+ * rows of the groups 0..t and to the [MASK] rows 1..j of its own group, never to a [MASK] row
+ * of another group: every group sees what the inference draft step sees after t more real
+ * tokens.  Outputs as ps_draft_step with n_groups in the place of B ([n_groups][k+1]...).
+ * The slot's committed length is unchanged (cache rows beyond it are used as scratch).
+ * PS_ERR_CAPACITY if len + n_groups + k > max_ctx. */
+ps_status ps_group_forward(ps_ctx* ctx, int slot, int n_groups, const void* hidden,
+                           const int* tokens, int top_n, int* top_ids, float* top_logit,
+                           float* row_max, float* row_lse, float* logits_out, float* feat_out,
+                           void* stream);
+
 /* Lossless verification of a drafted chain (Eq. 1; Algorithm 1 with one child per node).
  * For position i = 0..n_draft-1 of sequence b, with p = softmax(target_logits[b][i]/T),
  * q = softmax(draft_logits[b][i]/T) and x = draft_tokens[b][i]: accept iff

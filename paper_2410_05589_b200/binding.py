@@ -29,7 +29,7 @@ EXPORTS = (
     "ps_workspace_bytes", "ps_init", "ps_kv_append", "ps_draft_step", "ps_verify", "ps_round_host",
     "ps_kv_len", "ps_kv_reset", "ps_kv_export", "ps_kv_import", "ps_poll", "ps_launch_count",
     "ps_last_error", "ps_destroy", "ps_philox_fill", "ps_profile", "ps_profile_read",
-    "ps_verify_static", "ps_debug_buffer", "ps_verify_tree", "ps_draft_step_sampled",
+    "ps_verify_static", "ps_debug_buffer", "ps_verify_tree", "ps_draft_step_sampled", "ps_group_forward",
 )
 
 
@@ -76,6 +76,7 @@ def load_library(path: str | None = None) -> C.CDLL:
                                   vp, vp, vp, vp]
     lib.ps_draft_step_sampled.argtypes = [vp, C.c_int, ip, vp, vp, C.c_float, C.c_uint64, C.c_uint64, vp,
                                           C.c_int, vp, vp, vp, vp, vp, vp, vp]
+    lib.ps_group_forward.argtypes = [vp, C.c_int, C.c_int, vp, vp, C.c_int, vp, vp, vp, vp, vp, vp, vp]
     lib.ps_verify_tree.argtypes = [vp, C.c_int, C.c_int, ip, vp, vp, vp, C.c_float, C.c_uint64, C.c_uint64,
                                    vp, vp, vp, vp, vp]
     lib.ps_kv_len.argtypes = [vp, C.c_int, ip]
@@ -250,6 +251,23 @@ class Drafter:
             self.h, B, _iarr(seq_slot), _dptr(hidden_last), _dptr(token_last), top_n,
             _dptr(o["top_ids"]), _dptr(o["top_logit"]), _dptr(o["row_max"]), _dptr(o["row_lse"]),
             _dptr(o.get("logits")), _dptr(o.get("feat")), _stream(stream)))
+        return o
+
+    def group_forward(self, slot: int, hidden: torch.Tensor, tokens: torch.Tensor, top_n: int = 1,
+                      want_logits: bool = True, want_feat: bool = False, stream=None) -> dict:
+        """ps_group_forward: the group-wise training layout, forward only.  hidden [n][H], tokens
+        [n] int32; outputs shaped [n][k+1]..."""
+        n, R, V, H = tokens.shape[0], self.rows, self.cfg.vocab, self.cfg.hidden
+        dev = "cuda"
+        o = {"top_ids": torch.empty((n, R, max(top_n, 1)), dtype=torch.int32, device=dev),
+             "top_logit": torch.empty((n, R, max(top_n, 1)), dtype=torch.float32, device=dev),
+             "row_max": torch.empty((n, R), dtype=torch.float32, device=dev),
+             "row_lse": torch.empty((n, R), dtype=torch.float32, device=dev),
+             "logits": torch.empty((n, R, V), dtype=torch.float32, device=dev) if want_logits else None,
+             "feat": torch.empty((n, R, H), dtype=torch.float32, device=dev) if want_feat else None}
+        self._check(self.lib.ps_group_forward(
+            self.h, slot, n, _dptr(hidden), _dptr(tokens), top_n, _dptr(o["top_ids"]), _dptr(o["top_logit"]),
+            _dptr(o["row_max"]), _dptr(o["row_lse"]), _dptr(o["logits"]), _dptr(o["feat"]), _stream(stream)))
         return o
 
     def draft_step_sampled(self, seq_slot, hidden_last: torch.Tensor, token_last: torch.Tensor,

@@ -130,8 +130,10 @@ __global__ void k_rmsnorm(const float* x, const WT* g, int H, float eps, float* 
 // RoPE on q (in place) and on k; k and v are written to the cache slab at the row's absolute
 // position.  One block per row.  kv_tmp row = [k (Hkv) ; v (Hkv)] fp32.  The pair
 // (i, i + d/2) of a head is rotated by pos * base^(-2i/d); angles are formed in double.
+// With `side` != nullptr the new k / v rows go to side[m][2 * Hkv] (k then v) instead of the
+// cache: a draft step leaves the cache untouched, and several groups may share one slot.
 template <typename WT>
-__global__ void k_rope_store(SeqMap sm, float* q, const float* kv_tmp, WT* kcache, WT* vcache,
+__global__ void k_rope_store(SeqMap sm, float* q, const float* kv_tmp, WT* kcache, WT* vcache, WT* side,
                              int n_heads, int n_kv_heads, int d, int max_ctx, float rope_base) {
   extern __shared__ float cs[];  // cos[d/2], sin[d/2]
   int m = blockIdx.x;
@@ -163,21 +165,29 @@ __global__ void k_rope_store(SeqMap sm, float* q, const float* kv_tmp, WT* kcach
   for (int t = threadIdx.x; t < n_kv_heads * half; t += blockDim.x) {
     int h = t / half, i = t - h * half;
     float x = kr[h * d + i], y = kr[h * d + i + half];
-    size_t base = ((slab + h) * max_ctx + pos) * d;
-    store_as(kcache + base + i, x * cs[i] - y * cs[half + i]);
-    store_as(kcache + base + i + half, y * cs[i] + x * cs[half + i]);
-    store_as(vcache + base + i, vr[h * d + i]);
-    store_as(vcache + base + i + half, vr[h * d + i + half]);
+    WT *kd, *vd;
+    if (side) {
+      kd = side + (size_t)m * 2 * Hkv + h * d;
+      vd = kd + Hkv;
+    } else {
+      const size_t base = ((slab + h) * max_ctx + pos) * d;
+      kd = kcache + base;
+      vd = vcache + base;
+    }
+    store_as(kd + i, x * cs[i] - y * cs[half + i]);
+    store_as(kd + i + half, y * cs[i] + x * cs[half + i]);
+    store_as(vd + i, vr[h * d + i]);
+    store_as(vd + i + half, vr[h * d + i + half]);
   }
 }
 
 // Attention under the parallel-draft mask: row j of a sequence sees cache rows [0, len) and
-// the new rows 0..j, which sit at slab rows len..len+j.  One block (4 warps) per (head, b);
+// the new rows 0..j, which sit in side[m][2 * Hkv] (k then v).  One block (4 warps) per (head, b);
 // warps take keys round-robin, each lane owns D/32 channels; online softmax per (warp, row).
 template <typename WT, int D>
 __global__ void __launch_bounds__(128) k_attention(SeqMap sm, const float* q, const WT* kcache,
-                                                   const WT* vcache, int n_heads, int n_kv_heads,
-                                                   int max_ctx, float* attn) {
+                                                   const WT* vcache, const WT* side, int n_heads,
+                                                   int n_kv_heads, int max_ctx, float* attn) {
   constexpr int C = D / 32;
   constexpr int RMAX = kMaxRowsPerSeq;
   __shared__ float s_m[4][RMAX], s_l[4][RMAX];
@@ -208,9 +218,12 @@ __global__ void __launch_bounds__(128) k_attention(SeqMap sm, const float* q, co
   for (int t = warp; t < L + R; t += 4) {
     float kx[C], vx[C];
 #pragma unroll
+    const WT* kr = t < L ? kb + (size_t)t * D : side + (size_t)(m0 + t - L) * 2 * n_kv_heads * D + hk * D;
+    const WT* vr = t < L ? vb + (size_t)t * D : kr + n_kv_heads * D;
+#pragma unroll
     for (int c = 0; c < C; ++c) {
-      kx[c] = to_f32(kb[(size_t)t * D + lane + 32 * c]);
-      vx[c] = to_f32(vb[(size_t)t * D + lane + 32 * c]);
+      kx[c] = to_f32(kr[lane + 32 * c]);
+      vx[c] = to_f32(vr[lane + 32 * c]);
     }
     int jmin = t < L ? 0 : t - L;  // rows that may see key t
 #pragma unroll
@@ -398,8 +411,9 @@ ps_status fc_norm_kv(ps_ctx* c, const SeqMap& sm, int rows, int all_real, const 
   if ((s = linear<WT>(c, c->xn, H, w.w_k, nullptr, nullptr, 0, c->kv_tmp, 2 * Hkv, rows, Hkv, H, st))) return s;
   if ((s = linear<WT>(c, c->xn, H, w.w_v, nullptr, nullptr, 0, c->kv_tmp + Hkv, 2 * Hkv, rows, Hkv, H, st))) return s;
   k_rope_store<WT><<<rows, 128, g.head_dim * sizeof(float), st>>>(
-      sm, with_q ? c->q : nullptr, c->kv_tmp, (WT*)c->kcache, (WT*)c->vcache, g.n_heads,
-      g.n_kv_heads, g.head_dim, g.max_ctx, g.rope_base);
+      sm, with_q ? c->q : nullptr, c->kv_tmp, (WT*)c->kcache, (WT*)c->vcache,
+      with_q ? (WT*)c->kv_side : nullptr,   // a draft step keeps its new rows out of the cache
+      g.n_heads, g.n_kv_heads, g.head_dim, g.max_ctx, g.rope_base);
   c->launches++;
   prof_mark(c, st, "qkv_rope");
   return cuda_check(c, cudaGetLastError(), "fc_norm_kv");
@@ -419,10 +433,10 @@ ps_status draft_impl(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last
   dim3 ag(g.n_heads, B);
   if (g.head_dim == 64)
     k_attention<WT, 64><<<ag, 128, 0, st>>>(sm, c->q, (const WT*)c->kcache, (const WT*)c->vcache,
-                                            g.n_heads, g.n_kv_heads, g.max_ctx, c->attn);
+                                            (const WT*)c->kv_side, g.n_heads, g.n_kv_heads, g.max_ctx, c->attn);
   else
     k_attention<WT, 128><<<ag, 128, 0, st>>>(sm, c->q, (const WT*)c->kcache, (const WT*)c->vcache,
-                                             g.n_heads, g.n_kv_heads, g.max_ctx, c->attn);
+                                             (const WT*)c->kv_side, g.n_heads, g.n_kv_heads, g.max_ctx, c->attn);
   c->launches++;
   prof_mark(c, st, "attention");
   if ((s = linear<WT>(c, c->attn, Hq, w.w_o, nullptr, c->x0, H, c->a, H, M, H, Hq, st))) return s;

@@ -77,6 +77,7 @@ size_t carve(const ps_config& g, ps_ctx* c, char* base) {
   void* xn = take(Mx * H * 4);
   void* q = take(Md * Hq * 4);
   void* kv_tmp = take(Mx * 2 * Hkv * 4);
+  void* kv_side = take(Md * 2 * Hkv * elem_bytes(g));
   void* attn = take(Md * Hq * 4);
   void* a = take(Md * H * 4);
   void* an = take(Md * H * 4);
@@ -98,7 +99,7 @@ size_t carve(const ps_config& g, ps_ctx* c, char* base) {
     c->vrec = (VerifyRec*)vrec;
     c->trec = (TreeRec*)trec; c->tree_tickets = (unsigned*)ttick;
     c->x_in = (float*)x_in; c->x0 = (float*)x0; c->xn = (float*)xn; c->q = (float*)q;
-    c->kv_tmp = (float*)kv_tmp; c->attn = (float*)attn; c->a = (float*)a; c->an = (float*)an;
+    c->kv_tmp = (float*)kv_tmp; c->kv_side = kv_side; c->attn = (float*)attn; c->a = (float*)a; c->an = (float*)an;
     c->gate = (float*)gate; c->up = (float*)up; c->hdn = (float*)hdn; c->hn = (float*)hn;
     c->logits = (float*)logits;
     c->fused_scratch = fused;
@@ -369,6 +370,55 @@ ps_status ps_draft_step_sampled(ps_ctx* c, int B, const int* seq_slot, const voi
   sa.sampled = sampled_ids;
   return draft_common(c, B, seq_slot, hidden_last, token_last, top_n, top_ids, top_logit, row_max, row_lse,
                       logits_out, feat_out, &sa, stream);
+}
+
+ps_status ps_group_forward(ps_ctx* c, int slot, int n_groups, const void* hidden, const int* tokens,
+                           int top_n, int* top_ids, float* top_logit, float* row_max, float* row_lse,
+                           float* logits_out, float* feat_out, void* stream) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  const ps_config& g = c->cfg;
+  if (slot < 0 || slot >= g.max_batch) return fail(c, PS_ERR_INVALID_ARG, "slot out of range");
+  if (n_groups < 1) return fail(c, PS_ERR_INVALID_ARG, "n_groups must be positive");
+  if ((!hidden && !(g.flags & PS_FLAG_NO_FC)) || !tokens) return fail(c, PS_ERR_INVALID_ARG, "null hidden / tokens");
+  if (top_n < 0 || top_n > PS_MAX_TOP_N || top_n > g.vocab) return fail(c, PS_ERR_INVALID_ARG, "top_n out of range");
+  if (top_n > 0 && (!top_ids || !top_logit)) return fail(c, PS_ERR_INVALID_ARG, "null top-n output");
+  const int R = g.k_masks + 1, L0 = c->len[slot];
+  if (L0 + n_groups + g.k_masks > g.max_ctx) return fail(c, PS_ERR_CAPACITY, "no room for the groups");
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t eb = g.dtype == PS_DTYPE_F32 ? 4 : 2;
+  ps_status s;
+  // 1. the real rows' k / v at cache rows [L0, L0 + n): beyond the committed length, so the
+  //    context stays as it was
+  SeqMap sm;
+  std::memset(&sm, 0, sizeof(sm));
+  sm.B = 1; sm.slot[0] = slot; sm.len[0] = L0; sm.row_off[0] = 0; sm.row_off[1] = n_groups;
+  for (int r0 = 0; r0 < n_groups; r0 += kAppendChunk) {
+    sm.row_base = r0;
+    if ((s = plain_kv_append(c, sm, std::min(kAppendChunk, n_groups - r0), hidden, tokens, st)) != PS_OK) return s;
+  }
+  // 2. the groups as a batch of draft steps on the same slot: group t sees cache rows
+  //    [0, L0 + t), i.e. the prefix and the real rows before it, and its own k + 1 new rows
+  const int chunk = std::min(g.max_batch, (int)PS_MAX_BATCH);
+  for (int g0 = 0; g0 < n_groups; g0 += chunk) {
+    const int B = std::min(chunk, n_groups - g0);
+    std::memset(&sm, 0, sizeof(sm));
+    sm.B = B;
+    for (int b = 0; b < B; ++b) { sm.slot[b] = slot; sm.len[b] = L0 + g0 + b; sm.row_off[b] = b * R; }
+    sm.row_off[B] = B * R;
+    const size_t r0 = (size_t)g0 * R;
+    const void* h = hidden ? (const char*)hidden + (size_t)g0 * g.hidden * eb : nullptr;
+    int* ti = top_ids ? top_ids + r0 * top_n : nullptr;
+    float* tl = top_logit ? top_logit + r0 * top_n : nullptr;
+    float* rm = row_max ? row_max + r0 : nullptr;
+    float* rl = row_lse ? row_lse + r0 : nullptr;
+    float* lo = logits_out ? logits_out + r0 * g.vocab : nullptr;
+    float* fo = feat_out ? feat_out + r0 * g.hidden : nullptr;
+    s = fused_supported(c, B * R)
+            ? fused_draft_step(c, sm, B, h, tokens + g0, top_n, ti, tl, rm, rl, lo, fo, nullptr, st)
+            : plain_draft_step(c, sm, B, h, tokens + g0, top_n, ti, tl, rm, rl, lo, fo, nullptr, st);
+    if (s != PS_OK) return s;
+  }
+  return PS_OK;
 }
 
 ps_status ps_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draft_tokens,

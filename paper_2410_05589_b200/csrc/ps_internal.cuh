@@ -125,6 +125,7 @@ struct ps_ctx {
   ps::TreeRec* trec;        // [max_batch][PS_MAX_TREE_NODES+1]
   unsigned* tree_tickets;   // [max_batch], zero between calls
   float *x_in, *x0, *xn, *q, *kv_tmp, *attn, *a, *an, *gate, *up, *hdn, *hn, *logits;
+  void* kv_side;            // [max_rows][2 * Hkv] storage dtype: k / v of a draft step's new rows (plain kernels)
   // staging for ps_round_host
   void* fused_scratch;      // buffers of the fused bf16 path (see fused_kernels.cu)
   void* umma_maps = nullptr;   // tensor maps of the tensor-core GEMMs, built on first use

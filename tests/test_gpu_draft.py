@@ -201,3 +201,30 @@ def test_embedding_only_drafter(name, B):
     ref = p.gpu_step(top_n=2)
     assert np.array_equal(out["logits"].cpu().numpy(), ref["logits"])
     assert p.g.poll() == 0
+
+
+@pytest.mark.parametrize("name,n,max_batch", [("mini", 11, 3), ("mini", 7, 16), ("tiny", 9, 4), ("mini32", 5, 1)])
+def test_group_wise_training_forward(name, n, max_batch):
+    """ps_group_forward (Sec. 4.1 "Group-wise Parallel Training", Fig. 3) against the oracle's
+    forward over the whole group layout; groups run in chunks of max_batch on the tensor-core
+    path (a few groups) or the plain kernels, after a committed prefix."""
+    import paper_2410_05589_b200 as ps
+    s = synth.CONFIGS[name]
+    p = Pair(s, max_batch, lens=[13] + [0] * (max_batch - 1), oracle_seqs=[0], extra_ctx=n + 4)
+    h, t = synth.hidden_states(s, "grp", n), synth.token_ids(s, "grp", n)
+    want = p.o.group_forward(0, h, t)
+    out = p.g.group_forward(0, p.to_device(h), p.to_device(t), top_n=1, want_feat=True)
+    torch.cuda.synchronize()
+    got = {k: v.cpu().numpy() for k, v in out.items()}
+    for g in range(n):
+        assert logits_close(got["logits"][g], want["logits"][g], s.dtype) <= 1.0, g
+        assert logits_close(got["feat"][g], want["feat"][g], s.dtype) <= 1.0, g
+        for j in range(s.rows):
+            check_top(got["top_ids"][g, j], got["top_logit"][g, j], want["logits"][g, j], s.dtype)
+    # forward only: the context is as it was, and an ordinary draft step still agrees
+    assert p.g.kv_len(0) == 13
+    step = p.g.draft_step([0], p.to_device(p.hidden_last[:1]), p.to_device(p.token_last[:1]), top_n=1)
+    torch.cuda.synchronize()
+    ref = p.oracle_step(0)
+    assert logits_close(step["logits"][0].cpu().numpy(), ref["logits"], s.dtype) <= 1.0
+    assert p.g.poll() == 0
