@@ -374,10 +374,13 @@ static ps_status launch_attn_t(ps_ctx* c, const SeqMap& sm, int B, int max_len, 
   // several of them per block
   auto kern = k_attn_mma<D, NB>;
   static int blocks_per_sm[kTileMax / 16 + 1];   // per tile size, asked once (0 = not yet)
+  // the partial buffers hold 16 rows x kAttnMaxSplit splits: more rows, fewer splits
+  const int M_rows = B * (g.k_masks + 1);
+  const int max_split = std::max(1, std::min(kAttnMaxSplit, 16 * kAttnMaxSplit / std::max(M_rows, 1)));
   int tile = kTileMax, n_split = 0;
   for (int cand = kTileMax; cand >= 32; cand -= 16) {
     const int tiles = (max_len + cand - 1) / cand;
-    if (tiles > kAttnMaxSplit) break;
+    if (tiles > max_split) break;
     int& bps = blocks_per_sm[cand / 16];
     if (bps == 0) {
       const size_t bytes = attn_smem_bytes(D, NB, cand);
@@ -390,7 +393,7 @@ static ps_status launch_attn_t(ps_ctx* c, const SeqMap& sm, int B, int max_len, 
   }
   if (n_split == 0) {
     const int want = (3 * c->n_sm + B * g.n_heads - 1) / (B * g.n_heads);
-    n_split = std::max(1, std::min(std::min(want, kAttnMaxSplit), (max_len + tile - 1) / tile));
+    n_split = std::max(1, std::min(std::min(want, max_split), (max_len + tile - 1) / tile));
   }
   const size_t bytes = attn_smem_bytes(D, NB, tile);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);

@@ -419,8 +419,9 @@ struct FusedScratch {
   size_t bytes;
 };
 
-// One carve-up for sizing (base == nullptr) and for use; always kMaxM rows and kMaxSm CTAs.
+// One carve-up for sizing (base == nullptr) and for use; always the largest row and CTA counts.
 FusedScratch carve_fused(const ps_config& g, char* base) {
+  constexpr int kRows = umma::kMaxRows;   // rows the tensor-core path can take (the mma.sync kernels: kMaxM)
   const size_t Hq = (size_t)g.n_heads * g.head_dim, Hkv = (size_t)g.n_kv_heads * g.head_dim;
   size_t off = 0;
   auto take = [&](size_t bytes) {
@@ -430,24 +431,25 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
   };
   auto planes = [&](size_t width) {
     Planes p;
-    p.hi = (__nv_bfloat16*)take((size_t)kMaxM * width * 2);
-    p.lo = (__nv_bfloat16*)take((size_t)kMaxM * width * 2);
+    p.hi = (__nv_bfloat16*)take((size_t)kRows * width * 2);
+    p.lo = (__nv_bfloat16*)take((size_t)kRows * width * 2);
     return p;
   };
   FusedScratch s;
-  s.qkv = (float*)take((size_t)kMaxM * (Hq + 2 * Hkv) * 4);
+  s.qkv = (float*)take((size_t)kRows * (Hq + 2 * Hkv) * 4);
+  // (rows x splits is bounded: the attention launcher takes fewer splits when there are more rows)
   s.att_ml = (float*)take((size_t)kMaxM * g.n_heads * kAttnMaxSplit * 2 * 4);
   s.att_o = (float*)take((size_t)kMaxM * g.n_heads * kAttnMaxSplit * g.head_dim * 4);
-  s.act = (float*)take((size_t)kMaxM * g.ffn * 4);
+  s.act = (float*)take((size_t)kRows * g.ffn * 4);
   // per-CTA (mma.sync path) or per-tile (tensor-core path) summaries
   const int tiles_v = (g.vocab + 127) / 128, tiles_h = (g.hidden + 127) / 128;
   s.n_part_rows = std::max(kMaxSm, std::max(tiles_v, tiles_h));
-  s.parts = (LmPart*)take((size_t)s.n_part_rows * kMaxM * sizeof(LmPart));
+  s.parts = (LmPart*)take((size_t)s.n_part_rows * kRows * sizeof(LmPart));
   s.ticket = (unsigned*)take(256);
   s.attn_tickets = (unsigned*)take((size_t)PS_MAX_BATCH * g.n_heads * 4);
-  for (int i = 0; i < 3; ++i) s.ssq[i] = (float*)take((size_t)s.n_part_rows * kMaxM * 4);
-  s.xin = (__nv_bfloat16*)take((size_t)kMaxM * 2 * g.hidden * 2);
-  s.partials = (float*)take((size_t)kMaxSm * 2 * 16 * 128 * 4);
+  for (int i = 0; i < 3; ++i) s.ssq[i] = (float*)take((size_t)s.n_part_rows * kRows * 4);
+  s.xin = (__nv_bfloat16*)take((size_t)kRows * 2 * g.hidden * 2);
+  s.partials = (float*)take((size_t)kMaxSm * 2 * kRows * 128 * 4);
   const size_t max_tiles = std::max<size_t>({(size_t)tiles_v, (size_t)(g.ffn + 63) / 64,
                                              (Hq + 127) / 128 + 2 * ((Hkv + 127) / 128), (size_t)tiles_h});
   s.tile_tickets = (unsigned*)take(max_tiles * 4);
@@ -463,6 +465,7 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
 // =============================================================================================
 struct UArgs {
   int N, K, M;
+  int Mp;                  // M padded to 16, 32, 64 or 128: rows of a plane box, half the MMA's N
   int n_tiles, KB;         // tiles of 128 weight rows (64 features when zipped), k-blocks of 64
   int zip;                 // 1: a tile is 64 rows of matrix 0 (gate) over 64 rows of matrix 1 (up)
   int lo;                  // 0: the activation operand is exact bf16 (no lo plane)
@@ -554,12 +557,14 @@ __device__ __forceinline__ int tile_feature(const UArgs& a, int t, int r, bool& 
   return a.mat_off[m] + local;
 }
 
-// Epilogue of one finished tile; called by the 128 epilogue threads after each has put its
-// accumulator row r (= 32 * q + lane) into ctl.acc[m * 128 + r], m = activation row.  The loops
+// Epilogue of one finished tile for the activation rows [m0, m0 + mc), mc <= 16; called by the
+// 128 epilogue threads after each has put its accumulator row r (= 32 * q + lane) of those
+// rows into ctl.acc[(m - m0) * 128 + r].  The loops
 // over m are rolled on purpose: this code runs once or twice per CTA, so what it costs is the
 // fetch of its instructions, not their execution.
 template <int EPI>
-__device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane) {
+__device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane,
+                                              int m0, int mc) {
   using namespace umma;
   const int et = r;
   bool valid;
@@ -569,15 +574,15 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
     const float bias = (a.bias && valid) ? __bfloat162float(a.bias[n]) : 0.f;
     const float gain = (a.gain_next && valid) ? __bfloat162float(a.gain_next[n]) : 1.f;
 #pragma unroll 1
-    for (int m = 0; m < a.M; ++m) {
+    for (int m = 0; m < mc; ++m) {
       float sq = 0.f;
       if (valid) {
-        float x = acc[m * 128] * ctl.scale[m] + bias;
-        if (a.res) x += a.res[(size_t)m * a.ldr + n];
-        a.out[(size_t)m * a.ldo + n] = x;
+        float x = acc[m * 128] * ctl.scale[m0 + m] + bias;
+        if (a.res) x += a.res[(size_t)(m0 + m) * a.ldr + n];
+        a.out[(size_t)(m0 + m) * a.ldo + n] = x;
         sq = x * x;
         if (a.out_hi)
-          split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, x * gain);
+          split_store(a.out_hi + (size_t)(m0 + m) * a.ld_plane + n, a.out_lo + (size_t)(m0 + m) * a.ld_plane + n, x * gain);
       }
       if (a.ssq_out) {
         sq = warp_sum(sq);
@@ -586,30 +591,30 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
     }
     if (a.ssq_out) {
       epi_sync();
-      if (et < a.M) a.ssq_out[(size_t)t * a.M + et] = (ctl.red[0][et] + ctl.red[1][et]) + (ctl.red[2][et] + ctl.red[3][et]);
+      if (et < mc) a.ssq_out[(size_t)t * a.M + m0 + et] = (ctl.red[0][et] + ctl.red[1][et]) + (ctl.red[2][et] + ctl.red[3][et]);
       epi_sync();
     }
   } else if (EPI == EPI_SWIGLU) {
     if (r >= 64) {
 #pragma unroll 1
-      for (int m = 0; m < a.M; ++m) ctl.xch[m * 64 + (r - 64)] = acc[m * 128] * ctl.scale[m];
+      for (int m = 0; m < mc; ++m) ctl.xch[m * 64 + (r - 64)] = acc[m * 128] * ctl.scale[m0 + m];
     }
     epi_sync();
     if (r < 64 && valid) {
 #pragma unroll 1
-      for (int m = 0; m < a.M; ++m) {
-        const float gv = acc[m * 128] * ctl.scale[m], uv = ctl.xch[m * 64 + r];
+      for (int m = 0; m < mc; ++m) {
+        const float gv = acc[m * 128] * ctl.scale[m0 + m], uv = ctl.xch[m * 64 + r];
         const float act = gv / (1.f + __expf(-gv)) * uv;
-        if (a.out) a.out[(size_t)m * a.ldo + n] = act;
-        split_store(a.out_hi + (size_t)m * a.ld_plane + n, a.out_lo + (size_t)m * a.ld_plane + n, act);
+        if (a.out) a.out[(size_t)(m0 + m) * a.ldo + n] = act;
+        split_store(a.out_hi + (size_t)(m0 + m) * a.ld_plane + n, a.out_lo + (size_t)(m0 + m) * a.ld_plane + n, act);
       }
     }
     epi_sync();
   } else {  // EPI_LMHEAD: logits, and the tile's softmax / top-n summary per row
 #pragma unroll 1
-    for (int m = 0; m < a.M; ++m) {
-      const float x = acc[m * 128] * ctl.scale[m];
-      if (valid && a.logits_out) a.logits_out[(size_t)m * a.N + n] = x;
+    for (int m = 0; m < mc; ++m) {
+      const float x = acc[m * 128] * ctl.scale[m0 + m];
+      if (valid && a.logits_out) a.logits_out[(size_t)(m0 + m) * a.N + n] = x;
       float mx = valid ? x : -FLT_MAX;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -617,14 +622,14 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
     }
     epi_sync();
 #pragma unroll 1
-    for (int m = 0; m < a.M; ++m) {
+    for (int m = 0; m < mc; ++m) {
       const float bmax = fmaxf(fmaxf(ctl.red[0][m], ctl.red[1][m]), fmaxf(ctl.red[2][m], ctl.red[3][m]));
-      const float s = warp_sum(valid ? __expf(acc[m * 128] * ctl.scale[m] - bmax) : 0.f);
+      const float s = warp_sum(valid ? __expf(acc[m * 128] * ctl.scale[m0 + m] - bmax) : 0.f);
       if (lane == 0) ctl.red2[q][m] = s;
     }
     epi_sync();
-    if (et < a.M) {
-      LmPart* p = a.parts + (size_t)t * a.M + et;
+    if (et < mc) {
+      LmPart* p = a.parts + (size_t)t * a.M + m0 + et;
       p->vmax = fmaxf(fmaxf(ctl.red[0][et], ctl.red[1][et]), fmaxf(ctl.red[2][et], ctl.red[3][et]));
       p->sumexp = (ctl.red2[0][et] + ctl.red2[1][et]) + (ctl.red2[2][et] + ctl.red2[3][et]);
     }
@@ -632,8 +637,8 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
 #pragma unroll 1
     for (int tn = 0; tn < a.top_n; ++tn) {
 #pragma unroll 1
-      for (int m = 0; m < a.M; ++m) {
-        const float x = acc[m * 128] * ctl.scale[m];
+      for (int m = 0; m < mc; ++m) {
+        const float x = acc[m * 128] * ctl.scale[m0 + m];
         const float pv = tn ? ctl.prev_v[m] : FLT_MAX;
         const int pi = tn ? ctl.prev_i[m] : -1;
         const bool after = valid && ((x < pv) || (x == pv && n > pi));
@@ -648,7 +653,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
         if (lane == 0) { ctl.cand_v[q][m] = bv; ctl.cand_i[q][m] = bi; }
       }
       epi_sync();
-      if (et < a.M) {
+      if (et < mc) {
         float bv = ctl.cand_v[0][et]; int bi = ctl.cand_i[0][et];
 #pragma unroll
         for (int w = 1; w < 4; ++w) {
@@ -656,7 +661,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
           if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
         ctl.prev_v[et] = bv; ctl.prev_i[et] = bi;
-        LmPart* p = a.parts + (size_t)t * a.M + et;
+        LmPart* p = a.parts + (size_t)t * a.M + m0 + et;
         p->top_v[tn] = bv; p->top_i[tn] = bi;
         if (tn == 0) { p->v0 = bv; p->i0 = bi; }
       }
@@ -664,13 +669,13 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
     }
     if (a.sample) {   // Gumbel-max candidate of this vocabulary range per row
 #pragma unroll 1
-      for (int m = 0; m < a.M; ++m) {
-        const int sb = m / a.R;
-        const uint32_t row_id = (uint32_t)sb | ((uint32_t)(m - sb * a.R) << 8);
+      for (int m = 0; m < mc; ++m) {
+        const int sb = (m0 + m) / a.R;
+        const uint32_t row_id = (uint32_t)sb | ((uint32_t)(m0 + m - sb * a.R) << 8);
         float bv = -FLT_MAX;
         int bi = 0x7fffffff;
         if (valid) {
-          bv = acc[m * 128] * ctl.scale[m] * a.sa.inv_temp + gumbel_noise(a.sa, (uint32_t)n, row_id);
+          bv = acc[m * 128] * ctl.scale[m0 + m] * a.sa.inv_temp + gumbel_noise(a.sa, (uint32_t)n, row_id);
           bi = n;
         }
 #pragma unroll
@@ -682,14 +687,14 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
         if (lane == 0) { ctl.cand_v[q][m] = bv; ctl.cand_i[q][m] = bi; }
       }
       epi_sync();
-      if (et < a.M) {
+      if (et < mc) {
         float bv = ctl.cand_v[0][et]; int bi = ctl.cand_i[0][et];
 #pragma unroll
         for (int w = 1; w < 4; ++w) {
           const float ov = ctl.cand_v[w][et]; const int oi = ctl.cand_i[w][et];
           if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
-        LmPart* p = a.parts + (size_t)t * a.M + et;
+        LmPart* p = a.parts + (size_t)t * a.M + m0 + et;
         p->sv = bv; p->si = bi;
       }
     }
@@ -719,7 +724,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   }
   if (warp == 1) {   // tensor memory for two accumulators
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
-                 "r"(kTmemCols)
+                 "r"(tmem_cols(a.Mp))
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -732,17 +737,19 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   const int u0 = unit_begin(blockIdx.x, U, G), u1 = unit_begin(blockIdx.x + 1, U, G);
   const Segs segs(u0, u1, a.KB);
   volatile int* abort_flag = &ctl.abort_flag;
+  const int Mp = a.Mp, sbytes = stage_bytes(Mp), nst = n_stages(Mp), ksplit = k_split(Mp), acols = acc_cols(Mp);
+  const int plane_bytes = Mp * kBK * 2;
 
   if (warp == 0) {
     if (lane == 0) {   // ---- TMA producer
-      const uint32_t bytes = kABytes + kBBytes * (a.lo ? 2 : 1);
+      const uint32_t bytes = kABytes + plane_bytes * (a.lo ? 2 : 1);
       // The weights do not depend on the kernel before this one, its activations do: the
       // weight boxes of the first kStages units are requested first, then the thread waits for
       // that kernel and adds their activation boxes.
-      const int n_units = u1 - u0, n_early = min(kStages, n_units);
+      const int n_units = u1 - u0, n_early = min(nst, n_units);
       UnitWalk w;
       auto load_a = [&](const UnitWalk& uw, int st_i) {
-        const uint32_t dst = base + st_i * kStageBytes;
+        const uint32_t dst = base + st_i * sbytes;
         const int x = uw.kb * kBK;
         mbar_arrive_expect_tx(&ctl.full[st_i], bytes);
         if (a.zip) {
@@ -753,10 +760,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         }
       };
       auto load_b = [&](const UnitWalk& uw, int st_i) {
-        const uint32_t dst = base + st_i * kStageBytes + kABytes;
+        const uint32_t dst = base + st_i * sbytes + kABytes;
         const int x = uw.kb * kBK;
         tma_load_2d(dst, &tBh, x, 0, &ctl.full[st_i]);
-        if (a.lo) tma_load_2d(dst + kBBytes, &tBl, x, 0, &ctl.full[st_i]);
+        if (a.lo) tma_load_2d(dst + plane_bytes, &tBl, x, 0, &ctl.full[st_i]);
       };
       w.start(segs, a);
       for (int i = 0; i < n_early; ++i) { load_a(w, i); w.next(segs, a); }
@@ -770,7 +777,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         load_a(w, stage);
         load_b(w, stage);
         w.next(segs, a);
-        if (++stage == kStages) { stage = 0; parity ^= 1; }
+        if (++stage == nst) { stage = 0; parity ^= 1; }
       }
     }
   } else if (warp == 1) {
@@ -778,25 +785,28 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       int stage = 0;
       uint32_t parity = 0;
       bool alive = true;
-      const uint32_t id = a.lo ? idesc(2 * kN) : idesc(kN);   // hi and lo planes as one N = 32 operand
+      const uint32_t id = a.lo ? idesc(2 * Mp) : idesc(Mp);   // hi and lo planes as one operand of N = 2 Mp
       for (int si = 0; si < segs.n && alive; ++si) {
         int t, b, e;
         segs.get(si, t, b, e);
         const int buf = si & 1;
         if (!mbar_wait(&ctl.acc_empty[buf], ((si >> 1) & 1) ^ 1, abort_flag)) break;
         fence_after_sync();
-        const uint32_t d = tmem + buf * kAccCols;
+        const uint32_t d = tmem + buf * acols;
         uint32_t acc = 0;
         for (int j = b; j < e; ++j) {
           if (!mbar_wait(&ctl.full[stage], parity, abort_flag)) { alive = false; break; }
           fence_after_sync();
-          const uint32_t sa = base + stage * kStageBytes;
+          const uint32_t sa = base + stage * sbytes;
 #pragma unroll
-          for (int k = 0; k < kAccSplit; ++k)   // four accumulators: no MMA waits for the one before
-            mma_f16(d + k * 2 * kN, smem_desc(sa + k * 32), smem_desc(sa + kABytes + k * 32), id, acc);
+          for (int k = 0; k < kBK / 16; ++k) {   // k step k goes to accumulator k % ksplit
+            const int ai = k % ksplit;
+            mma_f16(d + ai * 2 * Mp, smem_desc(sa + k * 32), smem_desc(sa + kABytes + k * 32), id,
+                    (acc || k >= ksplit) ? 1u : 0u);
+          }
           acc = 1;
           mma_commit(&ctl.empty[stage]);
-          if (++stage == kStages) { stage = 0; parity ^= 1; }
+          if (++stage == nst) { stage = 0; parity ^= 1; }
         }
         if (alive) mma_commit(&ctl.acc_full[buf]);
       }
@@ -825,33 +835,43 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       // all four warps take the same decision although each thread waits for itself
       if (epi_any(!mbar_wait(&ctl.acc_full[buf], (seg >> 1) & 1, abort_flag))) break;
       fence_after_sync();
-      float v[16];
-      {
-        const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + buf * kAccCols;
-        tmem_ld16(ta, v);
-#pragma unroll
-        for (int c = 1; c < 2 * kAccSplit; ++c) {   // 16-column chunks: k step c / 2, hi (even) or lo (odd)
-          if (a.lo || !(c & 1)) {
+      const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + buf * acols;
+      // sums of activation rows [m0, m0 + 16) for accumulator row r: the ksplit accumulators and
+      // their hi / lo halves added up
+      auto load_chunk = [&](int m0, float (&v)[16]) {
+        tmem_ld16(ta + m0, v);
+        for (int ai = 0; ai < ksplit; ++ai) {
+          for (int half = 0; half < (a.lo ? 2 : 1); ++half) {
+            if (ai == 0 && half == 0) continue;
             float vp[16];
-            tmem_ld16(ta + c * kN, vp);
+            tmem_ld16(ta + ai * 2 * Mp + half * Mp + m0, vp);
 #pragma unroll
             for (int m = 0; m < 16; ++m) v[m] += vp[m];
           }
         }
+      };
+      const int slot = (t == segs.t0) ? 0 : 1;   // partial tiles: 0 = this CTA's first segment, 1 = its last
+      float* P = a.partials + ((size_t)blockIdx.x * 2 + slot) * kMaxRows * 128;
+      for (int m0 = 0; m0 < a.M; m0 += 16) {
+        float v[16];
+        load_chunk(m0, v);
+        if (whole) {
+#pragma unroll
+          for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
+          if (m0 + 16 >= a.M) {   // the accumulator is read: the MMA warp may reuse it
+            fence_before_sync();
+            mbar_arrive(&ctl.acc_empty[buf]);
+          }
+          tile_epilogue<EPI>(a, ctl, t, r, q, lane, m0, min(16, a.M - m0));
+        } else {
+#pragma unroll
+          for (int m = 0; m < 16; ++m)
+            if (m0 + m < a.M) P[(m0 + m) * 128 + r] = v[m];
+        }
       }
-      fence_before_sync();
-      mbar_arrive(&ctl.acc_empty[buf]);
-      bool finish = whole;   // this CTA runs the tile's epilogue
-      if (whole) {
-#pragma unroll
-        for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
-      } else {
-        // partial tile: slot 0 = this CTA's first segment, slot 1 = its last one
-        const int slot = (t == segs.t0) ? 0 : 1;
-        float* P = a.partials + ((size_t)blockIdx.x * 2 + slot) * 16 * 128;
-#pragma unroll
-        for (int m = 0; m < 16; ++m)
-          if (m < a.M) P[m * 128 + r] = v[m];
+      if (!whole) {
+        fence_before_sync();
+        mbar_arrive(&ctl.acc_empty[buf]);
         epi_sync();
         const int c_first = unit_owner(t_begin, U, G), c_last = unit_owner(t_end - 1, U, G);
         if (et == 0) {
@@ -869,38 +889,40 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         const bool last = ctl.tile_last != 0;
         epi_sync();   // everyone has read the flag before a later segment rewrites it
         if (last) {
-          // sum of the partials in CTA order (it does not depend on who came last); the loads
-          // of up to eight contributors are issued together
-          for (int m = 0; m < a.M; ++m) ctl.acc[m * 128 + r] = 0.f;
-          for (int cb0 = c_first; cb0 <= c_last; cb0 += 8) {
-            int off[8];   // element offset of contributor cb0 + j's partial, -1: none
+          // sum of the partials in CTA order (it does not depend on who came last), 16 rows at a
+          // time; the loads of up to eight contributors are issued together
+          for (int m0 = 0; m0 < a.M; m0 += 16) {
+            const int mc = min(16, a.M - m0);
+            for (int m = 0; m < mc; ++m) ctl.acc[m * 128 + r] = 0.f;
+            for (int cb0 = c_first; cb0 <= c_last; cb0 += 8) {
+              int off[8];   // element offset of contributor cb0 + j's partial, -1: none
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const int c = cb0 + j;
-              off[j] = -1;
-              if (c <= c_last) {
-                const int cb = unit_begin(c, U, G);
-                if (cb < unit_begin(c + 1, U, G)) {   // else a CTA without units
-                  const int sl = (c == c_first && cb / a.KB != t) ? 1 : 0;
-                  off[j] = (c * 2 + sl) * 16 * 128 + r;
+              for (int j = 0; j < 8; ++j) {
+                const int c = cb0 + j;
+                off[j] = -1;
+                if (c <= c_last) {
+                  const int cb = unit_begin(c, U, G);
+                  if (cb < unit_begin(c + 1, U, G)) {   // else a CTA without units
+                    const int sl = (c == c_first && cb / a.KB != t) ? 1 : 0;
+                    off[j] = (c * 2 + sl) * kMaxRows * 128 + m0 * 128 + r;
+                  }
                 }
               }
-            }
 #pragma unroll 1
-            for (int m = 0; m < a.M; ++m) {
-              float x[8];
+              for (int m = 0; m < mc; ++m) {
+                float x[8];
 #pragma unroll
-              for (int j = 0; j < 8; ++j) x[j] = off[j] >= 0 ? __ldcg(a.partials + off[j] + m * 128) : 0.f;
-              float sum = ctl.acc[m * 128 + r];
+                for (int j = 0; j < 8; ++j) x[j] = off[j] >= 0 ? __ldcg(a.partials + off[j] + m * 128) : 0.f;
+                float sum = ctl.acc[m * 128 + r];
 #pragma unroll
-              for (int j = 0; j < 8; ++j) sum += x[j];
-              ctl.acc[m * 128 + r] = sum;
+                for (int j = 0; j < 8; ++j) sum += x[j];
+                ctl.acc[m * 128 + r] = sum;
+              }
             }
+            tile_epilogue<EPI>(a, ctl, t, r, q, lane, m0, mc);
           }
-          finish = true;
         }
       }
-      if (finish) tile_epilogue<EPI>(a, ctl, t, r, q, lane);
     }
     fence_before_sync();
   }
@@ -1019,7 +1041,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   }
   if (warp == 1) {
     fence_after_sync();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols(a.Mp)) : "memory");
   }
 }
 
@@ -1110,10 +1132,19 @@ bool make_map(CUtensorMap* m, const void* base, size_t rows, size_t cols, int bo
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+struct PlaneMaps {   // one activation plane with boxes of 16, 32, 64 and 128 rows
+  CUtensorMap m[4];
+};
 struct UmmaMaps {
   CUtensorMap w_fc, w_q, w_k, w_v, w_o, w_gate, w_up, w_down, w_lm;
-  CUtensorMap xin, x0_hi, x0_lo, attn_hi, attn_lo, a_hi, a_lo, act_hi, act_lo, hdn_hi, hdn_lo;
+  PlaneMaps xin, x0_hi, x0_lo, attn_hi, attn_lo, a_hi, a_lo, act_hi, act_lo, hdn_hi, hdn_lo;
 };
+
+bool make_plane_maps(PlaneMaps* pm, const void* base, size_t cols) {
+  for (int i = 0; i < 4; ++i)
+    if (!make_map(&pm->m[i], base, umma::kMaxRows, cols, 16 << i)) return false;
+  return true;
+}
 
 UmmaMaps* build_maps(const ps_ctx* c, const FusedScratch& f) {
   const ps_config& g = c->cfg;
@@ -1129,12 +1160,12 @@ UmmaMaps* build_maps(const ps_ctx* c, const FusedScratch& f) {
             make_map(&u->w_o, w.w_o, H, Hq, 128) && make_map(&u->w_gate, w.w_gate, F, H, 64) &&
             make_map(&u->w_up, w.w_up, F, H, 64) && make_map(&u->w_down, w.w_down, H, F, 128) &&
             make_map(&u->w_lm, w.w_lm, V, H, 128);
-  ok = ok && make_map(&u->xin, f.xin, kMaxM, 2 * H, 16) && make_map(&u->x0_hi, f.x0p.hi, kMaxM, H, 16) &&
-       make_map(&u->x0_lo, f.x0p.lo, kMaxM, H, 16) && make_map(&u->attn_hi, f.attnp.hi, kMaxM, Hq, 16) &&
-       make_map(&u->attn_lo, f.attnp.lo, kMaxM, Hq, 16) && make_map(&u->a_hi, f.ap.hi, kMaxM, H, 16) &&
-       make_map(&u->a_lo, f.ap.lo, kMaxM, H, 16) && make_map(&u->act_hi, f.actp.hi, kMaxM, F, 16) &&
-       make_map(&u->act_lo, f.actp.lo, kMaxM, F, 16) && make_map(&u->hdn_hi, f.hdnp.hi, kMaxM, H, 16) &&
-       make_map(&u->hdn_lo, f.hdnp.lo, kMaxM, H, 16);
+  ok = ok && make_plane_maps(&u->xin, f.xin, 2 * H) && make_plane_maps(&u->x0_hi, f.x0p.hi, H) &&
+       make_plane_maps(&u->x0_lo, f.x0p.lo, H) && make_plane_maps(&u->attn_hi, f.attnp.hi, Hq) &&
+       make_plane_maps(&u->attn_lo, f.attnp.lo, Hq) && make_plane_maps(&u->a_hi, f.ap.hi, H) &&
+       make_plane_maps(&u->a_lo, f.ap.lo, H) && make_plane_maps(&u->act_hi, f.actp.hi, F) &&
+       make_plane_maps(&u->act_lo, f.actp.lo, F) && make_plane_maps(&u->hdn_hi, f.hdnp.hi, H) &&
+       make_plane_maps(&u->hdn_lo, f.hdnp.lo, H);
   if (!ok) {
     delete u;
     return nullptr;
@@ -1144,8 +1175,11 @@ UmmaMaps* build_maps(const ps_ctx* c, const FusedScratch& f) {
 
 template <int EPI>
 ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
-                      const CUtensorMap& bh, const CUtensorMap& bl, UArgs& a, const FusedScratch& f,
+                      const PlaneMaps& ph, const PlaneMaps& pl, UArgs& a, const FusedScratch& f,
                       cudaStream_t st) {
+  const int mi = a.M <= 16 ? 0 : a.M <= 32 ? 1 : a.M <= 64 ? 2 : 3;
+  a.Mp = 16 << mi;
+  const CUtensorMap &bh = ph.m[mi], &bl = pl.m[mi];
   a.KB = (a.K + umma::kBK - 1) / umma::kBK;
   if (a.zip) {
     a.n_tiles = (a.N + 63) / 64;
@@ -1277,11 +1311,12 @@ static void ensure_maps(ps_ctx* c) {
 bool fused_supported(ps_ctx* c, int M) {
   const ps_config& g = c->cfg;
   if (g.dtype != PS_DTYPE_BF16 || (g.flags & PS_FLAG_UNFUSED_KERNELS)) return false;
-  if (M > kMaxM || (g.head_dim != 64 && g.head_dim != 128)) return false;
+  if (M > umma::kMaxRows || (g.head_dim != 64 && g.head_dim != 128)) return false;
   const int Hq = g.n_heads * g.head_dim;
   if (g.hidden % 8 || Hq % 8 || g.ffn % 8) return false;   // 16-byte operand rows
   ensure_maps(c);
   if (c->umma_maps) return true;
+  if (M > kMaxM) return false;   // the mma.sync kernels take 16 rows
   const int lim = c->smem_optin, n = c->n_sm;
   return choose_pass_cols(M, 2 * g.hidden, rows_cap_for(g.hidden, n, false), lim) &&
          choose_pass_cols(M, g.hidden, rows_cap_for(Hq + 2 * g.n_kv_heads * g.head_dim, n, false), lim) &&
@@ -1303,10 +1338,10 @@ ps_status fused_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* by
   FusedScratch f = carve_fused(g, (char*)c->fused_scratch);
   if (!std::strcmp(name, "qkv")) {
     *ptr = f.qkv;
-    *bytes = (size_t)kMaxM * (g.n_heads + 2 * g.n_kv_heads) * g.head_dim * 4;
+    *bytes = (size_t)umma::kMaxRows * (g.n_heads + 2 * g.n_kv_heads) * g.head_dim * 4;
     return PS_OK;
   }
-  if (!std::strcmp(name, "act")) { *ptr = f.act; *bytes = (size_t)kMaxM * g.ffn * 4; return PS_OK; }
+  if (!std::strcmp(name, "act")) { *ptr = f.act; *bytes = (size_t)umma::kMaxRows * g.ffn * 4; return PS_OK; }
   return PS_ERR_INVALID_ARG;
 }
 

@@ -43,16 +43,26 @@ using ws::smem_u32;
 
 constexpr int kTile = 128;                        // weight rows per tile (MMA M)
 constexpr int kBK = 64;                           // k columns per unit: one 128-byte swizzle span
-constexpr int kN = 16;                            // activation rows (MMA N)
+constexpr int kN = 16;                            // activation rows per epilogue chunk
+constexpr int kMaxRows = 128;                     // activation rows of a launch (padded to 16, 32, 64 or 128)
 constexpr int kABytes = kTile * kBK * 2;          // 16 KB
-constexpr int kBBytes = kN * kBK * 2;             // 2 KB per plane
+constexpr int kBBytes = kN * kBK * 2;             // 2 KB per plane at 16 rows
 constexpr int kStageBytes = kABytes + 2 * kBBytes;
-constexpr int kStages = 10;
+constexpr int kStages = 10;                       // at 16 rows; fewer, larger stages for more rows
+constexpr int kRingBytes = kStages * kStageBytes;
 constexpr int kThreads = 192;
 constexpr int kEpiThreads = 128;
-constexpr int kAccSplit = kBK / 16;               // independent partial accumulators, one per k step of a unit
-constexpr int kAccCols = kAccSplit * 2 * kN;      // accumulator columns: per k step hi products, lo products
-constexpr int kTmemCols = 2 * kAccCols;           // two accumulators
+// Geometry of a launch with Mp padded activation rows (16, 32, 64 or 128): the hi and lo planes
+// form one MMA operand of N = 2 Mp columns; ksplit independent accumulators per tile (one per k
+// step of a unit while tensor memory allows: MMAs into one accumulator serialise); two tiles'
+// accumulators in tensor memory.
+__host__ __device__ constexpr int stage_bytes(int Mp) { return kABytes + 2 * Mp * kBK * 2; }
+__host__ __device__ constexpr int n_stages(int Mp) {
+  return kRingBytes / stage_bytes(Mp) < kStages ? kRingBytes / stage_bytes(Mp) : kStages;
+}
+__host__ __device__ constexpr int k_split(int Mp) { return 256 / (2 * Mp) < kBK / 16 ? 256 / (2 * Mp) : kBK / 16; }
+__host__ __device__ constexpr int acc_cols(int Mp) { return k_split(Mp) * 2 * Mp; }
+__host__ __device__ constexpr int tmem_cols(int Mp) { return 2 * acc_cols(Mp); }   // 256 or 512
 // Instruction descriptor of kind::f16: fp32 accumulator, bf16 x bf16, both operands K-major,
 // N / 8 in bits [17,23), M / 16 in bits [24,29).
 constexpr uint32_t idesc(int n) {
@@ -134,7 +144,7 @@ struct Ctl {
   int abort_flag;
   int is_last;
   int tile_last;
-  float scale[kN];
+  float scale[kMaxRows];
   float red[4][kN];           // one value per epilogue warp and activation row
   float red2[4][kN];
   float cand_v[4][kN];        // top-n candidates per epilogue warp, and the row's previous pick
@@ -142,7 +152,7 @@ struct Ctl {
   float prev_v[kN];
   int prev_i[kN];
   float xch[kN * 64];         // gate/up exchange: [m][feature of the tile]
-  float acc[kN * 128];        // a tile's sums, [m][accumulator row]: each thread reads back its own
+  float acc[kN * 128];        // a chunk of a tile's sums, [m][accumulator row]: each thread reads back its own
 };
 
 constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + 1024;   // + alignment slack
