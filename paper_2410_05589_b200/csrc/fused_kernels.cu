@@ -702,7 +702,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
   }
 }
 
-template <int EPI>
+template <int EPI, int MP>
 __global__ void __launch_bounds__(umma::kThreads, 1)
 k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUtensorMap tA1,
             const __grid_constant__ CUtensorMap tA2, const __grid_constant__ CUtensorMap tBh,
@@ -724,7 +724,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   }
   if (warp == 1) {   // tensor memory for two accumulators
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
-                 "r"(tmem_cols(a.Mp))
+                 "r"(tmem_cols(MP))
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -737,8 +737,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   const int u0 = unit_begin(blockIdx.x, U, G), u1 = unit_begin(blockIdx.x + 1, U, G);
   const Segs segs(u0, u1, a.KB);
   volatile int* abort_flag = &ctl.abort_flag;
-  const int Mp = a.Mp, sbytes = stage_bytes(Mp), nst = n_stages(Mp), ksplit = k_split(Mp), acols = acc_cols(Mp);
-  const int plane_bytes = Mp * kBK * 2;
+  constexpr int Mp = MP, sbytes = stage_bytes(Mp), nst = n_stages(Mp), ksplit = k_split(Mp), acols = acc_cols(Mp);
+  constexpr int plane_bytes = Mp * kBK * 2;
 
   if (warp == 0) {
     if (lane == 0) {   // ---- TMA producer
@@ -800,7 +800,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
           const uint32_t sa = base + stage * sbytes;
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k) {   // k step k goes to accumulator k % ksplit
-            const int ai = k % ksplit;
+            const int ai = k & (ksplit - 1);   // ksplit is 1, 2 or 4
             mma_f16(d + ai * 2 * Mp, smem_desc(sa + k * 32), smem_desc(sa + kABytes + k * 32), id,
                     (acc || k >= ksplit) ? 1u : 0u);
           }
@@ -840,40 +840,32 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       // their hi / lo halves added up
       auto load_chunk = [&](int m0, float (&v)[16]) {
         tmem_ld16(ta + m0, v);
-        for (int ai = 0; ai < ksplit; ++ai) {
-          for (int half = 0; half < (a.lo ? 2 : 1); ++half) {
-            if (ai == 0 && half == 0) continue;
-            float vp[16];
-            tmem_ld16(ta + ai * 2 * Mp + half * Mp + m0, vp);
 #pragma unroll
-            for (int m = 0; m < 16; ++m) v[m] += vp[m];
-          }
+        for (int c = 1; c < 2 * ksplit; ++c) {   // accumulator c / 2, its hi (even) or lo (odd) half
+          if (!a.lo && (c & 1)) continue;
+          float vp[16];
+          tmem_ld16(ta + (c >> 1) * 2 * Mp + (c & 1) * Mp + m0, vp);
+#pragma unroll
+          for (int m = 0; m < 16; ++m) v[m] += vp[m];
         }
       };
       const int slot = (t == segs.t0) ? 0 : 1;   // partial tiles: 0 = this CTA's first segment, 1 = its last
       float* P = a.partials + ((size_t)blockIdx.x * 2 + slot) * kMaxRows * 128;
-      for (int m0 = 0; m0 < a.M; m0 += 16) {
-        float v[16];
-        load_chunk(m0, v);
-        if (whole) {
-#pragma unroll
-          for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
-          if (m0 + 16 >= a.M) {   // the accumulator is read: the MMA warp may reuse it
-            fence_before_sync();
-            mbar_arrive(&ctl.acc_empty[buf]);
-          }
-          tile_epilogue<EPI>(a, ctl, t, r, q, lane, m0, min(16, a.M - m0));
-        } else {
+      bool finish = whole;   // this CTA runs the tile's epilogue
+      int c_first = 0, c_last = 0;
+      if (!whole) {
+        for (int m0 = 0; m0 < a.M; m0 += 16) {
+          float v[16];
+          load_chunk(m0, v);
 #pragma unroll
           for (int m = 0; m < 16; ++m)
             if (m0 + m < a.M) P[(m0 + m) * 128 + r] = v[m];
         }
-      }
-      if (!whole) {
         fence_before_sync();
         mbar_arrive(&ctl.acc_empty[buf]);
         epi_sync();
-        const int c_first = unit_owner(t_begin, U, G), c_last = unit_owner(t_end - 1, U, G);
+        c_first = unit_owner(t_begin, U, G);
+        c_last = unit_owner(t_end - 1, U, G);
         if (et == 0) {
           // one thread publishes the block's partial (the barrier above ordered the other
           // threads' stores before this release) and, if it came last, acquires the others'
@@ -886,15 +878,26 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
           ctl.tile_last = last;
         }
         epi_sync();
-        const bool last = ctl.tile_last != 0;
+        finish = ctl.tile_last != 0;
         epi_sync();   // everyone has read the flag before a later segment rewrites it
-        if (last) {
-          // sum of the partials in CTA order (it does not depend on who came last), 16 rows at a
-          // time; the loads of up to eight contributors are issued together
-          for (int m0 = 0; m0 < a.M; m0 += 16) {
-            const int mc = min(16, a.M - m0);
+      }
+      if (finish) {
+        // 16 activation rows at a time: the tile's sums into ctl.acc (from tensor memory, or the
+        // partials added in CTA order, which does not depend on who came last), then the epilogue
+        for (int m0 = 0; m0 < a.M; m0 += 16) {
+          const int mc = min(16, a.M - m0);
+          if (whole) {
+            float v[16];
+            load_chunk(m0, v);
+#pragma unroll
+            for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
+            if (m0 + 16 >= a.M) {   // the accumulator is read: the MMA warp may reuse it
+              fence_before_sync();
+              mbar_arrive(&ctl.acc_empty[buf]);
+            }
+          } else {
             for (int m = 0; m < mc; ++m) ctl.acc[m * 128 + r] = 0.f;
-            for (int cb0 = c_first; cb0 <= c_last; cb0 += 8) {
+            for (int cb0 = c_first; cb0 <= c_last; cb0 += 8) {   // loads of eight contributors at once
               int off[8];   // element offset of contributor cb0 + j's partial, -1: none
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
@@ -919,8 +922,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
                 ctl.acc[m * 128 + r] = sum;
               }
             }
-            tile_epilogue<EPI>(a, ctl, t, r, q, lane, m0, mc);
           }
+          tile_epilogue<EPI>(a, ctl, t, r, q, lane, m0, mc);
         }
       }
     }
@@ -1041,7 +1044,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   }
   if (warp == 1) {
     fence_after_sync();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols(a.Mp)) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols(MP)) : "memory");
   }
 }
 
@@ -1195,7 +1198,8 @@ ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, c
   }
   if ((long long)a.n_tiles * a.KB * (c->n_sm + 1) >= (1ll << 31)) return fail(c, PS_ERR_UNSUPPORTED, "too many GEMM units");
   a.partials = f.partials; a.tile_tickets = f.tile_tickets; a.status = c->dev_status;
-  auto kern = k_umma_gemm<EPI>;
+  auto kern = mi == 0 ? k_umma_gemm<EPI, 16> : mi == 1 ? k_umma_gemm<EPI, 32> : mi == 2 ? k_umma_gemm<EPI, 64>
+                                                                                     : k_umma_gemm<EPI, 128>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, umma::kSmemBytes);
   if (e != cudaSuccess) return cuda_check(c, e, "umma smem attribute");
   e = launch_after(kern, dim3(c->n_sm), dim3(umma::kThreads), umma::kSmemBytes, st, !c->prof, a0, a1, a2, bh, bl, a);

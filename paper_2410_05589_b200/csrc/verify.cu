@@ -337,14 +337,15 @@ struct CluScratch {
   double d[kCluWarps], d2[kCluWarps];
 };
 
-// (The cluster size is a launch attribute: 8 blocks, 16 for vocabularies beyond 65536.)
-__global__ void __launch_bounds__(kCluThreads) k_verify_cluster(VerifyArgs a) {
+// (NCLU blocks per cluster: 8, or 16 for vocabularies beyond 65536.)
+template <int NCLU>
+__device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
   namespace cg = cooperative_groups;
   cg::cluster_group cl = cg::this_cluster();
   __shared__ CluPart part;
   __shared__ CluScratch s;
   const int rank = (int)cl.block_rank();
-  const int nclu = (int)cl.num_blocks();
+  constexpr int nclu = NCLU;
   const int i = blockIdx.x / nclu, b = blockIdx.y, V = a.V;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool bonus = i >= a.n_draft;
@@ -568,6 +569,14 @@ __global__ void __launch_bounds__(kCluThreads) k_verify_cluster(VerifyArgs a) {
   cl.sync();   // no block leaves while another may still read its shared memory
 }
 
+
+// The 8-block cluster is fixed at compile time; the 16-block one (an opt-in size) is a launch attribute.
+__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads) k_verify_cluster(VerifyArgs a) {
+  verify_cluster_body<kClu>(a);
+}
+__global__ void __launch_bounds__(kCluThreads) k_verify_cluster16(VerifyArgs a) {
+  verify_cluster_body<16>(a);
+}
 
 // ---- token-tree verification (Algorithm 1 in full) -------------------------------------------
 // One cluster per (decision row, sequence): row u = 0 is the root, u = 1 + i the node i.  The
@@ -943,10 +952,16 @@ ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* 
   a.rec = c->vrec; a.tickets = c->tickets; a.status = c->dev_status;
   const bool aligned = (((uintptr_t)target_logits | (uintptr_t)draft_logits) & 15u) == 0;
   const int nclu = a.V <= kCluMaxVocab ? kClu : 16;
-  if (a.V % 4 == 0 && a.V <= kCluMaxVocab16 && aligned && cluster_size_ok(k_verify_cluster, nclu)) {
+  if (a.V % 4 == 0 && a.V <= kCluMaxVocab16 && aligned && (nclu == kClu || cluster_size_ok(k_verify_cluster16, 16))) {
     prof_mark(c, st, "begin");
     // (a plain launch: joining the dependent-launch chain here was measured to cost 7 us a step)
-    cudaError_t e = launch_cluster(k_verify_cluster, dim3(n_target * nclu, B), nclu, st, a);
+    cudaError_t e;
+    if (nclu == kClu) {
+      k_verify_cluster<<<dim3(n_target * kClu, B), kCluThreads, 0, st>>>(a);
+      e = cudaGetLastError();
+    } else {
+      e = launch_cluster(k_verify_cluster16, dim3(n_target * 16, B), 16, st, a);
+    }
     c->launches++;
     prof_mark(c, st, "verify");
     return cuda_check(c, e, "k_verify_cluster");

@@ -25,7 +25,8 @@ def test_workspace_bytes_and_config_checks_on_host():
     ok = ps_config(1, 5120, 40, 40, 128, 13824, 32000, 4, 1, 1024 + 5, 10000.0, 1e-5, 0)
     n = lib.ps_workspace_bytes(C.byref(ok))
     kv = 2 * 40 * 1029 * 128 * 2
-    assert kv < n < kv + (64 << 20)
+    # (scratch is sized for the 128 rows the tensor-core path takes, whatever max_batch is)
+    assert kv < n < kv + (160 << 20)
     for field, bad in (("head_dim", 96), ("hidden", 5121), ("k_masks", 16), ("max_batch", 0),
                        ("max_batch", 129), ("dtype", 2), ("n_kv_heads", 3), ("max_ctx", 2)):
         cfg = ps_config(1, 5120, 40, 40, 128, 13824, 32000, 4, 1, 1029, 10000.0, 1e-5, 0)
