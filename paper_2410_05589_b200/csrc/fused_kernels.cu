@@ -559,12 +559,13 @@ __device__ __forceinline__ int tile_feature(const UArgs& a, int t, int r, bool& 
 
 // Epilogue of one finished tile for the activation rows [m0, m0 + mc), mc <= 16; called by the
 // 128 epilogue threads after each has put its accumulator row r (= 32 * q + lane) of those
-// rows into ctl.acc[(m - m0) * 128 + r].  The loops
+// rows into ctl.acc[(m - m0) * 128 + r].  A dry call executes the same instructions and writes
+// nothing to global memory.  The loops
 // over m are rolled on purpose: this code runs once or twice per CTA, so what it costs is the
 // fetch of its instructions, not their execution.
 template <int EPI>
 __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane,
-                                              int m0, int mc) {
+                                              int m0, int mc, bool dry) {
   using namespace umma;
   const int et = r;
   bool valid;
@@ -573,25 +574,35 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
   if (EPI == EPI_STORE) {
     const float bias = (a.bias && valid) ? __bfloat162float(a.bias[n]) : 0.f;
     const float gain = (a.gain_next && valid) ? __bfloat162float(a.gain_next[n]) : 1.f;
+    // eight rows at a time, so that their residual loads are in flight together
 #pragma unroll 1
-    for (int m = 0; m < mc; ++m) {
-      float sq = 0.f;
-      if (valid) {
-        float x = acc[m * 128] * ctl.scale[m0 + m] + bias;
-        if (a.res) x += a.res[(size_t)(m0 + m) * a.ldr + n];
-        a.out[(size_t)(m0 + m) * a.ldo + n] = x;
-        sq = x * x;
-        if (a.out_hi)
-          split_store(a.out_hi + (size_t)(m0 + m) * a.ld_plane + n, a.out_lo + (size_t)(m0 + m) * a.ld_plane + n, x * gain);
-      }
-      if (a.ssq_out) {
-        sq = warp_sum(sq);
-        if (lane == 0) ctl.red[q][m] = sq;
+    for (int mg = 0; mg < mc; mg += 8) {
+      float rv[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        rv[j] = (a.res && valid && mg + j < mc) ? __ldcg(a.res + (size_t)(m0 + mg + j) * a.ldr + n) : 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int m = mg + j;
+        if (m < mc) {   // uniform across the threads
+          float sq = 0.f;
+          if (valid && !dry) {
+            const float x = acc[m * 128] * ctl.scale[m0 + m] + bias + rv[j];
+            a.out[(size_t)(m0 + m) * a.ldo + n] = x;
+            sq = x * x;
+            if (a.out_hi)
+              split_store(a.out_hi + (size_t)(m0 + m) * a.ld_plane + n, a.out_lo + (size_t)(m0 + m) * a.ld_plane + n, x * gain);
+          }
+          if (a.ssq_out) {
+            sq = warp_sum(sq);
+            if (lane == 0) ctl.red[q][m] = sq;
+          }
+        }
       }
     }
     if (a.ssq_out) {
       epi_sync();
-      if (et < mc) a.ssq_out[(size_t)t * a.M + m0 + et] = (ctl.red[0][et] + ctl.red[1][et]) + (ctl.red[2][et] + ctl.red[3][et]);
+      if (et < mc && !dry) a.ssq_out[(size_t)t * a.M + m0 + et] = (ctl.red[0][et] + ctl.red[1][et]) + (ctl.red[2][et] + ctl.red[3][et]);
       epi_sync();
     }
   } else if (EPI == EPI_SWIGLU) {
@@ -600,7 +611,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
       for (int m = 0; m < mc; ++m) ctl.xch[m * 64 + (r - 64)] = acc[m * 128] * ctl.scale[m0 + m];
     }
     epi_sync();
-    if (r < 64 && valid) {
+    if (r < 64 && valid && !dry) {
 #pragma unroll 1
       for (int m = 0; m < mc; ++m) {
         const float gv = acc[m * 128] * ctl.scale[m0 + m], uv = ctl.xch[m * 64 + r];
@@ -614,7 +625,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
 #pragma unroll 1
     for (int m = 0; m < mc; ++m) {
       const float x = acc[m * 128] * ctl.scale[m0 + m];
-      if (valid && a.logits_out) a.logits_out[(size_t)(m0 + m) * a.N + n] = x;
+      if (valid && a.logits_out && !dry) a.logits_out[(size_t)(m0 + m) * a.N + n] = x;
       float mx = valid ? x : -FLT_MAX;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -628,7 +639,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
       if (lane == 0) ctl.red2[q][m] = s;
     }
     epi_sync();
-    if (et < mc) {
+    if (et < mc && !dry) {
       LmPart* p = a.parts + (size_t)t * a.M + m0 + et;
       p->vmax = fmaxf(fmaxf(ctl.red[0][et], ctl.red[1][et]), fmaxf(ctl.red[2][et], ctl.red[3][et]));
       p->sumexp = (ctl.red2[0][et] + ctl.red2[1][et]) + (ctl.red2[2][et] + ctl.red2[3][et]);
@@ -661,9 +672,11 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
           if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
         ctl.prev_v[et] = bv; ctl.prev_i[et] = bi;
-        LmPart* p = a.parts + (size_t)t * a.M + m0 + et;
-        p->top_v[tn] = bv; p->top_i[tn] = bi;
-        if (tn == 0) { p->v0 = bv; p->i0 = bi; }
+        if (!dry) {
+          LmPart* p = a.parts + (size_t)t * a.M + m0 + et;
+          p->top_v[tn] = bv; p->top_i[tn] = bi;
+          if (tn == 0) { p->v0 = bv; p->i0 = bi; }
+        }
       }
       epi_sync();
     }
@@ -694,13 +707,17 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
           const float ov = ctl.cand_v[w][et]; const int oi = ctl.cand_i[w][et];
           if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
         }
-        LmPart* p = a.parts + (size_t)t * a.M + m0 + et;
-        p->sv = bv; p->si = bi;
+        if (!dry) {
+          LmPart* p = a.parts + (size_t)t * a.M + m0 + et;
+          p->sv = bv; p->si = bi;
+        }
       }
     }
     epi_sync();   // red / red2 / cand are free again
   }
 }
+
+static_assert(umma::kMaxCtas >= kMaxSm, "contributor table covers every CTA of a launch");
 
 template <int EPI, int MP>
 __global__ void __launch_bounds__(umma::kThreads, 1)
@@ -814,26 +831,34 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   } else {
     // ---- epilogue warps: accumulator row r = 32 q + lane
     const int q = warp & 3, r = 32 * q + lane, et = r;
-    pdl_wait();   // everything below reads or writes what the kernel before this one touches
-    for (int m = warp - 2; m < a.M; m += 4) {   // RMSNorm row scales of the input
-      float sc = 1.f;
-      if (a.ssq_in) {
-        float ss = 0.f;
-        for (int c = lane; c < a.ssq_n; c += 32) ss += a.ssq_in[(size_t)c * a.M + m];
-        ss = warp_sum(ss);
-        sc = rsqrtf(ss / (float)a.K + a.eps);
+    // Pass -1 is a rehearsal: the reduction and epilogue code below runs once per CTA or
+    // twice, at the very end for most CTAs, and its first execution costs several microseconds
+    // of instruction fetches.  The rehearsal takes them before the kernel ahead of this one has
+    // finished: it sums this CTA's own (stale) partial slot, runs the epilogue dry, and what it
+    // reads may be in flux because nothing of it is kept.
+    for (int seg = segs.n > 0 ? -1 : 0; seg < segs.n; ++seg) {
+      const bool dry = seg < 0;
+      if (seg == 0) {
+        pdl_wait();   // everything below reads or writes what the kernel before this one touches
+        for (int m = warp - 2; m < a.M; m += 4) {   // RMSNorm row scales of the input
+          float sc = 1.f;
+          if (a.ssq_in) {
+            float ss = 0.f;
+            for (int c = lane; c < a.ssq_n; c += 32) ss += a.ssq_in[(size_t)c * a.M + m];
+            ss = warp_sum(ss);
+            sc = rsqrtf(ss / (float)a.K + a.eps);
+          }
+          if (lane == 0) ctl.scale[m] = sc;
+        }
+        epi_sync();
       }
-      if (lane == 0) ctl.scale[m] = sc;
-    }
-    epi_sync();
-    for (int seg = 0; seg < segs.n; ++seg) {
       int t, sb, se;
-      segs.get(seg, t, sb, se);
+      segs.get(dry ? 0 : seg, t, sb, se);
       const int t_begin = t * a.KB, t_end = t_begin + a.KB;
-      const bool whole = se - sb == a.KB;
+      const bool whole = !dry && se - sb == a.KB;
       const int buf = seg & 1;
       // all four warps take the same decision although each thread waits for itself
-      if (epi_any(!mbar_wait(&ctl.acc_full[buf], (seg >> 1) & 1, abort_flag))) break;
+      if (!dry && epi_any(!mbar_wait(&ctl.acc_full[buf], (seg >> 1) & 1, abort_flag))) break;
       fence_after_sync();
       const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + buf * acols;
       // sums of activation rows [m0, m0 + 16) for accumulator row r: the ksplit accumulators and
@@ -851,9 +876,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       };
       const int slot = (t == segs.t0) ? 0 : 1;   // partial tiles: 0 = this CTA's first segment, 1 = its last
       float* P = a.partials + ((size_t)blockIdx.x * 2 + slot) * kMaxRows * 128;
-      bool finish = whole;   // this CTA runs the tile's epilogue
-      int c_first = 0, c_last = 0;
-      if (!whole) {
+      bool finish = whole || dry;   // this CTA runs the tile's epilogue
+      int c_first = blockIdx.x, c_last = blockIdx.x;
+      if (!whole && !dry) {
         for (int m0 = 0; m0 < a.M; m0 += 16) {
           float v[16];
           load_chunk(m0, v);
@@ -881,6 +906,18 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         finish = ctl.tile_last != 0;
         epi_sync();   // everyone has read the flag before a later segment rewrites it
       }
+      if (finish && !whole) {   // where each contributor's partial lies (a CTA without units has none)
+        for (int j = et; j <= c_last - c_first; j += kEpiThreads) {
+          const int c = c_first + j, cb = unit_begin(c, U, G);
+          int off = -1;
+          if (cb < unit_begin(c + 1, U, G)) {
+            const int sl = (c == c_first && cb / a.KB != t) ? 1 : 0;
+            off = (c * 2 + sl) * kMaxRows * 128;
+          }
+          ctl.coff[j] = off;
+        }
+        epi_sync();
+      }
       if (finish) {
         // 16 activation rows at a time: the tile's sums into ctl.acc (from tensor memory, or the
         // partials added in CTA order, which does not depend on who came last), then the epilogue
@@ -896,34 +933,38 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
               mbar_arrive(&ctl.acc_empty[buf]);
             }
           } else {
-            for (int m = 0; m < mc; ++m) ctl.acc[m * 128 + r] = 0.f;
-            for (int cb0 = c_first; cb0 <= c_last; cb0 += 8) {   // loads of eight contributors at once
-              int off[8];   // element offset of contributor cb0 + j's partial, -1: none
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                const int c = cb0 + j;
-                off[j] = -1;
-                if (c <= c_last) {
-                  const int cb = unit_begin(c, U, G);
-                  if (cb < unit_begin(c + 1, U, G)) {   // else a CTA without units
-                    const int sl = (c == c_first && cb / a.KB != t) ? 1 : 0;
-                    off[j] = (c * 2 + sl) * kMaxRows * 128 + m0 * 128 + r;
-                  }
-                }
-              }
+            // (row, contributor) pairs in row-major order, kN at a time: a rolled loop sends
+            // each pair's value on its way into shared memory (asynchronous copies, nothing
+            // waits on a register), one wait, a rolled loop adds them up.  The values come from
+            // L2 while the next launch's weight requests keep it busy, and the code runs once:
+            // round trips and instruction fetches are what it costs.
+            const int nc = c_last - c_first + 1, total = mc * nc;
+            const float* Pr = a.partials + m0 * 128 + r;
+            float* land = ctl.land + r;
+            int m = 0, j = 0, mm = 0, jj = 0;
+            float sum = 0.f;   // of row m so far, contributors in CTA order
 #pragma unroll 1
-              for (int m = 0; m < mc; ++m) {
-                float x[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) x[j] = off[j] >= 0 ? __ldcg(a.partials + off[j] + m * 128) : 0.f;
-                float sum = ctl.acc[m * 128 + r];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) sum += x[j];
-                ctl.acc[m * 128 + r] = sum;
+            for (int i0 = 0; i0 < total; i0 += kN) {
+              const int nb = min(kN, total - i0);
+#pragma unroll 1
+              for (int u = 0; u < nb; ++u) {
+                const int o = ctl.coff[jj];
+                if (o >= 0) cp_async_4(land + u * 128, Pr + o + mm * 128);
+                else land[u * 128] = 0.f;
+                if (++jj == nc) { jj = 0; ++mm; }
+              }
+              cp_async_wait_all();   // each thread reads back what it asked for itself
+#pragma unroll 1
+              for (int u = 0; u < nb; ++u) {
+                sum += land[u * 128];
+                if (++j == nc) {
+                  ctl.acc[m * 128 + r] = sum;
+                  sum = 0.f; j = 0; ++m;
+                }
               }
             }
           }
-          tile_epilogue<EPI>(a, ctl, t, r, q, lane, m0, mc);
+          tile_epilogue<EPI>(a, ctl, t, r, q, lane, m0, mc, dry);
         }
       }
     }
@@ -1448,6 +1489,3 @@ ps_status fused_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
 }
 
 }  // namespace ps
-
-
-

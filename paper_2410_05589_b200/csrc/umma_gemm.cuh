@@ -116,6 +116,14 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// 4-byte asynchronous copy global -> shared and the wait for this thread's copies.
+__device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+}
+
 __device__ __forceinline__ void epi_sync() {
   asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 }
@@ -135,6 +143,8 @@ __device__ __forceinline__ bool epi_any(bool pred) {
 }
 
 // ---- control block behind the stages ----------------------------------------------------------
+constexpr int kMaxCtas = 192;   // CTAs of one launch (one per SM)
+
 struct Ctl {
   uint64_t full[kStages];     // a stage's boxes have landed
   uint64_t empty[kStages];    // the MMAs that read a stage have completed
@@ -153,6 +163,8 @@ struct Ctl {
   int prev_i[kN];
   float xch[kN * 64];         // gate/up exchange: [m][feature of the tile]
   float acc[kN * 128];        // a chunk of a tile's sums, [m][accumulator row]: each thread reads back its own
+  float land[kN * 128];       // partials of a shared tile on their way in: [pair of a batch][accumulator row]
+  int coff[kMaxCtas];         // a shared tile's contributors: element offset of each one's partial, -1: none
 };
 
 constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(Ctl) + 1024;   // + alignment slack
