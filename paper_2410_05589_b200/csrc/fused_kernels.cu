@@ -684,7 +684,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
 #pragma unroll 1
       for (int m = 0; m < mc; ++m) {
         const int sb = (m0 + m) / a.R;
-        const uint32_t row_id = (uint32_t)sb | ((uint32_t)(m0 + m - sb * a.R) << 8);
+        const uint32_t row_id = ((uint32_t)sb + a.sa.b_base) | ((uint32_t)(m0 + m - sb * a.R) << 8);
         float bv = -FLT_MAX;
         int bi = 0x7fffffff;
         if (valid) {
@@ -1369,6 +1369,11 @@ bool fused_supported(ps_ctx* c, int M) {
          choose_pass_cols(M, g.hidden, rows_cap_for(g.ffn, n, true), lim) &&
          choose_pass_cols(M, g.ffn, rows_cap_for(g.hidden, n, false), lim) &&
          choose_pass_cols(M, g.hidden, rows_cap_for(g.vocab, n, false), lim);
+}
+
+int fused_row_limit(ps_ctx* c) {
+  if (fused_supported(c, umma::kMaxRows)) return umma::kMaxRows;
+  return fused_supported(c, kMaxM) ? kMaxM : 0;
 }
 
 size_t fused_scratch_bytes(const ps_config& g) { return carve_fused(g, nullptr).bytes; }

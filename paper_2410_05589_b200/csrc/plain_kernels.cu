@@ -331,7 +331,7 @@ __global__ void __launch_bounds__(256) k_gumbel_argmax(const float* logits, int 
   __shared__ float s_v[8];
   __shared__ int s_i[8];
   const int m = blockIdx.x, b = m / R, j = m - b * R;
-  const uint32_t row_id = (uint32_t)b | ((uint32_t)j << 8);
+  const uint32_t row_id = ((uint32_t)b + sa.b_base) | ((uint32_t)j << 8);
   const float* row = logits + (size_t)m * V;
   float bv = -FLT_MAX;
   int bi = 0x7fffffff;

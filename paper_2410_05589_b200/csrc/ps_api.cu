@@ -317,6 +317,45 @@ ps_status ps_kv_append(ps_ctx* c, int B, const int* seq_slot, const int* n_new,
   return PS_OK;
 }
 
+// Runs the draft rows of the B sequences in `sm` (R rows each, outputs laid out [B][R][...]).
+// The tensor-core path takes a bounded number of rows per launch, so a larger batch is cut into
+// groups of whole sequences (sequences are independent; each group streams the weights once);
+// shapes the fused kernels do not take run on the plain kernels in one piece.
+static ps_status run_draft_rows(ps_ctx* c, const SeqMap& sm, int B, const void* hidden, const int* tokens,
+                                int top_n, int* top_ids, float* top_logit, float* row_max, float* row_lse,
+                                float* logits_out, float* feat_out, const SampleArgs* sa, cudaStream_t st) {
+  const ps_config& g = c->cfg;
+  const int R = g.k_masks + 1;
+  if (fused_supported(c, B * R))
+    return fused_draft_step(c, sm, B, hidden, tokens, top_n, top_ids, top_logit, row_max, row_lse,
+                            logits_out, feat_out, sa, st);
+  const int per_max = fused_row_limit(c) / R;
+  if (per_max < 1)
+    return plain_draft_step(c, sm, B, hidden, tokens, top_n, top_ids, top_logit, row_max, row_lse,
+                            logits_out, feat_out, sa, st);
+  const int n_chunks = (B + per_max - 1) / per_max, per = (B + n_chunks - 1) / n_chunks;
+  const size_t eb = g.dtype == PS_DTYPE_F32 ? 4 : 2;
+  for (int b0 = 0; b0 < B; b0 += per) {
+    const int nb = std::min(per, B - b0);
+    SeqMap sub;
+    std::memset(&sub, 0, sizeof(sub));
+    sub.B = nb;
+    for (int b = 0; b < nb; ++b) { sub.slot[b] = sm.slot[b0 + b]; sub.len[b] = sm.len[b0 + b]; sub.row_off[b] = b * R; }
+    sub.row_off[nb] = nb * R;
+    const size_t r0 = (size_t)b0 * R;
+    SampleArgs sub_sa;
+    if (sa) { sub_sa = *sa; sub_sa.b_base = sa->b_base + (uint32_t)b0; sub_sa.sampled = sa->sampled + r0; }
+    ps_status s = fused_draft_step(
+        c, sub, nb, hidden ? (const char*)hidden + (size_t)b0 * g.hidden * eb : nullptr, tokens + b0, top_n,
+        top_ids ? top_ids + r0 * top_n : nullptr, top_logit ? top_logit + r0 * top_n : nullptr,
+        row_max ? row_max + r0 : nullptr, row_lse ? row_lse + r0 : nullptr,
+        logits_out ? logits_out + r0 * g.vocab : nullptr, feat_out ? feat_out + r0 * g.hidden : nullptr,
+        sa ? &sub_sa : nullptr, st);
+    if (s != PS_OK) return s;
+  }
+  return PS_OK;
+}
+
 static ps_status draft_common(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,
                               const int* token_last, int top_n, int* top_ids, float* top_logit,
                               float* row_max, float* row_lse, float* logits_out, float* feat_out,
@@ -340,11 +379,8 @@ static ps_status draft_common(ps_ctx* c, int B, const int* seq_slot, const void*
     if (sm.len[b] + R > c->cfg.max_ctx) return fail(c, PS_ERR_CAPACITY, "no room for the draft rows");
   }
   sm.row_off[B] = B * R;
-  if (fused_supported(c, B * R))
-    return fused_draft_step(c, sm, B, hidden_last, token_last, top_n, top_ids, top_logit, row_max,
-                            row_lse, logits_out, feat_out, sa, (cudaStream_t)stream);
-  return plain_draft_step(c, sm, B, hidden_last, token_last, top_n, top_ids, top_logit, row_max,
-                          row_lse, logits_out, feat_out, sa, (cudaStream_t)stream);
+  return run_draft_rows(c, sm, B, hidden_last, token_last, top_n, top_ids, top_logit, row_max, row_lse,
+                        logits_out, feat_out, sa, (cudaStream_t)stream);
 }
 
 ps_status ps_draft_step(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,
@@ -368,6 +404,7 @@ ps_status ps_draft_step_sampled(ps_ctx* c, int B, const int* seq_slot, const voi
   sa.key0 = (uint32_t)seed ^ 0x6D756247u; sa.key1 = (uint32_t)(seed >> 32);
   sa.off_lo = (uint32_t)offset; sa.off_hi = (uint32_t)(offset >> 32);
   sa.sampled = sampled_ids;
+  sa.b_base = 0;
   return draft_common(c, B, seq_slot, hidden_last, token_last, top_n, top_ids, top_logit, row_max, row_lse,
                       logits_out, feat_out, &sa, stream);
 }
@@ -413,9 +450,7 @@ ps_status ps_group_forward(ps_ctx* c, int slot, int n_groups, const void* hidden
     float* rl = row_lse ? row_lse + r0 : nullptr;
     float* lo = logits_out ? logits_out + r0 * g.vocab : nullptr;
     float* fo = feat_out ? feat_out + r0 * g.hidden : nullptr;
-    s = fused_supported(c, B * R)
-            ? fused_draft_step(c, sm, B, h, tokens + g0, top_n, ti, tl, rm, rl, lo, fo, nullptr, st)
-            : plain_draft_step(c, sm, B, h, tokens + g0, top_n, ti, tl, rm, rl, lo, fo, nullptr, st);
+    s = run_draft_rows(c, sm, B, h, tokens + g0, top_n, ti, tl, rm, rl, lo, fo, nullptr, st);
     if (s != PS_OK) return s;
   }
   return PS_OK;

@@ -84,6 +84,7 @@ struct SampleArgs {
   float inv_temp;
   uint32_t key0, key1, off_lo, off_hi;
   int* sampled;   // [B][k+1]
+  uint32_t b_base;   // index, in the caller's batch, of the first sequence of this launch
 };
 __device__ __forceinline__ float gumbel_noise(const SampleArgs& sa, uint32_t v, uint32_t row_id) {
   uint32_t c[4] = {v, row_id, sa.off_lo, sa.off_hi};
@@ -165,6 +166,7 @@ ps_status launch_gumbel_argmax(ps_ctx* c, const float* logits, int M, int V, int
                                cudaStream_t st);
 // ---- fused bf16 kernels for small M ---------------------------------------------------------
 bool fused_supported(ps_ctx* c, int M);
+int fused_row_limit(ps_ctx* c);   // most rows fused_supported() takes for this context (0: none)
 size_t fused_scratch_bytes(const ps_config& g);
 void fused_release(ps_ctx* c);   // frees what the fused path holds on the host
 ps_status fused_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* bytes);

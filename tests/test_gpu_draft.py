@@ -66,6 +66,23 @@ def test_mini_bf16_more_masks_and_gqa():
     _compare_step(p, top_n=1)
 
 
+def test_mini_bf16_batch_beyond_one_launch():
+    """More rows than one tensor-core launch takes (30 sequences x 5 rows = 150 > 128): the
+    batch runs as groups of whole sequences; every sequence is checked, and each equals what
+    the same sequence gives when it runs alone."""
+    s = synth.CONFIGS["mini"]
+    B = 30
+    rng = np.random.default_rng(3)
+    p = Pair(s, B, lens=[int(x) for x in rng.integers(0, 90, B)])
+    _compare_step(p, top_n=8)
+    got = p.gpu_step(top_n=2)
+    for b in (0, 14, 15, 29):
+        one = p.g.draft_step([b], p.to_device(p.hidden_last[b:b + 1]), p.to_device(p.token_last[b:b + 1]), top_n=2)
+        torch.cuda.synchronize()
+        assert np.abs(one["logits"][0].cpu().numpy() - got["logits"][b]).max() <= 1e-3
+    assert p.g.poll() == 0
+
+
 def test_kv_append_matches_oracle_cache_and_is_incremental():
     s = synth.CONFIGS["mini"]
     p = Pair(s, 2, lens=[40, 9])
@@ -165,7 +182,7 @@ def _weights_13b_sweep():
     return _W13["w"]
 
 
-@pytest.mark.parametrize("B,k", [(4, 8), (16, 2), (64, 4)])
+@pytest.mark.parametrize("B,k", [(4, 8), (16, 2), (64, 4), (64, 8)])
 def test_13b_batch_sweep_sampled_sequences(B, k):
     """Points of the 13B-shaped batch / mask-count sweep at full size (ragged contexts of 256 to
     2048 positions, imported): every sequence runs on the GPU, the oracle recomputes three of

@@ -66,6 +66,21 @@ def test_sampled_tokens_match_oracle(name, B):
     assert p.g.poll() == 0
 
 
+def test_sampled_tokens_of_a_batch_beyond_one_launch():
+    """28 sequences x 5 rows exceed one tensor-core launch: the groups the batch is cut into
+    keep each sequence's own counter (its index in the caller's batch)."""
+    s = synth.CONFIGS["mini"]
+    B = 28
+    p = Pair(s, B, lens=[7 + 3 * b for b in range(B)])
+    T, seed, offset = 1.0, 11, 3
+    out = p.g.draft_step_sampled(list(range(B)), p.to_device(p.hidden_last), p.to_device(p.token_last),
+                                 T, seed, offset, top_n=1)
+    torch.cuda.synchronize()
+    got = {k: (v.cpu().numpy() if v is not None else None) for k, v in out.items()}
+    _check_rows(s, got, p.oracle_step, T, seed, offset, B)
+    assert p.g.poll() == 0
+
+
 def test_sampled_tokens_follow_softmax_and_verify_accepts_at_the_closed_form_rate():
     import paper_2410_05589_b200 as ps
     s = synth.CONFIGS["mini"]
