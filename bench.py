@@ -1,7 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the ParallelSpec hot path: ps_draft_step + ps_verify steps per second.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 13b|7b|33b|tiny]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 13b|7b|33b|13b_sweep|tiny]
+                    [--batch B] [--k-masks k]     # a point of the batch / mask-count sweep
     python bench.py --impl reference ...      # the CPU checker timed on the host cores
 
 One "step" = one parallel draft step (all k+1 rows, logits stored) followed by one verify
@@ -34,7 +35,10 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="13b", choices=["13b", "7b", "33b", "llama3_8b", "tiny", "mini"])
+    ap.add_argument("--workload", default="13b",
+                    choices=["13b", "7b", "33b", "llama3_8b", "13b_sweep", "tiny", "mini"])
+    ap.add_argument("--batch", type=int, default=0, help="sequences per step (default: the workload's)")
+    ap.add_argument("--k-masks", type=int, default=-1, help="[MASK] positions per sequence (default: the workload's)")
     ap.add_argument("--temperature", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
@@ -279,7 +283,7 @@ def run_reference(args):
     import oracle
     import synth
 
-    s = synth.CONFIGS[args.workload]
+    s = workload_shape(args)
     B = s.batch
     lens = synth.ctx_lengths(s, B)
     o = oracle_setup(s, B, lens)
@@ -315,6 +319,16 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def workload_shape(args):
+    import synth
+    s = synth.CONFIGS[args.workload]
+    if args.batch > 0:
+        s = s.with_(batch=args.batch)
+    if args.k_masks >= 0:
+        s = s.with_(k_masks=args.k_masks)
+    return s
+
+
 def workload_config(s, B, lens):
     return {
         "workload": f"{s.name}: H{s.hidden} heads{s.n_heads}x{s.head_dim} F{s.ffn} V{s.vocab} "
@@ -347,7 +361,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    s = synth.CONFIGS[args.workload]
+    s = workload_shape(args)
     B, R, V, T = s.batch, s.rows, s.vocab, args.temperature
     lens = synth.ctx_lengths(s, B)
     W = synth.weights(s)
@@ -462,7 +476,7 @@ def main():
         h1.record()
         torch.cuda.synchronize()
         group = {"ms_per_call": h0.elapsed_time(h1) / 5, "groups": n_g, "rows": n_g * R,
-                 "note": "ps_group_forward; more than 16 rows per launch run on the plain (untuned) kernels"}
+                 "note": "ps_group_forward; the groups run as draft steps of up to 128 rows per launch"}
 
     # ---- token-tree verification (Algorithm 1 in full), timed on its own ---------------------
     tree = None

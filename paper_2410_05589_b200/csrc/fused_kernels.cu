@@ -467,6 +467,7 @@ struct UArgs {
   int N, K, M;
   int Mp;                  // M padded to 16, 32, 64 or 128: rows of a plane box, half the MMA's N
   int n_tiles, KB;         // tiles of 128 weight rows (64 features when zipped), k-blocks of 64
+  int split;               // blocks a tile's k range is dealt in, 1..KB (see cta_begin)
   int zip;                 // 1: a tile is 64 rows of matrix 0 (gate) over 64 rows of matrix 1 (up)
   int lo;                  // 0: the activation operand is exact bf16 (no lo plane)
   int n_mats;              // concatenated matrices (q|k|v): tiles never straddle two of them
@@ -492,6 +493,23 @@ __device__ __forceinline__ int unit_owner(int u, int U, int G) {
 }
 __device__ __forceinline__ int unit_begin(int c, int U, int G) {
   return (int)((unsigned)U * (unsigned)c / (unsigned)G);
+}
+// Units are dealt in blocks: the KB k-blocks of a tile are cut into a.split contiguous blocks
+// (block j of a tile starts at its k-block j KB / split) and CTA c owns blocks
+// [S c / G, S (c+1) / G) of the S = n_tiles * split blocks.  split = KB deals single units
+// (every CTA streams the same bytes: the choice for few activation rows, where streaming is
+// all that counts); split = 1 deals whole tiles (no tile is shared, nothing to reduce: the
+// choice once a tile's epilogue and reduction cost more than an uneven load).
+__device__ __forceinline__ int block_first_unit(const UArgs& a, int x) {
+  const int t = x / a.split, j = x - t * a.split;
+  return t * a.KB + (j * a.KB) / a.split;
+}
+__device__ __forceinline__ int cta_begin(const UArgs& a, int c, int G) {
+  return block_first_unit(a, unit_begin(c, a.n_tiles * a.split, G));
+}
+__device__ __forceinline__ int cta_of_unit(const UArgs& a, int u, int G) {
+  const int t = u / a.KB, w = u - t * a.KB;
+  return unit_owner(t * a.split + ((w + 1) * a.split - 1) / a.KB, a.n_tiles * a.split, G);
 }
 
 // The tiles a CTA's unit range [u0, u1) touches, in the order the CTA works through them.  A
@@ -560,10 +578,12 @@ __device__ __forceinline__ int tile_feature(const UArgs& a, int t, int r, bool& 
 // Epilogue of one finished tile for the activation rows [m0, m0 + mc), mc <= 16; called by the
 // 128 epilogue threads after each has put its accumulator row r (= 32 * q + lane) of those
 // rows into ctl.acc[(m - m0) * 128 + r].  A dry call executes the same instructions and writes
-// nothing to global memory.  The loops
-// over m are rolled on purpose: this code runs once or twice per CTA, so what it costs is the
-// fetch of its instructions, not their execution.
-template <int EPI>
+// nothing to global memory.  With UNR = 1
+// the loops over m are rolled on purpose: for up to 16 rows this code runs once or twice per
+// CTA, so what it costs is the fetch of its instructions, not their execution.  With more rows
+// it runs once per 16 rows of every tile and its single warp per scheduler is bound by the
+// latency of dependent instructions: UNR = 4 interleaves four rows.
+template <int EPI, int UNR>
 __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane,
                                               int m0, int mc, bool dry) {
   using namespace umma;
@@ -607,12 +627,12 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
     }
   } else if (EPI == EPI_SWIGLU) {
     if (r >= 64) {
-#pragma unroll 1
+#pragma unroll UNR
       for (int m = 0; m < mc; ++m) ctl.xch[m * 64 + (r - 64)] = acc[m * 128] * ctl.scale[m0 + m];
     }
     epi_sync();
     if (r < 64 && valid && !dry) {
-#pragma unroll 1
+#pragma unroll UNR
       for (int m = 0; m < mc; ++m) {
         const float gv = acc[m * 128] * ctl.scale[m0 + m], uv = ctl.xch[m * 64 + r];
         const float act = gv / (1.f + __expf(-gv)) * uv;
@@ -622,7 +642,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
     }
     epi_sync();
   } else {  // EPI_LMHEAD: logits, and the tile's softmax / top-n summary per row
-#pragma unroll 1
+#pragma unroll UNR
     for (int m = 0; m < mc; ++m) {
       const float x = acc[m * 128] * ctl.scale[m0 + m];
       if (valid && a.logits_out && !dry) a.logits_out[(size_t)(m0 + m) * a.N + n] = x;
@@ -632,7 +652,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
       if (lane == 0) ctl.red[q][m] = mx;
     }
     epi_sync();
-#pragma unroll 1
+#pragma unroll UNR
     for (int m = 0; m < mc; ++m) {
       const float bmax = fmaxf(fmaxf(ctl.red[0][m], ctl.red[1][m]), fmaxf(ctl.red[2][m], ctl.red[3][m]));
       const float s = warp_sum(valid ? __expf(acc[m * 128] * ctl.scale[m0 + m] - bmax) : 0.f);
@@ -647,7 +667,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
     // top-n per row: repeated block arg-max over the values after the previous pick
 #pragma unroll 1
     for (int tn = 0; tn < a.top_n; ++tn) {
-#pragma unroll 1
+#pragma unroll UNR
       for (int m = 0; m < mc; ++m) {
         const float x = acc[m * 128] * ctl.scale[m0 + m];
         const float pv = tn ? ctl.prev_v[m] : FLT_MAX;
@@ -681,7 +701,7 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
       epi_sync();
     }
     if (a.sample) {   // Gumbel-max candidate of this vocabulary range per row
-#pragma unroll 1
+#pragma unroll UNR
       for (int m = 0; m < mc; ++m) {
         const int sb = (m0 + m) / a.R;
         const uint32_t row_id = ((uint32_t)sb + a.sa.b_base) | ((uint32_t)(m0 + m - sb * a.R) << 8);
@@ -751,7 +771,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   const uint32_t tmem = *(volatile uint32_t*)&ctl.tmem_base;
 
   const int G = gridDim.x, U = a.n_tiles * a.KB;
-  const int u0 = unit_begin(blockIdx.x, U, G), u1 = unit_begin(blockIdx.x + 1, U, G);
+  // (up to 16 rows single units are dealt: split = KB, and the block arithmetic drops out)
+  auto begin_of = [&](int c) { return MP <= 16 ? unit_begin(c, U, G) : cta_begin(a, c, G); };
+  auto owner_of = [&](int u) { return MP <= 16 ? unit_owner(u, U, G) : cta_of_unit(a, u, G); };
+  const int u0 = begin_of(blockIdx.x), u1 = begin_of(blockIdx.x + 1);
   const Segs segs(u0, u1, a.KB);
   volatile int* abort_flag = &ctl.abort_flag;
   constexpr int Mp = MP, sbytes = stage_bytes(Mp), nst = n_stages(Mp), ksplit = k_split(Mp), acols = acc_cols(Mp);
@@ -840,15 +863,26 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       const bool dry = seg < 0;
       if (seg == 0) {
         pdl_wait();   // everything below reads or writes what the kernel before this one touches
-        for (int m = warp - 2; m < a.M; m += 4) {   // RMSNorm row scales of the input
+        if (MP <= 16) {
+          for (int m = warp - 2; m < a.M; m += 4) {   // RMSNorm row scales of the input
+            float sc = 1.f;
+            if (a.ssq_in) {
+              float ss = 0.f;
+              for (int c = lane; c < a.ssq_n; c += 32) ss += a.ssq_in[(size_t)c * a.M + m];
+              ss = warp_sum(ss);
+              sc = rsqrtf(ss / (float)a.K + a.eps);
+            }
+            if (lane == 0) ctl.scale[m] = sc;
+          }
+        } else if (et < a.M) {   // many rows: one thread per row, its loads independent of each other
           float sc = 1.f;
           if (a.ssq_in) {
             float ss = 0.f;
-            for (int c = lane; c < a.ssq_n; c += 32) ss += a.ssq_in[(size_t)c * a.M + m];
-            ss = warp_sum(ss);
+#pragma unroll 8
+            for (int c = 0; c < a.ssq_n; ++c) ss += a.ssq_in[(size_t)c * a.M + et];
             sc = rsqrtf(ss / (float)a.K + a.eps);
           }
-          if (lane == 0) ctl.scale[m] = sc;
+          ctl.scale[et] = sc;
         }
         epi_sync();
       }
@@ -889,13 +923,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         fence_before_sync();
         mbar_arrive(&ctl.acc_empty[buf]);
         epi_sync();
-        c_first = unit_owner(t_begin, U, G);
-        c_last = unit_owner(t_end - 1, U, G);
+        c_first = owner_of(t_begin);
+        c_last = owner_of(t_end - 1);
         if (et == 0) {
           // one thread publishes the block's partial (the barrier above ordered the other
           // threads' stores before this release) and, if it came last, acquires the others'
           int n_contrib = 0;   // CTAs between the owners of the tile's ends that hold any unit
-          for (int c = c_first; c <= c_last; ++c) n_contrib += unit_begin(c, U, G) < unit_begin(c + 1, U, G);
+          for (int c = c_first; c <= c_last; ++c) n_contrib += begin_of(c) < begin_of(c + 1);
           unsigned old;
           asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(&a.tile_tickets[t]) : "memory");
           const int last = old == (unsigned)(n_contrib - 1);
@@ -908,9 +942,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       }
       if (finish && !whole) {   // where each contributor's partial lies (a CTA without units has none)
         for (int j = et; j <= c_last - c_first; j += kEpiThreads) {
-          const int c = c_first + j, cb = unit_begin(c, U, G);
+          const int c = c_first + j, cb = begin_of(c);
           int off = -1;
-          if (cb < unit_begin(c + 1, U, G)) {
+          if (cb < begin_of(c + 1)) {
             const int sl = (c == c_first && cb / a.KB != t) ? 1 : 0;
             off = (c * 2 + sl) * kMaxRows * 128;
           }
@@ -921,7 +955,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       if (finish) {
         // 16 activation rows at a time: the tile's sums into ctl.acc (from tensor memory, or the
         // partials added in CTA order, which does not depend on who came last), then the epilogue
-        for (int m0 = 0; m0 < a.M; m0 += 16) {
+        const int m_end = dry ? min(a.M, 16) : a.M;   // the rehearsal takes one chunk
+        for (int m0 = 0; m0 < m_end; m0 += 16) {
           const int mc = min(16, a.M - m0);
           if (whole) {
             float v[16];
@@ -964,7 +999,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
               }
             }
           }
-          tile_epilogue<EPI>(a, ctl, t, r, q, lane, m0, mc, dry);
+          tile_epilogue<EPI, (MP > 16 ? 4 : 1)>(a, ctl, t, r, q, lane, m0, mc, dry);
         }
       }
     }
@@ -1217,6 +1252,30 @@ UmmaMaps* build_maps(const ps_ctx* c, const FusedScratch& f) {
   return u;
 }
 
+// Blocks per tile (UArgs::split) for a launch of M rows on G CTAs.  Up to 16 rows single units
+// are dealt (split = KB).  Beyond, a tile shared between CTAs costs more the more rows there
+// are (its partial sums come back 16 rows x one contributor at a time), so a model of the
+// slowest CTA picks the split.  Its constants are measured on a B200 with 30 to 125 rows: 0.3 us
+// per unit, 7 us of epilogue per 16 rows of a finished tile, 2 us per contributor and 16 rows
+// of a shared tile plus 1 us per 16 rows to publish a partial.
+static int choose_split(int M, int Mp, int n_tiles, int KB, int G) {
+  if (Mp <= 16) return KB;
+  const double t_unit = 0.3, t_epi = 7.0, t_trip = 2.0, t_part = 1.0;   // microseconds
+  const int chunks = (M + 15) / 16, finished = (n_tiles + G - 1) / G;
+  int best = 1;
+  double best_cost = 1e30;
+  for (int s = 1; s <= KB; s = (s < 16 ? s + 1 : (s < KB ? KB : KB + 1))) {
+    const long long S = (long long)n_tiles * s;
+    const int blocks = (int)((S + G - 1) / G), units = blocks * ((KB + s - 1) / s);
+    // contributors of a shared tile: its blocks lie on ceil(s / blocks) CTAs, one more when unaligned
+    const int contrib = std::min(s, (s + blocks - 1) / blocks + 1);
+    const double cost = units * t_unit + finished * chunks * t_epi +
+                        (s > 1 ? chunks * (contrib * t_trip + t_part) : 0.0);
+    if (cost < best_cost) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
 template <int EPI>
 ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
                       const PlaneMaps& ph, const PlaneMaps& pl, UArgs& a, const FusedScratch& f,
@@ -1238,6 +1297,7 @@ ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, c
     }
   }
   if ((long long)a.n_tiles * a.KB * (c->n_sm + 1) >= (1ll << 31)) return fail(c, PS_ERR_UNSUPPORTED, "too many GEMM units");
+  a.split = choose_split(a.M, a.Mp, a.n_tiles, a.KB, c->n_sm);
   a.partials = f.partials; a.tile_tickets = f.tile_tickets; a.status = c->dev_status;
   auto kern = mi == 0 ? k_umma_gemm<EPI, 16> : mi == 1 ? k_umma_gemm<EPI, 32> : mi == 2 ? k_umma_gemm<EPI, 64>
                                                                                      : k_umma_gemm<EPI, 128>;
@@ -1322,7 +1382,18 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
     if ((s = launch_umma<EPI_STORE>(c, u.w_down, u.w_down, u.w_down, u.act_hi, u.act_lo, a, f, st))) return s;
   }
   prof_mark(c, st, "ffn_down");
-  {  // S6 logits = W_lm rms(hdn), softmax statistics and top-n without a second pass over logits
+  if (M > 32 && logits_out) {
+    // S6 with many rows and the logits kept: the row statistics in the tile epilogue cost more
+    // than the weights' streaming then (they are serial in the rows), so the GEMM only stores
+    // the logits and one block per row reads them back from L2
+    UArgs a{};
+    a.N = V; a.K = H; a.M = M; a.n_mats = 1; a.mat_rows[0] = V; a.lo = 1;
+    a.ssq_in = f.ssq[2]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
+    a.out = logits_out; a.ldo = V;
+    if ((s = launch_umma<EPI_STORE>(c, u.w_lm, u.w_lm, u.w_lm, u.hdn_hi, u.hdn_lo, a, f, st))) return s;
+    if ((s = launch_row_stats(c, logits_out, M, V, top_n, top_ids, top_logit, row_max, row_lse, st))) return s;
+    if (sa && (s = launch_gumbel_argmax(c, logits_out, M, V, R, *sa, st))) return s;
+  } else {  // S6 logits = W_lm rms(hdn), softmax statistics and top-n without a second pass over logits
     UArgs a{};
     a.N = V; a.K = H; a.M = M; a.n_mats = 1; a.mat_rows[0] = V; a.lo = 1;
     a.ssq_in = f.ssq[2]; a.ssq_n = tiles_h; a.eps = g.rms_eps;

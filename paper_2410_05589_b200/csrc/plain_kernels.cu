@@ -455,10 +455,7 @@ ps_status draft_impl(ps_ctx* c, const SeqMap& sm, int B, const void* hidden_last
   c->launches++;
   float* logits = logits_out ? logits_out : c->logits;
   if ((s = linear<WT>(c, c->hn, H, w.w_lm, nullptr, nullptr, 0, logits, V, M, V, H, st))) return s;
-  if (top_n > 0 || row_max || row_lse) {
-    k_row_stats<<<M, 256, 0, st>>>(logits, V, top_n, top_ids, top_logit, row_max, row_lse);
-    c->launches++;
-  }
+  if ((s = launch_row_stats(c, logits, M, V, top_n, top_ids, top_logit, row_max, row_lse, st))) return s;
   if (sa && (s = launch_gumbel_argmax(c, logits, M, V, g.k_masks + 1, *sa, st))) return s;
   prof_mark(c, st, "lm_head");
   return cuda_check(c, cudaGetLastError(), "draft_step");
@@ -482,6 +479,14 @@ ps_status plain_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
                                  row_max, row_lse, logits_out, feat_out, sa, st)
              : draft_impl<__nv_bfloat16>(c, sm, B, hidden_last, token_last, top_n, top_ids,
                                          top_logit, row_max, row_lse, logits_out, feat_out, sa, st);
+}
+
+ps_status launch_row_stats(ps_ctx* c, const float* logits, int M, int V, int top_n, int* top_ids,
+                           float* top_logit, float* row_max, float* row_lse, cudaStream_t st) {
+  if (top_n <= 0 && !row_max && !row_lse) return PS_OK;
+  k_row_stats<<<M, 256, 0, st>>>(logits, V, top_n, top_ids, top_logit, row_max, row_lse);
+  c->launches++;
+  return cuda_check(c, cudaGetLastError(), "k_row_stats");
 }
 
 ps_status launch_gumbel_argmax(ps_ctx* c, const float* logits, int M, int V, int R, const SampleArgs& sa,

@@ -161,6 +161,9 @@ ps_status plain_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
                            const int* token_last, int top_n, int* top_ids, float* top_logit,
                            float* row_max, float* row_lse, float* logits_out, float* feat_out,
                            const SampleArgs* sa, cudaStream_t st);
+// One block per row of stored logits [M][V]: max, log-sum-exp and top-n of the row.
+ps_status launch_row_stats(ps_ctx* c, const float* logits, int M, int V, int top_n, int* top_ids,
+                           float* top_logit, float* row_max, float* row_lse, cudaStream_t st);
 // One block per row of stored logits [M][V]: the Gumbel-max token of the row (R rows per sequence).
 ps_status launch_gumbel_argmax(ps_ctx* c, const float* logits, int M, int V, int R, const SampleArgs& sa,
                                cudaStream_t st);

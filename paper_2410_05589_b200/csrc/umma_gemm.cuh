@@ -1,5 +1,8 @@
 // Weight-streaming small-M GEMM on the 5th-generation tensor cores:
-//   Y[m][n] = sum_k A[m][k] * W[n][k],  M = B*(k+1) <= 16 rows, W row-major bf16, fp32 sums.
+//   Y[m][n] = sum_k A[m][k] * W[n][k],  M = B*(k+1) <= 128 rows, W row-major bf16, fp32 sums.
+// (The description below is for up to 16 rows; with Mp = 32, 64 or 128 padded rows the planes
+// form an N = 2 Mp operand, stages grow and get fewer, and fewer accumulators fit: see
+// stage_bytes(), n_stages(), k_split() below.)
 //
 // The weights are the M side of tcgen05.mma (128 weight rows per instruction), the activation
 // rows its N side: the 16 rows of the hi plane and the 16 rows of the lo plane sit one after the
@@ -14,7 +17,8 @@
 //
 // Work is cut into units of (128-row tile, 64-column k-block); CTA c of a one-CTA-per-SM grid
 // takes the contiguous unit range [U c / G, U (c+1) / G) in tile-major order, so the load is
-// balanced to one 16 KB unit whatever N and K are.  A tile whose k range is shared by several
+// balanced to one 16 KB unit whatever N and K are (with more than 16 rows the units are dealt
+// in larger blocks, down to whole tiles: UArgs::split).  A tile whose k range is shared by several
 // CTAs is reduced through fp32 partials in global memory: every contributor writes its partial
 // and takes a ticket, the last one adds the partials in CTA order (the sum does not depend on
 // who was last) and runs the tile's epilogue.  No CTA waits for another.
