@@ -60,16 +60,24 @@ KERNEL_OF_STAGE = {
     "attention": "k_attn_mma", "o_proj": "k_umma_gemm<STORE>", "ffn_gate_up": "k_umma_gemm<SWIGLU>",
     "ffn_down": "k_umma_gemm<STORE>", "lm_head": "k_umma_gemm<LMHEAD>", "verify": "k_verify_cluster",
 }
+
+
+def kernel_of_stage(stage, rows):
+    if stage == "lm_head" and rows > 32:   # logits stored by the GEMM, statistics by one block per row
+        return "k_umma_gemm<STORE> + k_row_stats"
+    return KERNEL_OF_STAGE.get(stage, stage)
+
+
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
 # profiles/k_umma_gemm_13b_b1_k4.md, keyed by (workload, batch, k_masks, stage).  Valid for the
 # kernels as captured; set an entry to None when its kernel changes.
 NCU_DRAM_BYTES = {
-    ("13b", 1, 4, "fc_norm"): 105872384 + 4049152,
-    ("13b", 1, 4, "qkv_rope"): 157781248 + 3869440,
-    ("13b", 1, 4, "o_proj"): 52934144 + 5120,
-    ("13b", 1, 4, "ffn_gate_up"): 284786176 + 4916736,
-    ("13b", 1, 4, "ffn_down"): 143446272 + 4156416,
-    ("13b", 1, 4, "lm_head"): 329086208 + 4603136,
+    ("13b", 1, 4, "fc_norm"): 106259200 + 4141824,
+    ("13b", 1, 4, "qkv_rope"): 158127872 + 3880704,
+    ("13b", 1, 4, "o_proj"): 53316352 + 8960,
+    ("13b", 1, 4, "ffn_gate_up"): 285139968 + 4767232,
+    ("13b", 1, 4, "ffn_down"): 143910144 + 4637184,
+    ("13b", 1, 4, "lm_head"): 329474816 + 5147648,
 }
 
 
@@ -431,7 +439,7 @@ def main():
     roofline = None
     if dom:
         roofline = {
-            "bound": "hbm", "kernel": KERNEL_OF_STAGE.get(dom, dom), "stage": dom,
+            "bound": "hbm", "kernel": kernel_of_stage(dom, B * R), "stage": dom,
             "achieved": stages[dom]["gbs"], "peak": peak,
             "unit": "GB/s", "frac": round(stages[dom]["gbs"] / peak, 4),
             "traffic": NCU_DRAM_BYTES.get((args.workload, B, s.k_masks, dom)),
@@ -504,6 +512,32 @@ def main():
            "h2d_bytes_per_step": B * s.hidden * eb + B * 4 + B * R * V * 4,
            "d2h_bytes_per_step": B * (R + 3) * 4, "steps": n_e2e}
 
+    # ---- ps_kv_append (once per round, off the draft step's path): 4 accepted pairs a sequence ----
+    n_new = 4
+    ka_h = ps.to_device(synth.hidden_states(s, "app", B * n_new))
+    ka_t = ps.to_device(synth.token_ids(s, "app", B * n_new))
+    app_slots = slots[0]   # last leg on the device: these slots' contexts are not needed again
+
+    def append_once():
+        for x in app_slots:   # host bookkeeping only: the same cache rows are written every time
+            g.kv_reset(x)
+        g.kv_append(app_slots, [n_new] * B, ka_h, ka_t)
+
+    for i in range(3):
+        append_once()
+    torch.cuda.synchronize()
+    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    k0.record()
+    for i in range(50):
+        append_once()
+    k1.record()
+    torch.cuda.synchronize()
+    app_us = k0.elapsed_time(k1) / 50 * 1e3
+    app_bytes = eb * (2 * s.hidden * s.hidden + 2 * s.n_kv_heads * s.head_dim * s.hidden)
+    kv_append = {"us": round(app_us, 2), "rows": B * n_new, "bytes": app_bytes,
+                 "gbs": round(app_bytes / (app_us * 1e-6) / 1e9, 1),
+                 "note": "fc + k|v weights read once, 4 new real positions per sequence"}
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(s, B, lens, hl_np, tl_np, tgt_np[0], T, args.cpu_seconds)
@@ -527,7 +561,7 @@ def main():
             "hbm_frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
             "mean_tokens_per_round": n_accept,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "stages": stages, "sampled_drafts": sampled, "group_forward": group, "tree_verify": tree, "cpu_baseline": cpu,
+            "roofline": roofline, "stages": stages, "sampled_drafts": sampled, "group_forward": group, "tree_verify": tree, "kv_append": kv_append, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
     if world > 1:

@@ -119,7 +119,10 @@ ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* weights,
  *   row_offset   host [B+1], row_offset[0] = 0, row_offset[i+1] = row_offset[i] + n_new[i]
  *   hidden       device [total][H], config dtype
  *   tokens       device [total] int32 in [0, V)
- * PS_ERR_CAPACITY if len + n_new > max_ctx for a sequence (nothing is appended). */
+ * PS_ERR_CAPACITY if len + n_new > max_ctx for a sequence (nothing is appended).
+ * The same rows in the same calls give the same cache bits; grouping the rows into calls
+ * differently may flip the last bit of single bf16 cache entries (the GEMM's summation order
+ * depends on the number of rows of a launch). */
 ps_status ps_kv_append(ps_ctx* ctx, int B, const int* seq_slot, const int* n_new,
                        const int* row_offset, const void* hidden, const int* tokens, void* stream);
 

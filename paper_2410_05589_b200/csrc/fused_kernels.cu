@@ -1308,6 +1308,46 @@ ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, c
   return cuda_check(c, e, "k_umma_gemm");
 }
 
+// ps_kv_append on the tensor-core GEMM: rows [sm.row_base, sm.row_base + rows) of the call's real
+// (token, feature) pairs: gather, fc (+ the planes of its normalised output), k | v projection,
+// then RoPE and the store into the cache rows (the kernel the plain path uses).
+ps_status umma_kv_append(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int rows, const void* hidden,
+                         const int* tokens, cudaStream_t st) {
+  const ps_config& g = c->cfg;
+  const ps_weights& w = c->w;
+  const int H = g.hidden, Hkv = g.n_kv_heads * g.head_dim, V = g.vocab;
+  typedef const __nv_bfloat16* BP;
+  const FusedScratch f = carve_fused(g, (char*)c->fused_scratch);
+  const int tiles_h = (H + umma::kTile - 1) / umma::kTile;
+  ps_status s;
+  prof_mark(c, st, "begin");
+  // every row is a real position: with one row per "sequence" the gather takes row m's own pair
+  cudaError_t ge = launch_after(k_gather_x, dim3(rows), dim3(256), 0, st, !c->prof, (BP)w.embed, (BP)w.mask_embed,
+                                (BP)w.mask_feat, (BP)hidden + (size_t)sm.row_base * H, tokens + sm.row_base, H, V, 1,
+                                f.xin);
+  c->launches++;
+  if (ge != cudaSuccess) return cuda_check(c, ge, "k_gather_x");
+  {
+    UArgs a{};
+    a.N = H; a.K = 2 * H; a.M = rows; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 0;
+    a.out = c->x0; a.ldo = H; a.bias = (g.flags & PS_FLAG_FC_BIAS) ? (BP)w.b_fc : nullptr;
+    a.ssq_out = f.ssq[0];
+    a.out_hi = f.x0p.hi; a.out_lo = f.x0p.lo; a.ld_plane = H; a.gain_next = (BP)w.g_in;
+    if ((s = launch_umma<EPI_STORE>(c, u.w_fc, u.w_fc, u.w_fc, u.xin, u.xin, a, f, st))) return s;
+  }
+  prof_mark(c, st, "fc_norm");
+  {
+    UArgs a{};
+    a.N = 2 * Hkv; a.K = H; a.M = rows; a.n_mats = 2; a.mat_rows[0] = Hkv; a.mat_rows[1] = Hkv; a.lo = 1;
+    a.ssq_in = f.ssq[0]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
+    a.out = c->kv_tmp; a.ldo = 2 * Hkv;
+    if ((s = launch_umma<EPI_STORE>(c, u.w_k, u.w_v, u.w_v, u.x0_hi, u.x0_lo, a, f, st))) return s;
+  }
+  if ((s = launch_rope_store_kv(c, sm, rows, st))) return s;
+  prof_mark(c, st, "qkv_rope");
+  return PS_OK;
+}
+
 ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B, const void* hidden_last,
                           const int* token_last, int top_n, int* top_ids, float* top_logit, float* row_max,
                           float* row_lse, float* logits_out, float* feat_out, const SampleArgs* sa,
@@ -1445,6 +1485,17 @@ bool fused_supported(ps_ctx* c, int M) {
 int fused_row_limit(ps_ctx* c) {
   if (fused_supported(c, umma::kMaxRows)) return umma::kMaxRows;
   return fused_supported(c, kMaxM) ? kMaxM : 0;
+}
+
+// Rows per pass ps_kv_append may hand to fused_kv_append (0: the plain kernels serve).
+int fused_kv_rows(ps_ctx* c) {
+  if (c->cfg.flags & PS_FLAG_NO_FC) return 0;
+  return fused_supported(c, umma::kMaxRows) && c->umma_maps ? umma::kMaxRows : 0;
+}
+
+ps_status fused_kv_append(ps_ctx* c, const SeqMap& sm, int rows, const void* hidden, const int* tokens,
+                          cudaStream_t st) {
+  return umma_kv_append(c, *static_cast<const UmmaMaps*>(c->umma_maps), sm, rows, hidden, tokens, st);
 }
 
 size_t fused_scratch_bytes(const ps_config& g) { return carve_fused(g, nullptr).bytes; }

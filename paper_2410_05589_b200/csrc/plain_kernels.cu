@@ -280,6 +280,7 @@ __global__ void __launch_bounds__(256) k_row_stats(const float* logits, int V, i
   __shared__ int s_i[8];
   __shared__ float s_f[8];
   const float* row = logits + (size_t)blockIdx.x * V;
+  const int nv4 = (reinterpret_cast<uintptr_t>(row) & 15) == 0 ? V / 4 : 0;   // float4 part of the row
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   float prev_v = FLT_MAX;
   int prev_i = -1;
@@ -288,11 +289,16 @@ __global__ void __launch_bounds__(256) k_row_stats(const float* logits, int V, i
   for (int t = 0; t < passes; ++t) {
     float bv = -FLT_MAX;
     int bi = 0x7fffffff;
-    for (int v = threadIdx.x; v < V; v += blockDim.x) {
-      float x = row[v];
-      bool after = (x < prev_v) || (x == prev_v && v > prev_i);   // ranks after the last pick
+    auto consider = [&](float x, int v) {
+      const bool after = (x < prev_v) || (x == prev_v && v > prev_i);   // ranks after the last pick
       if (after && (x > bv || (x == bv && v < bi))) { bv = x; bi = v; }
+    };
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nv4; i += blockDim.x) {   // 16-byte loads, several in flight
+      const float4 x = __ldg(reinterpret_cast<const float4*>(row) + i);
+      consider(x.x, 4 * i); consider(x.y, 4 * i + 1); consider(x.z, 4 * i + 2); consider(x.w, 4 * i + 3);
     }
+    for (int v = 4 * nv4 + threadIdx.x; v < V; v += blockDim.x) consider(row[v], v);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       float ov = __shfl_xor_sync(0xffffffffu, bv, o);
@@ -313,7 +319,12 @@ __global__ void __launch_bounds__(256) k_row_stats(const float* logits, int V, i
     prev_v = bv; prev_i = bi;
   }
   float s = 0.f;
-  for (int v = threadIdx.x; v < V; v += blockDim.x) s += expf(row[v] - rmax);
+#pragma unroll 4
+  for (int i = threadIdx.x; i < nv4; i += blockDim.x) {
+    const float4 x = __ldg(reinterpret_cast<const float4*>(row) + i);
+    s += (expf(x.x - rmax) + expf(x.y - rmax)) + (expf(x.z - rmax) + expf(x.w - rmax));
+  }
+  for (int v = 4 * nv4 + threadIdx.x; v < V; v += blockDim.x) s += expf(row[v] - rmax);
   s = warp_sum(s);
   if (lane == 0) s_f[warp] = s;
   __syncthreads();
@@ -479,6 +490,20 @@ ps_status plain_draft_step(ps_ctx* c, const SeqMap& sm, int B, const void* hidde
                                  row_max, row_lse, logits_out, feat_out, sa, st)
              : draft_impl<__nv_bfloat16>(c, sm, B, hidden_last, token_last, top_n, top_ids,
                                          top_logit, row_max, row_lse, logits_out, feat_out, sa, st);
+}
+
+ps_status launch_rope_store_kv(ps_ctx* c, const SeqMap& sm, int rows, cudaStream_t st) {
+  const ps_config& g = c->cfg;
+  if (g.dtype == PS_DTYPE_F32)
+    k_rope_store<float><<<rows, 128, g.head_dim * sizeof(float), st>>>(
+        sm, nullptr, c->kv_tmp, (float*)c->kcache, (float*)c->vcache, nullptr, g.n_heads, g.n_kv_heads,
+        g.head_dim, g.max_ctx, g.rope_base);
+  else
+    k_rope_store<__nv_bfloat16><<<rows, 128, g.head_dim * sizeof(float), st>>>(
+        sm, nullptr, c->kv_tmp, (__nv_bfloat16*)c->kcache, (__nv_bfloat16*)c->vcache, nullptr, g.n_heads,
+        g.n_kv_heads, g.head_dim, g.max_ctx, g.rope_base);
+  c->launches++;
+  return cuda_check(c, cudaGetLastError(), "k_rope_store");
 }
 
 ps_status launch_row_stats(ps_ctx* c, const float* logits, int M, int V, int top_n, int* top_ids,

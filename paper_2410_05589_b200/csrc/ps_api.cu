@@ -281,6 +281,22 @@ ps_status ps_poll(ps_ctx* c, void* stream) {
   return PS_OK;
 }
 
+// k / v of `total` real rows (sm.row_off lays them out over the sequences) into the cache, in
+// passes of as many rows as the kernels take: the tensor-core GEMM where it serves, else the
+// plain kernels.
+static ps_status append_rows(ps_ctx* c, SeqMap& sm, int total, const void* hidden, const int* tokens,
+                             cudaStream_t st) {
+  const int fused_rows = fused_kv_rows(c), chunk = fused_rows > 0 ? fused_rows : kAppendChunk;
+  for (int r0 = 0; r0 < total; r0 += chunk) {
+    sm.row_base = r0;
+    const int rows = std::min(chunk, total - r0);
+    const ps_status s = fused_rows > 0 ? fused_kv_append(c, sm, rows, hidden, tokens, st)
+                                       : plain_kv_append(c, sm, rows, hidden, tokens, st);
+    if (s != PS_OK) return s;
+  }
+  return PS_OK;
+}
+
 ps_status ps_kv_append(ps_ctx* c, int B, const int* seq_slot, const int* n_new,
                        const int* row_offset, const void* hidden, const int* tokens, void* stream) {
   if (!c) return PS_ERR_INVALID_ARG;
@@ -307,12 +323,7 @@ ps_status ps_kv_append(ps_ctx* c, int B, const int* seq_slot, const int* n_new,
     sm.row_off[b] = row_offset[b];
   }
   sm.row_off[B] = total;
-  for (int r0 = 0; r0 < total; r0 += kAppendChunk) {
-    sm.row_base = r0;
-    int rows = std::min(kAppendChunk, total - r0);
-    s = plain_kv_append(c, sm, rows, hidden, tokens, (cudaStream_t)stream);
-    if (s != PS_OK) return s;
-  }
+  if ((s = append_rows(c, sm, total, hidden, tokens, (cudaStream_t)stream)) != PS_OK) return s;
   for (int b = 0; b < B; ++b) c->len[seq_slot[b]] += n_new[b];
   return PS_OK;
 }
@@ -429,10 +440,7 @@ ps_status ps_group_forward(ps_ctx* c, int slot, int n_groups, const void* hidden
   SeqMap sm;
   std::memset(&sm, 0, sizeof(sm));
   sm.B = 1; sm.slot[0] = slot; sm.len[0] = L0; sm.row_off[0] = 0; sm.row_off[1] = n_groups;
-  for (int r0 = 0; r0 < n_groups; r0 += kAppendChunk) {
-    sm.row_base = r0;
-    if ((s = plain_kv_append(c, sm, std::min(kAppendChunk, n_groups - r0), hidden, tokens, st)) != PS_OK) return s;
-  }
+  if ((s = append_rows(c, sm, n_groups, hidden, tokens, st)) != PS_OK) return s;
   // 2. the groups as a batch of draft steps on the same slot: group t sees cache rows
   //    [0, L0 + t), i.e. the prefix and the real rows before it, and its own k + 1 new rows
   const int chunk = std::min(g.max_batch, (int)PS_MAX_BATCH);

@@ -169,6 +169,11 @@ ps_status launch_gumbel_argmax(ps_ctx* c, const float* logits, int M, int V, int
                                cudaStream_t st);
 // ---- fused bf16 kernels for small M ---------------------------------------------------------
 bool fused_supported(ps_ctx* c, int M);
+int fused_kv_rows(ps_ctx* c);     // rows per pass of fused_kv_append (0: not available)
+ps_status fused_kv_append(ps_ctx* c, const SeqMap& sm, int rows, const void* hidden, const int* tokens,
+                          cudaStream_t st);
+// RoPE on the k half of kv_tmp rows [0, rows) and the store of k and v into the cache rows.
+ps_status launch_rope_store_kv(ps_ctx* c, const SeqMap& sm, int rows, cudaStream_t st);
 int fused_row_limit(ps_ctx* c);   // most rows fused_supported() takes for this context (0: none)
 size_t fused_scratch_bytes(const ps_config& g);
 void fused_release(ps_ctx* c);   // frees what the fused path holds on the host
