@@ -344,7 +344,9 @@ static ps_status run_draft_rows(ps_ctx* c, const SeqMap& sm, int B, const void* 
   if (per_max < 1)
     return plain_draft_step(c, sm, B, hidden, tokens, top_n, top_ids, top_logit, row_max, row_lse,
                             logits_out, feat_out, sa, st);
-  const int n_chunks = (B + per_max - 1) / per_max, per = (B + n_chunks - 1) / n_chunks;
+  // full groups first: a launch costs by its padded row count (16, 32, 64 or 128), so the
+  // remainder is better off alone in a small launch than evened out over large ones
+  const int per = per_max;
   const size_t eb = g.dtype == PS_DTYPE_F32 ? 4 : 2;
   for (int b0 = 0; b0 < B; b0 += per) {
     const int nb = std::min(per, B - b0);

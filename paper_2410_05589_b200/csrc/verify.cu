@@ -337,7 +337,7 @@ struct CluScratch {
   double d[kCluWarps], d2[kCluWarps];
 };
 
-// (NCLU blocks per cluster: 8, or 16 for vocabularies beyond 65536.)
+// (NCLU blocks per cluster: 8; 16 for vocabularies beyond 65536; 4 for batches of several waves.)
 template <int NCLU>
 __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
   namespace cg = cooperative_groups;
@@ -576,6 +576,13 @@ __global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads) k_ve
 }
 __global__ void __launch_bounds__(kCluThreads) k_verify_cluster16(VerifyArgs a) {
   verify_cluster_body<16>(a);
+}
+// Four blocks per row pair: for batches whose 8-block clusters would not be resident at once
+// (one block fills an SM), while a thread can still hold its share of a row (16 tokens).
+constexpr int kCluSmall = 4;
+constexpr int kCluSmallMaxVocab = kCluSmall * kCluThreads * 4 * kCluV4;
+__global__ void __cluster_dims__(kCluSmall, 1, 1) __launch_bounds__(kCluThreads) k_verify_cluster4(VerifyArgs a) {
+  verify_cluster_body<kCluSmall>(a);
 }
 
 // ---- token-tree verification (Algorithm 1 in full) -------------------------------------------
@@ -956,7 +963,10 @@ ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* 
     prof_mark(c, st, "begin");
     // (a plain launch: joining the dependent-launch chain here was measured to cost 7 us a step)
     cudaError_t e;
-    if (nclu == kClu) {
+    if (nclu == kClu && a.V <= kCluSmallMaxVocab && n_target * B * kClu > c->n_sm) {
+      k_verify_cluster4<<<dim3(n_target * kCluSmall, B), kCluThreads, 0, st>>>(a);   // half the waves
+      e = cudaGetLastError();
+    } else if (nclu == kClu) {
       k_verify_cluster<<<dim3(n_target * kClu, B), kCluThreads, 0, st>>>(a);
       e = cudaGetLastError();
     } else {

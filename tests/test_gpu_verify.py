@@ -78,7 +78,8 @@ def test_device_philox_equals_oracle_words():
 @pytest.mark.parametrize("T", [1.0, 0.6])
 def test_stochastic_verify_matches_oracle(V, n_draft, bonus, T):
     # vocabularies that are a multiple of 4 take the cluster kernel (8 blocks per row up to 65536,
-    # 16 up to 131072), the rest the one-block-per-row kernel
+    # 16 up to 131072; 4 blocks up to 32768 when the batch's 8-block clusters exceed the SMs, as
+    # these batches do), the rest the one-block-per-row kernel
     B = 96 if V < 20000 else 24
     g = _ctx(V)
     tl = synth.gauss_logits(1, ("t", V), (B, n_draft + bonus, V))
