@@ -432,8 +432,10 @@ def main():
     stages = {}
     for name, (tot, cnt) in prof.items():
         if cnt and name in sb:
-            us = tot / cnt * 1e3
-            stages[name] = {"us": round(us, 2), "gbs": round(sb[name] / (us * 1e-6) / 1e9, 1)}
+            # per step, not per launch: a batch beyond 128 rows runs a stage several times a step
+            us = tot / n_prof * 1e3
+            stages[name] = {"us": round(us, 2), "gbs": round(sb[name] / (us * 1e-6) / 1e9, 1),
+                            "launches_per_step": round(cnt / n_prof, 2)}
     dom = max(stages, key=lambda k: stages[k]["us"]) if stages else None
     step_bytes = sum(sb.values())
     roofline = None

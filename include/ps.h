@@ -130,8 +130,11 @@ ps_status ps_kv_append(ps_ctx* ctx, int B, const int* seq_slot, const int* n_new
  * For each sequence: row 0 is the last real position (token_last, hidden_last), rows 1..k are
  * [MASK]_1..[MASK]_k; row j sits at position len+j, attends to the cached real positions and
  * to rows 0..j, and its logits are the drafter's distribution for the token j places after
- * the next one.  The committed cache length does not change; rows [len, len+k] of the slab
- * are overwritten as scratch.  Calling it twice gives identical outputs.
+ * the next one.  Neither the committed cache length nor the cache rows change (the new rows'
+ * k / v live in a side buffer of the workspace).  Calling it twice gives identical outputs.
+ * A batch of more than 128 rows B*(k+1) runs as several launches per stage, each over a group
+ * of whole sequences; a sequence's outputs do not depend on which other sequences are in the
+ * call beyond fp32 rounding (the GEMMs' summation order follows the rows of a launch).
  *   B            sequences (1..max_batch);  seq_slot host [B], distinct
  *   hidden_last  device [B][H], config dtype;  token_last device [B] int32
  *   top_n        0..PS_MAX_TOP_N entries per row (0: top_ids/top_logit unused)
