@@ -49,7 +49,7 @@ enum {
   PS_FLAG_FC_BIAS = 1,          /* ps_weights.b_fc is used */
   PS_FLAG_UNFUSED_KERNELS = 2,  /* force the unfused fp32-activation kernels (debugging aid) */
   PS_FLAG_MMA_SYNC_GEMM = 4,    /* fused path: mma.sync GEMM kernels instead of the tcgen05 ones */
-  PS_FLAG_NO_FC = 8             /* embedding-only input (the Medusa integration, Sec. 4.2): x0 is the token /
+  PS_FLAG_NO_FC = 8             /* embedding-only input (the Medusa integration, Sec. 4.3): x0 is the token /
                                    [MASK] embedding, there is no fc layer and no target feature; w_fc,
                                    mask_feat and every `hidden` argument are ignored and may be NULL */
 };
@@ -236,11 +236,15 @@ ps_status ps_verify_tree(ps_ctx* ctx, int B, int n_nodes, const int* parent, con
                          int* n_out, int* path, void* stream);
 
 /* Host-buffer convenience for one draft+verify round: copies hidden_last / token_last /
- * target_logits from host memory, runs ps_draft_step (arg-max drafts of all k+1 rows) and
- * ps_verify (n_draft = n_target = k+1) on `stream`, copies accept_len / out_tokens / n_out
- * back and waits for the stream.  All pointers except ctx are host memory; pinned memory
- * makes the copies asynchronous.  The target logits travel on a stream of the context's own
- * (created by the first call) while the draft step runs.
+ * target_logits from host memory, runs the draft step for all k+1 rows and ps_verify
+ * (n_draft = n_target = k+1) on `stream`, copies accept_len / out_tokens / n_out back and waits
+ * for the stream.  At temperature 0 the drafts are the rows' arg-max tokens and verify is greedy;
+ * at temperature > 0 they are drawn from softmax(draft logits / temperature) by
+ * ps_draft_step_sampled with the same seed and offset, and verify gets those draft logits as q:
+ * the round then emits tokens that follow the target distribution (Eq. 1 holds for drafts drawn
+ * from q, not for arg-max drafts with a full q).  All pointers except ctx are host memory; pinned
+ * memory makes the copies asynchronous.  The target logits travel on a stream of the context's
+ * own (created by the first call) while the draft step runs.
  *   hidden_last [B][H] config dtype, token_last [B], target_logits [B][k+1][V] float,
  *   accept_len [B], out_tokens [B][k+2], n_out [B]. */
 ps_status ps_round_host(ps_ctx* ctx, int B, const int* seq_slot, const void* hidden_last,

@@ -51,7 +51,7 @@ struct Config {
   int max_batch, max_ctx;
   double rope_base, rms_eps;
   int has_fc_bias;
-  int no_fc;  // embedding-only input (the Medusa integration of Sec. 4.2): x0 = the embedding half
+  int no_fc;  // embedding-only input (the Medusa integration of Sec. 4.3): x0 = the embedding half
 };
 
 struct Weights {
@@ -230,7 +230,10 @@ int argmax_row(const float* row, int V) {
 // Inverse-CDF draw from unnormalised non-negative weights w[0..V): the first v whose
 // running sum exceeds u*W; if rounding leaves none, the last v with positive weight.
 // *margin receives the distance of u*W to the nearest running-sum boundary, over W.
-int inverse_cdf(const std::vector<double>& w, double W, double u, double* margin) {
+// nb (optional) receives the positive-weight tokens next to the pick in the running sum:
+// nb[0] the one before it, nb[1] the one after it (-1 if there is none) -- the only other
+// tokens a draw whose sampling point sits on a boundary may land on.
+int inverse_cdf(const std::vector<double>& w, double W, double u, double* margin, int* nb = nullptr) {
   double target = u * W, run = 0.0, best = std::numeric_limits<double>::infinity();
   int pick = -1, last_pos = -1;
   for (size_t v = 0; v < w.size(); ++v) {
@@ -244,6 +247,11 @@ int inverse_cdf(const std::vector<double>& w, double W, double u, double* margin
   }
   if (pick < 0) pick = last_pos;
   if (margin) *margin = (W > 0.0) ? best / W : 0.0;
+  if (nb) {
+    nb[0] = nb[1] = -1;
+    for (int v = pick - 1; v >= 0 && nb[0] < 0; --v) if (w[v] > 0.0) nb[0] = v;
+    for (size_t v = (size_t)(pick + 1); pick >= 0 && v < w.size() && nb[1] < 0; ++v) if (w[v] > 0.0) nb[1] = (int)v;
+  }
   return pick;
 }
 
@@ -560,11 +568,12 @@ void pso_uniforms(uint64_t seed, uint64_t offset, int b, int i, double* r, doubl
 //   margin_accept[B][n_draft] = |r - min(1,p/q)| at each examined position (inf if not
 //   examined or T=0); margin_cdf[B] = distance of the sampling point to the nearest CDF
 //   boundary, as a fraction of the total weight (inf if nothing was sampled);
-//   nonfinite[B] = 1 if a NaN/+inf logit was met.
+//   nonfinite[B] = 1 if a NaN/+inf logit was met; neighbours[B][2] (optional) = the
+//   positive-weight tokens before / after the sampled one in the running sum (-1: none).
 int pso_verify(int B, int n_draft, int n_target, int V, const int* draft_tokens,
                const float* draft_logits, const float* target_logits, double temperature,
                uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
-               double* margin_accept, double* margin_cdf, int* nonfinite) {
+               double* margin_accept, double* margin_cdf, int* nonfinite, int* neighbours) {
   if (n_target != n_draft && n_target != n_draft + 1) return -1;
   const double INF = std::numeric_limits<double>::infinity();
 #pragma omp parallel for schedule(dynamic, 64)
@@ -573,6 +582,7 @@ int pso_verify(int B, int n_draft, int n_target, int V, const int* draft_tokens,
     for (int i = 0; i <= n_draft; ++i) out[i] = -1;
     if (margin_accept) for (int i = 0; i < n_draft; ++i) margin_accept[(size_t)b * n_draft + i] = INF;
     if (margin_cdf) margin_cdf[b] = INF;
+    int nbr[2] = {-1, -1};
     int bad = 0, a = 0, emitted = -1;
     bool stopped = false;
     for (int i = 0; i < n_draft && !stopped; ++i) {
@@ -618,7 +628,7 @@ int pso_verify(int B, int n_draft, int n_target, int V, const int* draft_tokens,
           for (int v = 0; v < V; ++v) { w[v] = prob(t, v, temperature, st); W += w[v]; }
         }
         double mg;
-        emitted = inverse_cdf(w, W, u2, &mg);
+        emitted = inverse_cdf(w, W, u2, &mg, nbr);
         if (margin_cdf) margin_cdf[b] = mg;
       } else {
         emitted = argmax_row(t, V);  // defined fallback for poisoned rows
@@ -639,7 +649,7 @@ int pso_verify(int B, int n_draft, int n_target, int V, const int* draft_tokens,
           double W = 0.0;
           for (int v = 0; v < V; ++v) { w[v] = prob(t, v, temperature, st); W += w[v]; }
           double mg;
-          emitted = inverse_cdf(w, W, u2, &mg);
+          emitted = inverse_cdf(w, W, u2, &mg, nbr);
           if (margin_cdf) margin_cdf[b] = mg;
         }
       }
@@ -649,6 +659,7 @@ int pso_verify(int B, int n_draft, int n_target, int V, const int* draft_tokens,
     if (emitted >= 0) out[n++] = emitted;
     n_out[b] = n;
     if (nonfinite) nonfinite[b] = bad;
+    if (neighbours) { neighbours[2 * b] = nbr[0]; neighbours[2 * b + 1] = nbr[1]; }
   }
   return 0;
 }
@@ -694,11 +705,12 @@ int pso_gumbel_sample(const double* logits, int n_rows, int V, double temperatur
 // Outputs: accept_len[B] accepted nodes; path[B][max_depth] their ids (-1 unused);
 //   out_tokens[B][max_depth+1] their tokens followed by the token sampled at the node where
 //   the walk stopped (-1 unused); n_out[B] = accept_len + 1; margin_accept[B] = the smallest
-//   |r - min(1, p/q)| over the tests made; margin_cdf[B] as in pso_verify; nonfinite[B].
+//   |r - min(1, p/q)| over the tests made; margin_cdf[B], neighbours[B][2] (optional) as in
+//   pso_verify; nonfinite[B].
 int pso_verify_tree(int B, int n_nodes, int max_depth, int V, const int* parent, const int* tokens,
                     const float* draft_logits, const float* target_logits, double temperature,
                     uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
-                    int* path, double* margin_accept, double* margin_cdf, int* nonfinite) {
+                    int* path, double* margin_accept, double* margin_cdf, int* nonfinite, int* neighbours) {
   const double INF = std::numeric_limits<double>::infinity();
   std::vector<int> depth(n_nodes);
   for (int i = 0; i < n_nodes; ++i) {
@@ -714,6 +726,7 @@ int pso_verify_tree(int B, int n_nodes, int max_depth, int V, const int* parent,
     for (int i = 0; i <= max_depth; ++i) out[i] = -1;
     for (int i = 0; i < max_depth; ++i) pth[i] = -1;
     double m_acc = INF, m_cdf = INF;
+    int nbr[2] = {-1, -1};
     int bad = 0, a = 0, emitted = -1;
     int u = 0;                                   // decision row: 0 = root, 1 + node id
     std::vector<double> p(V), q(V);
@@ -765,7 +778,7 @@ int pso_verify_tree(int B, int n_nodes, int max_depth, int V, const int* parent,
       double r_unused, u2, W = 0.0;
       pso_uniforms(seed, offset, b, u, &r_unused, &u2);
       for (int v = 0; v < V; ++v) W += p[v];
-      emitted = inverse_cdf(p, W, u2, &m_cdf);
+      emitted = inverse_cdf(p, W, u2, &m_cdf, nbr);
       break;
     }
     accept_len[b] = a;
@@ -774,6 +787,7 @@ int pso_verify_tree(int B, int n_nodes, int max_depth, int V, const int* parent,
     if (margin_accept) margin_accept[b] = m_acc;
     if (margin_cdf) margin_cdf[b] = m_cdf;
     if (nonfinite) nonfinite[b] = bad;
+    if (neighbours) { neighbours[2 * b] = nbr[0]; neighbours[2 * b + 1] = nbr[1]; }
   }
   return 0;
 }

@@ -77,7 +77,7 @@ def _load():
             C.c_uint64, C.c_uint64, C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double),
         ]
         _lib.pso_verify.argtypes = (
-            [C.c_int] * 4 + [C.c_void_p] * 3 + [C.c_double, C.c_uint64, C.c_uint64] + [C.c_void_p] * 6
+            [C.c_int] * 4 + [C.c_void_p] * 3 + [C.c_double, C.c_uint64, C.c_uint64] + [C.c_void_p] * 7
         )
     return _lib
 
@@ -257,14 +257,16 @@ def verify(draft_tokens, draft_logits, target_logits, temperature: float, seed: 
     margin_accept = np.empty((B, n_draft), np.float64)
     margin_cdf = np.empty(B, np.float64)
     nonfinite = np.empty(B, np.int32)
+    neighbours = np.empty((B, 2), np.int32)
     rc = _load().pso_verify(B, n_draft, n_target, V, _ptr(draft_tokens), _ptr(draft_logits),
                             _ptr(target_logits), float(temperature), seed, offset, _ptr(accept_len),
                             _ptr(out_tokens), _ptr(n_out), _ptr(margin_accept), _ptr(margin_cdf),
-                            _ptr(nonfinite))
+                            _ptr(nonfinite), _ptr(neighbours))
     if rc != 0:
         raise ValueError(f"oracle verify status {rc}")
     return dict(accept_len=accept_len, out_tokens=out_tokens, n_out=n_out,
-                margin_accept=margin_accept, margin_cdf=margin_cdf, nonfinite=nonfinite)
+                margin_accept=margin_accept, margin_cdf=margin_cdf, nonfinite=nonfinite,
+                neighbours=neighbours)
 
 
 def verify_tree(parent, tokens, draft_logits, target_logits, temperature: float, seed: int, offset: int,
@@ -295,15 +297,17 @@ def verify_tree(parent, tokens, draft_logits, target_logits, temperature: float,
     lib.pso_verify_tree.restype = C.c_int
     lib.pso_verify_tree.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p, C.c_double, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p,
-                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    neighbours = np.empty((B, 2), np.int32)
     rc = lib.pso_verify_tree(B, n_nodes, max_depth, V, _ptr(parent), _ptr(tokens), _ptr(draft_logits),
                              _ptr(target_logits), float(temperature), seed, offset, _ptr(accept_len),
                              _ptr(out_tokens), _ptr(n_out), _ptr(path), _ptr(margin_accept), _ptr(margin_cdf),
-                             _ptr(nonfinite))
+                             _ptr(nonfinite), _ptr(neighbours))
     if rc != 0:
         raise ValueError(f"oracle verify_tree status {rc}")
     return dict(accept_len=accept_len, out_tokens=out_tokens, n_out=n_out, path=path,
-                margin_accept=margin_accept, margin_cdf=margin_cdf, nonfinite=nonfinite)
+                margin_accept=margin_accept, margin_cdf=margin_cdf, nonfinite=nonfinite,
+                neighbours=neighbours)
 
 
 def gumbel_sample(logits, temperature: float, seed: int, offset: int, row_id):

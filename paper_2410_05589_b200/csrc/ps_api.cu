@@ -506,6 +506,7 @@ ps_status ps_round_host(ps_ctx* c, int B, const int* seq_slot, const void* hidde
   if (s != PS_OK) return s;
   if (!hidden_last || !token_last || !target_logits || !accept_len || !out_tokens || !n_out)
     return fail(c, PS_ERR_INVALID_ARG, "null pointer");
+  if (!(temperature >= 0.f)) return fail(c, PS_ERR_INVALID_ARG, "temperature must be >= 0");
   cudaStream_t st = (cudaStream_t)stream;
   const ps_config& g = c->cfg;
   const int R = g.k_masks + 1;
@@ -526,9 +527,17 @@ ps_status ps_round_host(ps_ctx* c, int B, const int* seq_slot, const void* hidde
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(c->st_tok, token_last, (size_t)B * 4, cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return cuda_check(c, e, "ps_round_host h2d");
-  // top_n = 1: top_ids is then exactly the [B][k+1] chain of arg-max drafts.
-  s = ps_draft_step(c, B, seq_slot, c->st_hidden, c->st_tok, 1, c->st_top, (float*)(c->st_top + (size_t)c->max_rows),
-                    nullptr, nullptr, c->st_dlogits, nullptr, st);
+  // Drafts.  At temperature 0 the chain of arg-max tokens (top_n = 1: top_ids is then exactly
+  // [B][k+1]) meets a greedy verify.  Above 0 the acceptance rule keeps the target distribution
+  // only for drafts DRAWN from the q it is given (Eq. 1), so the tokens are sampled from
+  // softmax(draft logits / T) in the LM head with the round's seed and offset (the sampler's
+  // Philox key differs from verify's, so its uniforms are independent of the acceptance tests).
+  if (temperature > 0.f)
+    s = ps_draft_step_sampled(c, B, seq_slot, c->st_hidden, c->st_tok, temperature, seed, offset, c->st_top, 0,
+                              nullptr, nullptr, nullptr, nullptr, c->st_dlogits, nullptr, st);
+  else
+    s = ps_draft_step(c, B, seq_slot, c->st_hidden, c->st_tok, 1, c->st_top, (float*)(c->st_top + (size_t)c->max_rows),
+                      nullptr, nullptr, c->st_dlogits, nullptr, st);
   if (s != PS_OK) return s;
   int* r_acc = c->st_res;
   int* r_n = c->st_res + B;

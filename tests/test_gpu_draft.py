@@ -54,10 +54,25 @@ def test_mini32_ragged_batch():
     _compare_step(p, top_n=8)
 
 
-def test_mini_bf16_ragged_batch():
+@pytest.mark.parametrize("flags", [0, 2, 4], ids=["tcgen05", "unfused", "mma_sync"])
+def test_mini_bf16_ragged_batch(flags):
+    """The bf16 shape on each of the three kernel sets the library holds: the tcgen05 GEMMs, the
+    plain one-kernel-per-stage path (PS_FLAG_UNFUSED_KERNELS) and the mma.sync weight-streaming
+    GEMMs (PS_FLAG_MMA_SYNC_GEMM); contexts built by ps_kv_append on the same path."""
     s = synth.CONFIGS["mini"]
-    p = Pair(s, s.batch)
+    p = Pair(s, s.batch, flags=flags)
     _compare_step(p, top_n=8)
+    assert p.g.poll() == 0
+
+
+@pytest.mark.parametrize("flags", [2, 4], ids=["unfused", "mma_sync"])
+def test_fallback_kernels_more_rows_gqa_and_bias(flags):
+    """The two fall-back kernel sets beyond their single-launch sizes: 7 sequences x 3 rows (the
+    mma.sync GEMMs take 16 rows a launch), grouped-query attention, fc bias, top-1 only."""
+    s = synth.CONFIGS["mini"].with_(k_masks=2, n_kv_heads=2, batch=7, ctx_lo=3, ctx_hi=150)
+    p = Pair(s, 7, flags=flags, with_bias=True)
+    _compare_step(p, top_n=1)
+    assert p.g.poll() == 0
 
 
 def test_mini_bf16_more_masks_and_gqa():
@@ -217,7 +232,7 @@ def test_33b_batch16_k8_sampled_sequences():
 
 @pytest.mark.parametrize("name,B", [("mini", 3), ("mini", 1), ("tiny", 1)])
 def test_embedding_only_drafter(name, B):
-    """PS_FLAG_NO_FC: the drafter of the Medusa integration (Sec. 4.2), no fc and no target
+    """PS_FLAG_NO_FC: the drafter of the Medusa integration (Sec. 4.3), no fc and no target
     feature; contexts built by ps_kv_append, the tensor-core path (mini) and the plain one."""
     s = synth.CONFIGS[name]
     p = Pair(s, B, flags=8)

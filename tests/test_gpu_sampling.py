@@ -50,10 +50,12 @@ def _check_rows(s, got, want_logits_of, T, seed, offset, B):
                 assert margin[0] <= 2 * tol, (b, j, tok, int(t_o[0]), margin[0])
 
 
-@pytest.mark.parametrize("name,B", [("mini", 3), ("tiny", 1), ("mini", 1)])
-def test_sampled_tokens_match_oracle(name, B):
+@pytest.mark.parametrize("name,B,flags", [("mini", 3, 0), ("tiny", 1, 0), ("mini", 1, 0), ("mini", 3, 4), ("mini", 2, 2)])
+def test_sampled_tokens_match_oracle(name, B, flags):
+    """flags 4 / 2: the mma.sync GEMMs and the plain kernels, where one block per row draws the
+    token from the stored logits."""
     s = synth.CONFIGS[name]
-    p = Pair(s, B)
+    p = Pair(s, B, flags=flags)
     T, seed, offset = 0.8, 5, 12
     out = p.g.draft_step_sampled(list(range(B)), p.to_device(p.hidden_last), p.to_device(p.token_last),
                                  T, seed, offset, top_n=1)
@@ -127,3 +129,64 @@ def test_sampling_argument_errors():
     p = Pair(s, 1, lens=[10])
     with pytest.raises(ps.PsError):
         p.g.draft_step_sampled([0], p.to_device(p.hidden_last), p.to_device(p.token_last), 0.0, 1, 0)
+
+
+@pytest.mark.parametrize("name", ["mini", "tiny"])
+def test_round_host_is_lossless(name):
+    """ps_round_host (host buffers in, results out).  At temperature > 0 its drafts are drawn from
+    q = softmax(draft logits / T), the only case in which Eq. 1 keeps the target distribution:
+    (a) every round equals the oracle's verify applied to the tokens ps_draft_step_sampled draws
+    with the same seed and offset, (b) over many offsets the first emitted token follows
+    softmax(target row 0) (chi-square on 12 bins of equal mass) although the draft distribution
+    differs from it, (c) at temperature 0 the round is the greedy chain."""
+    from harness import assert_verify_same
+    s = synth.CONFIGS[name]
+    p = Pair(s, 1, lens=[33])
+    V, R, T, seed = s.vocab, s.rows, 1.0, 21
+    hl_d, tl_d = p.to_device(p.hidden_last), p.to_device(p.token_last)
+    ref = p.g.draft_step([0], hl_d, tl_d, top_n=1)
+    torch.cuda.synchronize()
+    logits = ref["logits"].cpu().numpy()
+    tgt = synth.noisy_draft_logits(s.seed, "rh", logits, 0.8 * float(logits.std()))
+    hl_h = torch.from_numpy(p.hidden_last.view(np.int16) if p.hidden_last.dtype == np.uint16 else p.hidden_last).pin_memory()
+    tl_h = torch.from_numpy(p.token_last).pin_memory()
+    tgt_h = torch.from_numpy(tgt).pin_memory()
+    n = 2400
+    first = np.empty(n, np.int64)
+    n_acc = 0
+    s_out, r_out = {}, {}
+    for off in range(n):
+        p.g.round_host([0], hl_h, tl_h, tgt_h, T, seed, off, out=r_out)
+        first[off] = int(r_out["out_tokens"][0, 0])
+        n_acc += int(r_out["accept_len"][0])
+        if off < 24:
+            o = p.g.draft_step_sampled([0], hl_d, tl_d, T, seed, off, top_n=1, out=s_out)
+            torch.cuda.synchronize()
+            want = oracle.verify(o["sampled"].cpu().numpy(), o["logits"].cpu().numpy(), tgt, T, seed, off)
+            got = {k: r_out[k].numpy().copy() for k in ("accept_len", "out_tokens", "n_out")}
+            assert_verify_same(got, want, max_excused=1)
+    assert 0 < n_acc < n * R          # acceptances and rejections both happened
+    z = tgt[0, 0].astype(np.float64) / T
+    pr = np.exp(z - z.max())
+    pr /= pr.sum()
+    order = np.argsort(-pr)
+    edges = np.searchsorted(np.cumsum(pr[order]), np.linspace(0, 1, 13)[1:-1])
+    bin_of = np.empty(V, np.int64)
+    bin_of[order] = np.searchsorted(edges, np.arange(V), side="right")
+    exp = np.bincount(bin_of, weights=pr, minlength=12) * n
+    obs = np.bincount(bin_of[first], minlength=12)
+    keep = exp > 5
+    assert stats.chisquare(obs[keep], exp[keep] * obs[keep].sum() / exp[keep].sum()).pvalue > 1e-3
+    # the arg-max drafts of the old behaviour would be accepted too often: the drafter's own
+    # distribution q_0 is not the law of the first token unless it equals p_0
+    zq = logits[0, 0].astype(np.float64) / T
+    q = np.exp(zq - zq.max())
+    q /= q.sum()
+    exp_q = np.bincount(bin_of, weights=q, minlength=12) * n
+    assert stats.chisquare(obs[keep], exp_q[keep] * obs[keep].sum() / exp_q[keep].sum()).pvalue < 1e-3
+    # temperature 0: greedy chain of arg-max drafts
+    p.g.round_host([0], hl_h, tl_h, tgt_h, 0.0, seed, 0, out=r_out)
+    want = oracle.verify(logits.argmax(-1).astype(np.int32), None, tgt, 0.0, seed, 0)
+    for k in ("accept_len", "out_tokens", "n_out"):
+        assert np.array_equal(r_out[k].numpy(), want[k]), k
+    assert p.g.poll() == 0

@@ -58,7 +58,14 @@ def _assert_same(got, want):
         if same:
             continue
         if np.array_equal(got["path"][b], want["path"][b]):
+            # same walk, another emitted token: only the neighbouring positive-weight token of the
+            # oracle's running sum is acceptable, and only when the draw sat on a CDF step
             assert want["margin_cdf"][b] < CDF_BAND, (b, want["margin_cdf"][b])
+            a = int(want["accept_len"][b])
+            assert got["accept_len"][b] == a and got["n_out"][b] == want["n_out"][b]
+            assert np.array_equal(got["out_tokens"][b, :a], want["out_tokens"][b, :a])
+            nb = [int(x) for x in want["neighbours"][b] if x >= 0]
+            assert int(got["out_tokens"][b, a]) in nb, (b, got["out_tokens"][b, a], nb)
         else:
             assert want["margin_accept"][b] < ACCEPT_BAND, (b, want["margin_accept"][b])
         excused += 1

@@ -232,6 +232,69 @@ def test_bf16_cache_rows_are_bf16_values(oracle_mod):
     assert np.isfinite(out["logits"]).all()
 
 
+def test_bf16_storage_against_library_layer(oracle_mod):
+    """The bf16 storage branch (weights, hidden states and cache given as bf16 bit patterns) against
+    the library layer fed the same values widened to float64.  The fc output involves no rounding
+    on either side, so it must agree to fp64 accuracy: a wrong widening of the bit patterns or a
+    wrong index in the bf16 matrix product fails here.  The logits differ only by the bf16
+    rounding of the k / v rows (relative 2^-9 per entry, Sec. 5.1 shapes use bf16 caches)."""
+    s = synth.CONFIGS["mini"].with_(hidden=256, n_heads=2, n_kv_heads=1, ffn=520, vocab=400, k_masks=3,
+                                    ctx_lo=9, ctx_hi=9)
+    W = synth.weights(s)
+    assert W["w_fc"].dtype == np.uint16
+    L = 9
+    ctx_h, ctx_t = synth.hidden_states(s, "c", L), synth.token_ids(s, "c", L)
+    hl, tl = synth.hidden_states(s, "l", 1), int(synth.token_ids(s, "l", 1)[0])
+    o = Oracle(_cfg(s), W)
+    assert o.kv_append(0, ctx_h, ctx_t) == 0
+    got = o.draft_step(0, hl, tl, taps=True)
+    x_in = _inputs(s, W, ctx_h, ctx_t, hl, tl, s.k_masks)
+    # (a) exact part: x_in rows and x0 = W_fc x_in of the k+1 new rows
+    np.testing.assert_array_equal(got["x_in"], x_in[L:])
+    x0 = x_in[L:] @ _as_f64(W["w_fc"], 1).T
+    np.testing.assert_allclose(got["x0"], x0, rtol=1e-12, atol=1e-13)
+    ms = (x0 ** 2).mean(1, keepdims=True)
+    np.testing.assert_allclose(got["xn"], x0 / np.sqrt(ms + s.rms_eps) * _as_f64(W["g_in"], 1), rtol=1e-12)
+    # (b) the whole layer: equal up to the bf16 rounding of cached k / v
+    for j in (0, s.k_masks):
+        ref_logits, ref_hdn = _library_forward(s, W, x_in[: L + 1 + j])
+        scale = np.abs(ref_logits[-1]).max()
+        err = np.abs(got["logits"][j] - ref_logits[-1]).max()
+        assert err < 4e-3 * scale, (j, err, scale)
+        assert err > 0.0                      # the cache really is rounded
+    # (c) the new rows' k / v are what a bf16 cache slot would hold
+    for name in ("k_new", "v_new"):
+        f = got[name].astype(np.float32)
+        assert np.array_equal(f.astype(np.float64), got[name])
+        assert np.all((f.view(np.uint32) & 0xFFFF) == 0)
+
+
+def test_bf16_cache_rounding_is_nearest_even(oracle_mod):
+    """Values stored in a bf16 cache are rounded to nearest, ties to even (R14: the cache is a
+    bf16 data structure).  Checked on exact halfway points and their fp32 neighbours, which
+    truncation, round-half-up and round-half-away each get wrong somewhere."""
+    s = synth.CONFIGS["mini"].with_(hidden=128, n_heads=1, n_kv_heads=1, head_dim=64, ffn=128, vocab=64)
+    o = Oracle(_cfg(s, max_batch=1, max_ctx=16), synth.weights(s))
+    cases = []   # (fp32 bits, expected bf16 bits)
+    for hi in (0x3F80, 0x3F81, 0x4049, 0x404A, 0xC2F6, 0xC2F7, 0x0080, 0x7F7E):
+        up = hi + 1
+        cases += [((hi << 16) | 0x8000, hi if hi % 2 == 0 else up),   # tie: to the even neighbour
+                  ((hi << 16) | 0x8001, up), ((hi << 16) | 0x7FFF, hi),
+                  ((hi << 16) | 0x0001, hi), ((hi << 16) | 0xFFFF, up), (hi << 16, hi)]
+    bits = np.array([c[0] for c in cases], np.uint32)
+    want = (np.array([c[1] for c in cases], np.uint32) << 16).view(np.float32).astype(np.float64)
+    vals = bits.view(np.float32).astype(np.float64)
+    w = s.n_kv_heads * s.head_dim
+    n = -(-len(vals) // w)
+    K = np.zeros((n, w)); V = np.zeros((n, w))
+    K.flat[: len(vals)] = vals
+    V.flat[: len(vals)] = -vals
+    o.kv_import(0, K, V)
+    Ke, Ve = o.kv_export(0)
+    np.testing.assert_array_equal(Ke.flat[: len(vals)], want)
+    np.testing.assert_array_equal(Ve.flat[: len(vals)], -want)
+
+
 def test_row_stats():
     rng = np.random.default_rng(0)
     x = rng.normal(size=(3, 50))
@@ -246,7 +309,7 @@ def test_row_stats():
 
 
 def test_embedding_only_input_is_the_identity_fc(oracle_mod):
-    """The embedding-only drafter of the Medusa integration (Sec. 4.2: shared embedding and LM
+    """The embedding-only drafter of the Medusa integration (Sec. 4.3: shared embedding and LM
     head, no target feature) is the pinned layer with fc = [I 0]: same logits, bit for bit."""
     from oracle import Oracle, OracleConfig
     s = synth.CONFIGS["mini32"].with_(k_masks=3)

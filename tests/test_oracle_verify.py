@@ -202,5 +202,53 @@ def test_margins_and_nonfinite(oracle_mod):
     bad[3, 0, 10] = np.nan
     res = oracle.verify(toks, draft, bad, 1.0, 1, 0)
     assert res["nonfinite"][3] == 1 and res["accept_len"][3] == 0 and res["nonfinite"].sum() == 1
+    # reading R17: the poisoned position is rejected and the arg-max over the row's non-NaN
+    # target logits is emitted (NaN counts as -inf, ties to the lower id)
+    row = bad[3, 0].astype(np.float64)
+    row[np.isnan(row)] = -np.inf
+    assert res["out_tokens"][3, 0] == int(np.argmax(row)) and res["n_out"][3] == 1
+    assert (res["out_tokens"][3, 1:] == -1).all()
+    bad2 = target.copy()
+    bad2[5, 0, :] = -1.0
+    bad2[5, 0, 0] = np.nan                       # NaN at id 0 must not win the tie among the rest
+    bad2[5, 0, [7, 9]] = 2.5
+    res = oracle.verify(toks, draft, bad2, 1.0, 1, 0)
+    assert res["nonfinite"][5] == 1 and res["out_tokens"][5, 0] == 7
+    # a poisoned DRAFT row rejects too and emits the target row's arg-max
+    badd = draft.copy()
+    badd[6, 0, 3] = np.inf
+    res = oracle.verify(toks, badd, target, 1.0, 1, 0)
+    assert res["nonfinite"][6] == 1 and res["accept_len"][6] == 0
+    assert res["out_tokens"][6, 0] == int(target[6, 0].argmax())
     with pytest.raises(ValueError):
         oracle.verify(toks, draft, target[:, :2], 1.0, 1, 0)
+
+
+def test_cdf_neighbours_are_the_adjacent_positive_weight_tokens(oracle_mod):
+    """The verify routines report, beside the sampled token, the positive-weight tokens on either
+    side of it in the running sum -- the only tokens a draw on a CDF boundary may turn into.
+    Checked by brute force on a residual with many zero-weight tokens."""
+    B, V = 200, 48
+    target = synth.gauss_logits(8, "nb", (B, 2, V))
+    draft = synth.noisy_draft_logits(8, "nb", target[:, :1], 1.5)
+    toks = synth.sample_from_logits(8, "nb", draft)
+    res = oracle.verify(toks, draft, target, 1.0, 4, 0)
+    p, q = _softmax(target.astype(np.float64)), _softmax(draft.astype(np.float64))
+    seen_zero_gap = 0
+    for b in range(B):
+        a = int(res["accept_len"][b])
+        w = np.maximum(p[b, 0] - q[b, 0], 0.0) if a == 0 else p[b, 1]
+        tok = int(res["out_tokens"][b, a])
+        assert w[tok] > 0.0
+        pos = np.flatnonzero(w > 0.0)
+        k = int(np.searchsorted(pos, tok))
+        lo = int(pos[k - 1]) if k > 0 else -1
+        hi = int(pos[k + 1]) if k + 1 < len(pos) else -1
+        assert list(res["neighbours"][b]) == [lo, hi], (b, tok, lo, hi, res["neighbours"][b])
+        seen_zero_gap += (lo >= 0 and tok - lo > 1) or (hi >= 0 and hi - tok > 1)
+    assert seen_zero_gap > 10      # the zero-weight gaps were really skipped
+    # a draw at the very end of the running sum has no successor
+    t1 = np.full((1, 1, V), -np.inf, np.float32)
+    t1[0, 0, 5] = 0.0
+    r1 = oracle.verify(np.array([[3]], np.int32), None, t1, 1.0, 1, 0)
+    assert r1["out_tokens"][0, 0] == 5 and list(r1["neighbours"][0]) == [-1, -1]
