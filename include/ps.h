@@ -235,6 +235,26 @@ ps_status ps_verify_tree(ps_ctx* ctx, int B, int n_nodes, const int* parent, con
                          uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,
                          int* n_out, int* path, void* stream);
 
+/* Drafts a token tree of a static shape from one parallel draft step (Algorithm 1, the lines
+ * that build the tree before the target pass; appendix "Token Tree Verification": the
+ * highest-probability tokens of every drafted position are the candidates, fewer of them the
+ * deeper the position).  The parallel drafter gives ONE distribution per depth, whatever the
+ * path, so node i of depth t = depth(i) takes the rank[i]-th most likely token of row t of the
+ * draft step: tokens[b][i] = top_ids[b][t][rank[i]]; where sampled_ids is given, rank 0 takes
+ * sampled_ids[b][t] instead (the token ps_draft_step_sampled drew for that row), and a rank
+ * r > 0 whose top-n entry equals that sampled token takes entry 0 (so that siblings stay
+ * distinct).  parent[] as in ps_verify_tree; the outputs feed ps_verify_tree unchanged, with the
+ * first D rows of the draft step's logits as its draft_logits.
+ *   parent, rank  HOST [n_nodes] int32; 0 <= rank[i] < top_n; siblings must differ in rank
+ *   top_ids       device [B][k+1][top_n] int32 (ps_draft_step's output), top_n >= 1
+ *   sampled_ids   device [B][k+1] int32 or NULL
+ *   tokens        device [B][n_nodes] int32 (output)
+ * PS_ERR_INVALID_ARG for a malformed tree, a depth beyond k, a rank beyond top_n or two siblings
+ * of the same rank.  Nothing runs on the host but the validation. */
+ps_status ps_build_tree(ps_ctx* ctx, int B, int n_nodes, const int* parent, const int* rank,
+                        const int* top_ids, int top_n, const int* sampled_ids, int* tokens,
+                        void* stream);
+
 /* Host-buffer convenience for one draft+verify round: copies hidden_last / token_last /
  * target_logits from host memory, runs the draft step for all k+1 rows and ps_verify
  * (n_draft = n_target = k+1) on `stream`, copies accept_len / out_tokens / n_out back and waits

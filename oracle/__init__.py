@@ -7,6 +7,7 @@ from .ps_oracle import (  # noqa: F401
     Oracle,
     OracleConfig,
     build_oracle,
+    build_tree,
     gumbel_sample,
     num_threads,
     philox4x32,

@@ -18,6 +18,9 @@
 //   pso_verify_tree Algorithm 1 in full: a token tree, children tried in turn, the
 //                   target distribution replaced by its normalised residual after
 //                   every rejection
+//   pso_build_tree  Algorithm 1's drafting of the tree N and the appendix "Token Tree
+//                   Verification": the candidates of a position are its highest-probability
+//                   tokens; with a parallel drafter every node of one depth shares one row
 //   pso_gumbel_sample  Algorithm 1's "sampling from the parallel draft model": one token per
 //                   row drawn from softmax(logits/T) by the Gumbel-max rule with Philox uniforms
 //   pso_philox4x32  Salmon et al., "Parallel random numbers: as easy as 1, 2, 3"
@@ -688,6 +691,35 @@ int pso_gumbel_sample(const double* logits, int n_rows, int V, double temperatur
     tokens[r] = arg;
     if (margin) margin[r] = best - second;
   }
+  return 0;
+}
+
+// The draft tree of Algorithm 1 for a static shape (appendix "Token Tree Verification": each
+// position's candidates are its most probable tokens).  The parallel drafter yields one
+// distribution per depth, so node i at depth t carries the rank[i]-th entry of that depth's
+// top-n list; when sampled tokens are given, rank 0 carries the sampled token of the depth and a
+// deeper rank whose entry is that very token carries entry 0 instead.
+//   parent[n_nodes] (-1: child of the root), rank[n_nodes], top_ids [B][R][top_n] (R rows per
+//   sequence), sampled [B][R] or NULL  ->  tokens [B][n_nodes].  Returns -1 for a bad tree.
+int pso_build_tree(int B, int n_nodes, int R, int top_n, const int* parent, const int* rank, const int* top_ids,
+                   const int* sampled, int* tokens) {
+  std::vector<int> depth(n_nodes);
+  for (int i = 0; i < n_nodes; ++i) {
+    if (parent[i] >= i || parent[i] < -1) return -1;
+    depth[i] = parent[i] < 0 ? 0 : depth[parent[i]] + 1;
+    if (depth[i] >= R || rank[i] < 0 || rank[i] >= top_n) return -1;
+  }
+  for (int b = 0; b < B; ++b)
+    for (int i = 0; i < n_nodes; ++i) {
+      const int* list = top_ids + ((size_t)b * R + depth[i]) * top_n;
+      int tok = list[rank[i]];
+      if (sampled) {
+        const int sx = sampled[(size_t)b * R + depth[i]];
+        if (rank[i] == 0) tok = sx;
+        else if (tok == sx) tok = list[0];
+      }
+      tokens[(size_t)b * n_nodes + i] = tok;
+    }
   return 0;
 }
 

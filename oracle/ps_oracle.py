@@ -310,6 +310,27 @@ def verify_tree(parent, tokens, draft_logits, target_logits, temperature: float,
                 neighbours=neighbours)
 
 
+def build_tree(parent, rank, top_ids, sampled=None):
+    """The draft tree of a static shape from per-depth top-n lists: parent, rank [n_nodes];
+    top_ids [B][R][top_n] int32; sampled [B][R] int32 or None.  Returns tokens [B][n_nodes]."""
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    rank = np.ascontiguousarray(rank, dtype=np.int32)
+    top_ids = np.ascontiguousarray(top_ids, dtype=np.int32)
+    B, R, top_n = top_ids.shape
+    if sampled is not None:
+        sampled = np.ascontiguousarray(sampled, dtype=np.int32)
+        assert sampled.shape == (B, R)
+    tokens = np.empty((B, len(parent)), np.int32)
+    lib = _load()
+    lib.pso_build_tree.restype = C.c_int
+    lib.pso_build_tree.argtypes = [C.c_int] * 4 + [C.c_void_p] * 5
+    rc = lib.pso_build_tree(B, len(parent), R, top_n, _ptr(parent), _ptr(rank), _ptr(top_ids), _ptr(sampled),
+                            _ptr(tokens))
+    if rc != 0:
+        raise ValueError(f"oracle build_tree status {rc}")
+    return tokens
+
+
 def gumbel_sample(logits, temperature: float, seed: int, offset: int, row_id):
     """One token per row from softmax(logits / T) by the Gumbel-max rule with the Philox stream
     of the draft sampler.  logits [rows][V] float64, row_id [rows] int (b | j << 8).

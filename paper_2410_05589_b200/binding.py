@@ -30,6 +30,7 @@ EXPORTS = (
     "ps_kv_len", "ps_kv_reset", "ps_kv_export", "ps_kv_import", "ps_poll", "ps_launch_count",
     "ps_last_error", "ps_destroy", "ps_philox_fill", "ps_profile", "ps_profile_read",
     "ps_verify_static", "ps_debug_buffer", "ps_verify_tree", "ps_draft_step_sampled", "ps_group_forward",
+    "ps_build_tree",
 )
 
 
@@ -79,6 +80,7 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.ps_group_forward.argtypes = [vp, C.c_int, C.c_int, vp, vp, C.c_int, vp, vp, vp, vp, vp, vp, vp]
     lib.ps_verify_tree.argtypes = [vp, C.c_int, C.c_int, ip, vp, vp, vp, C.c_float, C.c_uint64, C.c_uint64,
                                    vp, vp, vp, vp, vp]
+    lib.ps_build_tree.argtypes = [vp, C.c_int, C.c_int, ip, ip, vp, C.c_int, vp, vp, vp]
     lib.ps_kv_len.argtypes = [vp, C.c_int, ip]
     lib.ps_kv_reset.argtypes = [vp, C.c_int]
     lib.ps_kv_export.argtypes = [vp, C.c_int, vp, vp, vp]
@@ -335,6 +337,18 @@ class Drafter:
             float(temperature), seed, offset, _dptr(o["accept_len"]), _dptr(o["out_tokens"]),
             _dptr(o["n_out"]), _dptr(o["path"]), _stream(stream)))
         return o
+
+    def build_tree(self, parent, rank, top_ids: torch.Tensor, sampled_ids=None, out=None, stream=None):
+        """ps_build_tree.  parent, rank: host lists [n_nodes]; top_ids [B][k+1][top_n] int32 (a draft
+        step's output); sampled_ids [B][k+1] int32 or None.  Returns tokens [B][n_nodes] int32."""
+        B, R, top_n = top_ids.shape
+        assert R == self.rows and top_ids.dtype == torch.int32 and top_ids.is_contiguous()
+        n_nodes = len(parent)
+        assert len(rank) == n_nodes
+        tokens = out if out is not None else torch.empty((B, n_nodes), dtype=torch.int32, device="cuda")
+        self._check(self.lib.ps_build_tree(self.h, B, n_nodes, _iarr(parent), _iarr(rank), _dptr(top_ids), top_n,
+                                           _dptr(sampled_ids), _dptr(tokens), _stream(stream)))
+        return tokens
 
     def round_host(self, seq_slot, hidden_last: torch.Tensor, token_last: torch.Tensor,
                    target_logits: torch.Tensor, temperature: float, seed: int, offset: int,

@@ -497,6 +497,16 @@ ps_status ps_verify_tree(ps_ctx* c, int B, int n_nodes, const int* parent, const
                             offset, accept_len, out_tokens, n_out, path, nullptr, (cudaStream_t)stream);
 }
 
+ps_status ps_build_tree(ps_ctx* c, int B, int n_nodes, const int* parent, const int* rank, const int* top_ids,
+                        int top_n, const int* sampled_ids, int* tokens, void* stream) {
+  if (!c) return PS_ERR_INVALID_ARG;
+  if (B < 1 || B > PS_MAX_BATCH) return fail(c, PS_ERR_INVALID_ARG, "bad batch");
+  if (n_nodes < 1 || n_nodes > PS_MAX_TREE_NODES) return fail(c, PS_ERR_CAPACITY, "tree of 1..PS_MAX_TREE_NODES nodes");
+  if (!parent || !rank || !top_ids || !tokens) return fail(c, PS_ERR_INVALID_ARG, "null pointer");
+  if (top_n < 1 || top_n > PS_MAX_TOP_N) return fail(c, PS_ERR_INVALID_ARG, "top_n out of range");
+  return launch_build_tree(c, B, n_nodes, parent, rank, top_ids, top_n, sampled_ids, tokens, (cudaStream_t)stream);
+}
+
 ps_status ps_round_host(ps_ctx* c, int B, const int* seq_slot, const void* hidden_last,
                         const int* token_last, const float* target_logits, float temperature,
                         uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens,

@@ -194,6 +194,8 @@ ps_status launch_verify_tree(ps_ctx* c, int B, int n_nodes, const int* parent, c
                              const float* draft_logits, const float* target_logits, float temperature,
                              uint64_t seed, uint64_t offset, int* accept_len, int* out_tokens, int* n_out,
                              int* path, int* max_depth_out, cudaStream_t st);
+ps_status launch_build_tree(ps_ctx* c, int B, int n_nodes, const int* parent, const int* rank, const int* top_ids,
+                            int top_n, const int* sampled_ids, int* tokens, cudaStream_t st);
 ps_status launch_kv_copy(ps_ctx* c, int slot, int len, void* K, void* V, bool to_cache,
                          cudaStream_t st);
 }  // namespace ps

@@ -903,7 +903,48 @@ __global__ void __launch_bounds__(kCluThreads) k_verify_tree(TreeArgs a) {
   cl.sync();   // no block leaves while another may still read its shared memory
 }
 
+// Token tree from the top-n lists of a draft step (see ps_build_tree): one thread per node.
+struct BuildArgs {
+  int B, n_nodes, R, top_n;
+  unsigned char depth[PS_MAX_TREE_NODES], rank[PS_MAX_TREE_NODES];
+  const int* top_ids; const int* sampled; int* tokens;
+};
+__global__ void k_build_tree(BuildArgs a) {
+  const int i = threadIdx.x, b = blockIdx.x;
+  if (i >= a.n_nodes) return;
+  const int t = a.depth[i], r = a.rank[i];
+  const int* top = a.top_ids + ((size_t)b * a.R + t) * a.top_n;
+  int tok = top[r];
+  if (a.sampled) {
+    const int sx = a.sampled[(size_t)b * a.R + t];
+    if (r == 0) tok = sx;
+    else if (tok == sx) tok = top[0];
+  }
+  a.tokens[(size_t)b * a.n_nodes + i] = tok;
+}
+
 }  // namespace
+
+ps_status launch_build_tree(ps_ctx* c, int B, int n_nodes, const int* parent, const int* rank, const int* top_ids,
+                            int top_n, const int* sampled_ids, int* tokens, cudaStream_t st) {
+  BuildArgs a;
+  a.B = B; a.n_nodes = n_nodes; a.R = c->cfg.k_masks + 1; a.top_n = top_n;
+  a.top_ids = top_ids; a.sampled = sampled_ids; a.tokens = tokens;
+  for (int i = 0; i < n_nodes; ++i) {
+    if (parent[i] >= i || parent[i] < -1) return fail(c, PS_ERR_INVALID_ARG, "parent[i] must be -1 or a node before i");
+    const int d = parent[i] < 0 ? 0 : a.depth[parent[i]] + 1;
+    if (d >= a.R) return fail(c, PS_ERR_INVALID_ARG, "the tree is deeper than the k+1 rows of a draft step");
+    if (rank[i] < 0 || rank[i] >= top_n) return fail(c, PS_ERR_INVALID_ARG, "rank[i] must be in [0, top_n)");
+    for (int j = 0; j < i; ++j)
+      if (parent[j] == parent[i] && rank[j] == rank[i])
+        return fail(c, PS_ERR_INVALID_ARG, "two siblings of the same rank would carry the same token");
+    a.depth[i] = (unsigned char)d;
+    a.rank[i] = (unsigned char)rank[i];
+  }
+  k_build_tree<<<B, PS_MAX_TREE_NODES, 0, st>>>(a);
+  c->launches++;
+  return cuda_check(c, cudaGetLastError(), "k_build_tree");
+}
 
 // Launch with a cluster of nclu blocks along x (a launch attribute, not a compile-time one).
 template <class Args>

@@ -131,3 +131,69 @@ def test_tree_argument_errors_and_nonfinite():
     _assert_same(got, want)
     assert want["nonfinite"][2] == 1 and got["accept_len"][2] == 0
     assert g.poll() == -6   # PS_ERR_NONFINITE
+
+
+@pytest.mark.parametrize("sampled", [False, True])
+def test_draft_step_build_tree_verify_tree_chain(sampled):
+    """A whole tree round with nothing on the host (Algorithm 1): ps_draft_step (top-4 per row) ->
+    ps_build_tree (static 26-node shape, rank = position among the siblings) -> target logits ->
+    ps_verify_tree.  The top-n lists are checked against the oracle's draft step, the tree tokens
+    against the oracle's build_tree bit for bit, the walk against the oracle's verify_tree on the
+    kernel's draft logits, at temperatures 1 and 0."""
+    import paper_2410_05589_b200 as ps
+    from harness import Pair, check_top
+    s = synth.CONFIGS["mini"].with_(k_masks=5)
+    B = 3
+    p = Pair(s, B, lens=[21, 60, 5])
+    parent = TREE26
+    depth = _depths(parent)
+    rank = []
+    for i, par in enumerate(parent):
+        rank.append(sum(1 for j in range(i) if parent[j] == par))
+    D = int(depth.max()) + 1
+    assert D <= s.rows and max(rank) < 4
+    hl, tl_ = p.to_device(p.hidden_last), p.to_device(p.token_last)
+    if sampled:
+        out = p.g.draft_step_sampled(list(range(B)), hl, tl_, 1.0, 5, 2, top_n=4)
+    else:
+        out = p.g.draft_step(list(range(B)), hl, tl_, top_n=4)
+    toks_d = p.g.build_tree(parent, rank, out["top_ids"], out["sampled"] if sampled else None)
+    torch.cuda.synchronize()
+    top_ids = out["top_ids"].cpu().numpy()
+    for b in range(B):
+        want = p.oracle_step(b)
+        for j in range(s.rows):
+            check_top(top_ids[b, j], out["top_logit"][b, j].cpu().numpy(), want["logits"][j], s.dtype)
+    toks = toks_d.cpu().numpy()
+    smp = out["sampled"].cpu().numpy() if sampled else None
+    assert np.array_equal(toks, oracle.build_tree(parent, rank, top_ids, smp))
+    for b in range(B):          # siblings carry distinct tokens
+        for par in set(parent):
+            kids = [i for i in range(len(parent)) if parent[i] == par]
+            assert len({int(toks[b, i]) for i in kids}) == len(kids)
+    dl = out["logits"][:, :D].contiguous()
+    dl_np = dl.cpu().numpy()
+    # target rows: the drafter's row of the node's depth plus noise, so that deep paths occur
+    tgt = synth.gauss_logits(9, "chain_t", (B, len(parent) + 1, s.vocab), sigma=1.0)
+    tgt[:, 0] += dl_np[:, 0]
+    for i in range(len(parent)):
+        if depth[i] + 1 < D:
+            tgt[:, 1 + i] += dl_np[:, depth[i] + 1]
+    hits = 0
+    for T in (1.0, 0.0):
+        for off in range(4):
+            got = p.g.verify_tree(parent, toks_d, dl, ps.to_device(tgt), T, 3, off)
+            torch.cuda.synchronize()
+            got = {k: v.cpu().numpy() for k, v in got.items()}
+            want = oracle.verify_tree(parent, toks, dl_np, tgt, T, 3, off, max_depth=D)
+            _assert_same(got, want)
+            hits += int(want["accept_len"].sum())
+    assert hits > 0
+    # malformed requests come back as a status
+    with pytest.raises(ps.PsError):
+        p.g.build_tree([-1, -1], [0, 0], out["top_ids"])            # two siblings of one rank
+    with pytest.raises(ps.PsError):
+        p.g.build_tree([-1, 0], [0, 4], out["top_ids"])             # rank beyond top_n
+    with pytest.raises(ps.PsError):
+        p.g.build_tree(list(range(-1, 6)), [0] * 7, out["top_ids"])  # deeper than k+1 rows
+    assert p.g.poll() == 0

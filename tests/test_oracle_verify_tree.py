@@ -167,3 +167,102 @@ def test_malformed_trees_are_rejected(oracle_mod):
         oracle.verify_tree(np.array([1, -1]), toks, draft, target, 1.0, 1, 0)      # parent after child
     with pytest.raises(ValueError):
         oracle.verify_tree(np.array([-1, 0]), toks, draft, target, 1.0, 1, 0)      # depth 1 needs 2 rows of q
+
+
+def _full_tree(fan):
+    """parent / rank lists of the tree whose nodes at depth t are all combinations of ranks
+    below fan[t] (breadth-first node ids), and each node's tuple of ranks from the root."""
+    parent, rank, ranks_of = [], [], []
+    level = [(-1, ())]
+    for f in fan:
+        nxt = []
+        for pid, pr in level:
+            for r in range(f):
+                parent.append(pid)
+                rank.append(r)
+                ranks_of.append(pr + (r,))
+                nxt.append((len(parent) - 1, pr + (r,)))
+        level = nxt
+    return parent, rank, ranks_of
+
+
+def test_build_tree_paths_are_the_product_of_the_top_lists(oracle_mod):
+    """Drafting the tree (Algorithm 1; appendix "Token Tree Verification"): with one draft
+    distribution per depth, the root-to-leaf token paths of the tree with fan-out fan[t] at depth t
+    are exactly the Cartesian product of the depths' top-fan[t] lists, written here with
+    itertools; a chain of rank 0 is the arg-max chain."""
+    import itertools
+    rng = np.random.default_rng(5)
+    B, R, top_n, V = 3, 4, 4, 50
+    top = np.stack([np.stack([rng.permutation(V)[:top_n] for _ in range(R)]) for _ in range(B)]).astype(np.int32)
+    fan = (3, 2, 2)
+    parent, rank, ranks_of = _full_tree(fan)
+    toks = oracle.build_tree(parent, rank, top)
+    leaves = [i for i in range(len(parent)) if i not in set(parent)]
+    for b in range(B):
+        paths = set()
+        for leaf in leaves:
+            path, i = [], leaf
+            while i >= 0:
+                path.append(int(toks[b, i]))
+                i = parent[i]
+            paths.add(tuple(reversed(path)))
+        want = set(itertools.product(*[top[b, t, :fan[t]].tolist() for t in range(len(fan))]))
+        assert paths == want
+    chain = oracle.build_tree([-1, 0, 1, 2], [0, 0, 0, 0], top)
+    assert np.array_equal(chain, top[:, :, 0])
+    with pytest.raises(ValueError):
+        oracle.build_tree([-1, 0, 1, 2, 3], [0] * 5, top)          # deeper than the R rows
+    with pytest.raises(ValueError):
+        oracle.build_tree([-1, 0], [0, top_n], top)                # rank beyond the list
+
+
+def test_build_tree_with_sampled_tokens_keeps_siblings_distinct(oracle_mod):
+    rng = np.random.default_rng(6)
+    B, R, top_n, V = 64, 3, 4, 12
+    top = np.stack([np.stack([rng.permutation(V)[:top_n] for _ in range(R)]) for _ in range(B)]).astype(np.int32)
+    sampled = rng.integers(0, V, size=(B, R)).astype(np.int32)
+    sampled[::2] = top[::2, :, 2]                                    # often one of the listed tokens
+    parent, rank, ranks_of = _full_tree((4, 3))
+    toks = oracle.build_tree(parent, rank, top, sampled)
+    for b in range(B):
+        for i in range(len(parent)):
+            t = len(ranks_of[i]) - 1
+            if rank[i] == 0:
+                assert toks[b, i] == sampled[b, t]
+        for p in set(parent):
+            kids = [i for i in range(len(parent)) if parent[i] == p]
+            assert len({int(toks[b, i]) for i in kids}) == len(kids)   # no token twice among siblings
+
+
+def test_greedy_tree_round_accepts_while_the_target_token_is_listed(oracle_mod):
+    """build_tree + verify_tree at temperature 0 against a closed form: with the full tree of
+    fan-out n, the walk goes on exactly as long as the target's arg-max after the accepted path
+    is among the drafter's n most likely tokens of that depth."""
+    rng = np.random.default_rng(7)
+    B, R, top_n, V = 40, 3, 3, 30
+    fan = (3, 3, 3)
+    parent, rank, ranks_of = _full_tree(fan)
+    n = len(parent)
+    top = np.stack([np.stack([rng.permutation(V)[:top_n] for _ in range(R)]) for _ in range(B)]).astype(np.int32)
+    toks = oracle.build_tree(parent, rank, top)
+    tl = rng.normal(0, 1, size=(B, n + 1, V)).astype(np.float32)
+    # make the target's arg-max a listed token with probability ~2/3 at every decision row
+    for b in range(B):
+        for u in range(n + 1):
+            t = 0 if u == 0 else len(ranks_of[u - 1])
+            if t < R and rng.random() < 0.67:
+                tl[b, u, top[b, t, rng.integers(0, top_n)]] = 9.0
+    res = oracle.verify_tree(parent, toks, None, tl, 0.0, 1, 0, max_depth=len(fan))
+    for b in range(B):
+        u, acc = 0, 0
+        while acc < len(fan):
+            star = int(tl[b, u].argmax())
+            kids = [i for i in range(n) if parent[i] == u - 1]
+            hit = [i for i in kids if toks[b, i] == star]
+            if not hit:
+                break
+            u, acc = hit[0] + 1, acc + 1
+        assert res["accept_len"][b] == acc
+        assert res["out_tokens"][b, acc] == int(tl[b, u].argmax())
+    assert res["accept_len"].max() == len(fan) and res["accept_len"].min() == 0
