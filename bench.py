@@ -3,15 +3,21 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 13b|7b|33b|13b_sweep|tiny]
                     [--batch B] [--k-masks k]     # a point of the batch / mask-count sweep
+                    [--flags F]                   # ps_config.flags (2: plain kernels, 4: mma.sync GEMMs)
+                    [--no-configs]                # skip the other workloads' sub-records
     python bench.py --impl reference ...      # the CPU checker timed on the host cores
 
 One "step" = one parallel draft step (all k+1 rows, logits stored) followed by one verify
-call on synthetic target logits, for the workload's batch.  N > 1 (under torchrun) runs N
-independent replicas, one per GPU, with no data-path collective.  Rank 0 prints ONE JSON line.
+call on synthetic target logits, for the workload's batch.  At temperature > 0 the drafts are
+drawn from the draft distribution inside the LM head (ps_draft_step_sampled), which is what
+makes the round lossless (Eq. 1 needs x ~ q); at temperature 0 they are the rows' arg-max
+tokens.  N > 1 (under torchrun) runs N independent replicas, one per GPU, with no data-path
+collective.  Rank 0 prints ONE JSON line.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -27,6 +33,7 @@ METRIC = "draft+verify steps/sec"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 << 20
+VERIFY_SIGMA = 0.4     # draft logits = target + N(0, sigma^2): about 3.5 tokens a round at k = 4 (Table 1's regime)
 
 
 def parse_args():
@@ -40,8 +47,10 @@ def parse_args():
     ap.add_argument("--batch", type=int, default=0, help="sequences per step (default: the workload's)")
     ap.add_argument("--k-masks", type=int, default=-1, help="[MASK] positions per sequence (default: the workload's)")
     ap.add_argument("--temperature", type=float, default=1.0)
+    ap.add_argument("--flags", type=int, default=0, help="ps_config.flags of the context")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--no-configs", action="store_true", help="headline workload only")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
     return ap.parse_args()
 
 
@@ -68,17 +77,30 @@ def kernel_of_stage(stage, rows):
     return KERNEL_OF_STAGE.get(stage, stage)
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
-# profiles/k_umma_gemm_13b_b1_k4.md, keyed by (workload, batch, k_masks, stage).  Valid for the
-# kernels as captured; set an entry to None when its kernel changes.
-NCU_DRAM_BYTES = {
-    ("13b", 1, 4, "fc_norm"): 106259200 + 4141824,
-    ("13b", 1, 4, "qkv_rope"): 158127872 + 3880704,
-    ("13b", 1, 4, "o_proj"): 53316352 + 8960,
-    ("13b", 1, 4, "ffn_gate_up"): 285139968 + 4767232,
-    ("13b", 1, 4, "ffn_down"): 143910144 + 4637184,
-    ("13b", 1, 4, "lm_head"): 329474816 + 5147648,
-}
+def kernel_sources_digest():
+    """sha256 over the kernel sources: a counter capture is valid for the sources it was taken on."""
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2410_05589_b200", "csrc")
+    for name in sorted(os.listdir(d)):
+        if name.endswith((".cu", ".cuh")):
+            with open(os.path.join(d, name), "rb") as f:
+                h.update(name.encode())
+                h.update(f.read())
+    return h.hexdigest()
+
+
+def captured_dram_bytes(workload, B, k, stage):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the stage's kernel, from the
+    counter capture recorded under profiles/ -- or None when there is none for this workload or
+    the kernel sources have changed since it was taken."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_bytes_per_launch.json")) as f:
+            rec = json.load(f)
+        if rec.get("kernel_sources_sha256") != kernel_sources_digest():
+            return None
+        return rec["bytes"].get(f"{workload}/B{B}/k{k}/{stage}")
+    except Exception:
+        return None
 
 
 def stage_bytes(s, B, lens):
@@ -98,53 +120,6 @@ def stage_bytes(s, B, lens):
         "lm_head": e * V * H + 4 * M * V,
         "verify": 8 * M * V,
     }
-
-
-# A 26-node draft tree of the shape tree drafters use (4 children of the root, depth 6).
-TREE26 = [-1, -1, -1, -1, 0, 0, 0, 1, 1, 2, 4, 4, 5, 7, 10, 10, 11, 12, 13, 14, 14, 16, 18, 19, 21, 22]
-
-
-def tree_verify_leg(g, ps, s, B, T, peak, n_buf=6, reps=60):
-    """ps_verify_tree alone on the 26-node tree: synthetic target rows per node, one draft row
-    per depth (noisy copies, so that paths of several nodes are accepted), node tokens drawn
-    from the draft rows.  Buffers rotate so that rows come from HBM, not from L2."""
-    import numpy as np
-    import torch
-
-    import synth
-    n = len(TREE26)
-    depth = []
-    for p in TREE26:
-        depth.append(0 if p < 0 else depth[p] + 1)
-    D, V = max(depth) + 1, s.vocab
-    sets = []
-    for i in range(n_buf):
-        tl = synth.gauss_logits(s.seed, ("tree_t", i), (B, n + 1, V))
-        dl = synth.noisy_draft_logits(s.seed, ("tree_d", i), np.repeat(tl[:, :1], D, axis=1), 0.6)
-        for j in range(n):
-            if depth[j] + 1 < D:
-                tl[:, 1 + j] = dl[:, depth[j] + 1] + 0.5 * tl[:, 1 + j]
-        toks = synth.sample_from_logits(s.seed, ("tree_x", i), dl[:, depth], temperature=max(T, 0.5))
-        sets.append((ps.to_device(toks.astype(np.int32)), ps.to_device(dl), ps.to_device(tl)))
-    out = {}
-    for i in range(5):
-        t_, d_, l_ = sets[i % n_buf]
-        g.verify_tree(TREE26, t_, d_, l_, T, 1, i, out=out)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(reps):
-        t_, d_, l_ = sets[i % n_buf]
-        g.verify_tree(TREE26, t_, d_, l_, T, 1, 100 + i, out=out)
-    e1.record()
-    torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) / reps * 1e3
-    rows_with_children = len({p for p in TREE26})            # decision rows that read a draft row
-    nbytes = 4 * V * B * ((n + 1) + rows_with_children)
-    return {"us": round(us, 2), "nodes": n, "depth": D, "bytes": nbytes,
-            "gbs": round(nbytes / (us * 1e-6) / 1e9, 1), "frac_of_peak": round(nbytes / (us * 1e-6) / 1e9 / peak, 4),
-            "mean_accepted_nodes": float(out["accept_len"].float().mean().item()),
-            "note": "(n+1) target rows and one draft row per row with children, each read once"}
 
 
 def max_over_ranks(x: float, device="cuda") -> float:
@@ -222,6 +197,7 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
+# ---- the CPU checker as a timed baseline ---------------------------------------------------------
 def oracle_setup(s, B, lens):
     import oracle
     import synth
@@ -255,11 +231,13 @@ def oracle_time_step(o, s, b, k_use, hidden_last, token_last, target, T):
 
 
 def cpu_baseline(s, B, lens, hidden_last, token_last, target, T, budget_s):
-    """The CPU checker, as it stands, on a bounded sample of the same workload."""
+    """The CPU checker, as it stands, on a bounded sample of the same workload: on all host
+    cores, and (a shorter sample) on one."""
     import oracle
 
     o = oracle_setup(s, B, lens)
     R = s.rows
+    cores = oracle.num_threads()
     # first: one row of sequence 0 to size the sample
     t_row = oracle_time_step(o, s, 0, 0, hidden_last, token_last, target, T)
     full_step = t_row * R * B
@@ -278,16 +256,24 @@ def cpu_baseline(s, B, lens, hidden_last, token_last, target, T, budget_s):
     est_step = t * (B * R) / rows_done
     sample = (f"{reps} x ({n_seq} of {B} sequences x {k_use + 1} of {R} rows of one draft+verify "
               f"step), {t:.1f} s of CPU work, scaled by rows to a full step")
-    return {"value": 1.0 / est_step, "unit": "steps/s", "cores": oracle.num_threads(),
-            "kind": "oracle", "sample": sample}
+    # one thread: rows of sequence 0 for about a third of the budget
+    oracle.set_threads(1)
+    t1, rows1 = 0.0, 0
+    while rows1 == 0 or (t1 < budget_s / 3 and rows1 < 4 * R):
+        k1 = min(s.k_masks, 1)
+        t1 += oracle_time_step(o, s, 0, k1, hidden_last, token_last, target, T)
+        rows1 += k1 + 1
+    oracle.set_threads(cores)
+    one = {"value": rows1 / (t1 * B * R), "unit": "steps/s", "cores": 1,
+           "sample": f"{rows1} rows of sequence 0, {t1:.1f} s, scaled by rows to a full step"}
+    return {"value": 1.0 / est_step, "unit": "steps/s", "cores": cores,
+            "kind": "oracle", "sample": sample, "one_thread": one}
 
 
 def run_reference(args):
     """--impl reference: the CPU checker timed on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    import numpy as np
-
     import oracle
     import synth
 
@@ -318,7 +304,7 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(s, B, lens),
+        "config": workload_config(s, B, lens, args.temperature),
         "cpu_baseline": {"value": value, "unit": "steps/s", "cores": oracle.num_threads(),
                          "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -337,14 +323,243 @@ def workload_shape(args):
     return s
 
 
-def workload_config(s, B, lens):
+def workload_config(s, B, lens, T):
+    drafts = ("drafts drawn from q in the LM head (lossless round)" if T > 0 else "arg-max drafts, greedy verify")
     return {
         "workload": f"{s.name}: H{s.hidden} heads{s.n_heads}x{s.head_dim} F{s.ffn} V{s.vocab} "
                     f"B{B} k{s.k_masks} ctx{int(min(lens))}-{int(max(lens))} "
                     f"{'fp32' if s.dtype == 0 else 'bf16'}",
         "batch": B, "k_masks": s.k_masks, "rows_per_step": B * s.rows,
-        "verify": "n_draft=n_target=k+1, draft logits stored, Zipf(1.1)-biased target logits",
+        "verify": f"n_draft=n_target=k+1, draft logits stored, Zipf(1.1)-biased target logits, T={T:g}, {drafts}",
     }
+
+
+# ---- one workload resident on the GPU ------------------------------------------------------------
+class Workload:
+    """A drafter with its KV caches and the step's inputs resident in HBM.  The weights exceed L2
+    and are streamed every step; the KV caches rotate over enough distinct sets (and the target
+    logits over four buffers) that consecutive steps never find them in L2."""
+
+    def __init__(self, s, flags=0, extra_ctx=0, weights=None):
+        import numpy as np  # noqa: F401
+
+        import paper_2410_05589_b200 as ps
+        import synth
+
+        self.ps, self.s = ps, s
+        B, R, V = s.batch, s.rows, s.vocab
+        self.B, self.R = B, R
+        self.lens = synth.ctx_lengths(s, B)
+        W = weights if weights is not None else synth.weights(s)
+        kv_bytes_seq = 2 * s.n_kv_heads * s.head_dim * int(self.lens.mean()) * (4 if s.dtype == 0 else 2)
+        n_sets = 1 if kv_bytes_seq * B > 2 * L2_BYTES else max(2, min(16, -(-2 * L2_BYTES // max(1, kv_bytes_seq * B))))
+        self.n_sets = n_sets = max(1, min(n_sets, 128 // B))
+        self.max_ctx = int(self.lens.max()) + R + extra_ctx
+        self.g = ps.drafter_from_shape(s, W, max_batch=B * n_sets, max_ctx=self.max_ctx, flags=flags)
+        for b in range(B):
+            K, Vv = synth.kv_rows(s, ("kv", b), int(self.lens[b]))
+            Kd, Vd = ps.to_device(K), ps.to_device(Vv)
+            for i in range(n_sets):
+                self.g.kv_import(i * B + b, Kd, Vd)
+        self.hl_np, self.tl_np = synth.hidden_states(s, "last", B), synth.token_ids(s, "last", B)
+        self.tgt_np = [(synth.zipf_logits(s.seed, f"tgt{i}", B, R, V) if s.logits_kind == "zipf"
+                        else synth.gauss_logits(s.seed, f"tgt{i}", (B, R, V))) for i in range(min(max(n_sets, 2), 4))]
+        self.hl, self.tl = ps.to_device(self.hl_np), ps.to_device(self.tl_np)
+        self.tgt = [ps.to_device(t) for t in self.tgt_np]
+        self.slots = [[i * B + b for b in range(B)] for i in range(n_sets)]
+        self.d_out, self.v_out = {}, {}
+
+    def step(self, i, T):
+        g, B, R = self.g, self.B, self.R
+        if T > 0:
+            o = g.draft_step_sampled(self.slots[i % self.n_sets], self.hl, self.tl, T, 1, i, top_n=1,
+                                     want_logits=True, out=self.d_out)
+            g.verify(o["sampled"], o["logits"], self.tgt[i % len(self.tgt)], T, 1, i, out=self.v_out)
+        else:
+            o = g.draft_step(self.slots[i % self.n_sets], self.hl, self.tl, top_n=1, want_logits=True, out=self.d_out)
+            g.verify(o["top_ids"].view(B, R), None, self.tgt[i % len(self.tgt)], 0.0, 1, i, out=self.v_out)
+
+    def timed(self, steps, T, warmup=5):
+        """Milliseconds of `steps` back-to-back steps (CUDA events on the launching stream)."""
+        import torch
+        for i in range(warmup):
+            self.step(i, T)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            self.step(i, T)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    def stage_profile(self, n, T, peak):
+        """Per-stage time per step (events recorded by the library between stages: no overlap
+        between consecutive kernels, so the stages add up to more than a timed step) and GB/s of
+        the stage's algorithmic bytes."""
+        import torch
+        self.g.profile(True)
+        for i in range(n):
+            self.step(i, T)
+        torch.cuda.synchronize()
+        prof = self.g.profile_read()
+        self.g.profile(False)
+        sb = stage_bytes(self.s, self.B, self.lens)
+        stages = {}
+        for name, (tot, cnt) in prof.items():
+            if cnt and name in sb:
+                us = tot / n * 1e3   # per step: a batch beyond 128 rows runs a stage several times a step
+                gbs = sb[name] / (us * 1e-6) / 1e9
+                stages[name] = {"us": round(us, 2), "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4),
+                                "launches_per_step": round(cnt / n, 2)}
+        return stages, sb
+
+    def summary(self, steps, T, peak, n_prof=40):
+        """ms per step, bytes, fractions of the roofline and the stage table of this workload."""
+        ms = self.timed(steps, T) / steps
+        stages, sb = self.stage_profile(n_prof, T, peak)
+        total = sum(sb.values())
+        gbs = total / (ms * 1e-3) / 1e9
+        return {"ms_per_step": round(ms, 5), "steps": steps, "temperature": T, "step_bytes": total,
+                "step_gbs": round(gbs, 1), "hbm_frac_of_measured": round(gbs / peak, 4),
+                "hbm_frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
+                "drafted_tokens_per_s": round(self.B * self.R / (ms * 1e-3), 1), "stages": stages}
+
+    def close(self):
+        import torch
+        self.g = None
+        self.tgt = self.hl = self.tl = None
+        self.d_out, self.v_out = {}, {}
+        torch.cuda.empty_cache()
+
+
+# A 26-node draft tree of the shape tree drafters use (4 children of the root, depth 6).
+TREE26 = [-1, -1, -1, -1, 0, 0, 0, 1, 1, 2, 4, 4, 5, 7, 10, 10, 11, 12, 13, 14, 14, 16, 18, 19, 21, 22]
+
+
+def tree_legs(w, T, peak, n_buf=6, reps=60):
+    """Token-tree round (Algorithm 1 in full).  (1) ps_verify_tree alone on the 26-node tree:
+    synthetic target rows per node, one draft row per depth (noisy copies, so that paths of several
+    nodes are accepted), node tokens drawn from the draft rows; buffers rotate so that rows come
+    from HBM.  (2) the whole round on the device: ps_draft_step (top-4) -> ps_build_tree ->
+    ps_verify_tree."""
+    import numpy as np
+    import torch
+
+    import synth
+    g, ps, s, B = w.g, w.ps, w.s, w.B
+    n = len(TREE26)
+    depth = []
+    for p in TREE26:
+        depth.append(0 if p < 0 else depth[p] + 1)
+    D, V = max(depth) + 1, s.vocab
+    sets = []
+    for i in range(n_buf):
+        tl = synth.gauss_logits(s.seed, ("tree_t", i), (B, n + 1, V))
+        dl = synth.noisy_draft_logits(s.seed, ("tree_d", i), np.repeat(tl[:, :1], D, axis=1), 0.6)
+        for j in range(n):
+            if depth[j] + 1 < D:
+                tl[:, 1 + j] = dl[:, depth[j] + 1] + 0.5 * tl[:, 1 + j]
+        toks = synth.sample_from_logits(s.seed, ("tree_x", i), dl[:, depth], temperature=max(T, 0.5))
+        sets.append((ps.to_device(toks.astype(np.int32)), ps.to_device(dl), ps.to_device(tl)))
+    out = {}
+    for i in range(5):
+        t_, d_, l_ = sets[i % n_buf]
+        g.verify_tree(TREE26, t_, d_, l_, T, 1, i, out=out)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        t_, d_, l_ = sets[i % n_buf]
+        g.verify_tree(TREE26, t_, d_, l_, T, 1, 100 + i, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / reps * 1e3
+    rows_with_children = len({p for p in TREE26})            # decision rows that read a draft row
+    nbytes = 4 * V * B * ((n + 1) + rows_with_children)
+    alone = {"us": round(us, 2), "nodes": n, "depth": D, "bytes": nbytes,
+             "gbs": round(nbytes / (us * 1e-6) / 1e9, 1), "frac_of_peak": round(nbytes / (us * 1e-6) / 1e9 / peak, 4),
+             "mean_accepted_nodes": float(out["accept_len"].float().mean().item()),
+             "note": "(n+1) target rows and one draft row per row with children, each read once"}
+    # the whole round on the device: the tree cut to the depths a draft step of k+1 rows gives
+    keep = [i for i in range(n) if depth[i] < s.rows]
+    renum = {old: new for new, old in enumerate(keep)}
+    tree = [renum.get(TREE26[i], -1) for i in keep]
+    rank = [sum(1 for j in range(i) if tree[j] == tree[i]) for i in range(len(tree))]
+    Dt, nt = min(D, s.rows), len(tree)
+    tgt_sets = [t[2][:, :nt + 1].contiguous() for t in sets]
+    d_out, tok_out, t_out = {}, torch.empty((B, nt), dtype=torch.int32, device="cuda"), {}
+
+    def tree_round(i):
+        o = g.draft_step(w.slots[i % w.n_sets], w.hl, w.tl, top_n=4, want_logits=True, out=d_out)
+        g.build_tree(tree, rank, o["top_ids"], out=tok_out)
+        dl = o["logits"] if Dt == s.rows else o["logits"][:, :Dt].contiguous()
+        g.verify_tree(tree, tok_out, dl, tgt_sets[i % n_buf], T, 1, i, out=t_out)
+
+    for i in range(5):
+        tree_round(i)
+    torch.cuda.synchronize()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for i in range(reps):
+        tree_round(i)
+    f1.record()
+    torch.cuda.synchronize()
+    whole = {"ms_per_round": round(f0.elapsed_time(f1) / reps, 5), "rounds": reps, "nodes": nt, "depth": Dt,
+             "note": "ps_draft_step (top-4) -> ps_build_tree -> ps_verify_tree, nothing on the host"}
+    return alone, whole
+
+
+def verify_alone_leg(w, T, peak, n_host=12, n_dev=144, reps=288):
+    """ps_verify on its own in the acceptance regime of the paper's tables: draft logits = target
+    + N(0, sigma^2) with sigma chosen for about 3.5 tokens a round at k = 4, drafts drawn from q on
+    the host.  The logits rotate over `n_dev` device buffers (more than L2 holds), so every call
+    reads its rows from HBM."""
+    import numpy as np
+    import torch
+
+    import synth
+    g, ps, s, B, R, V = w.g, w.ps, w.s, w.B, w.R, w.s.vocab
+    per_set = 2 * B * R * V * 4
+    n_dev = max(4, min(n_dev, int(1.5 * L2_BYTES // per_set) + 1, (2 << 30) // per_set))
+    host = []
+    for i in range(min(n_host, n_dev)):
+        tl = (synth.zipf_logits(s.seed, ("va_t", i), B, R, V) if s.logits_kind == "zipf"
+              else synth.gauss_logits(s.seed, ("va_t", i), (B, R, V)))
+        dl = synth.noisy_draft_logits(s.seed, ("va_d", i), tl, VERIFY_SIGMA)
+        tk = synth.sample_from_logits(s.seed, ("va_x", i), dl, temperature=T if T > 0 else 1.0)
+        if T == 0:
+            tk = dl.argmax(-1).astype(np.int32)
+        host.append((ps.to_device(tk.astype(np.int32)), ps.to_device(dl), ps.to_device(tl)))
+    dev = [(host[i % len(host)][0], host[i % len(host)][1].clone(), host[i % len(host)][2].clone())
+           for i in range(n_dev)]
+    out = {}
+    for i in range(8):
+        tk, dl, tl = dev[i % n_dev]
+        g.verify(tk, dl if T > 0 else None, tl, T, 1, i, out=out)
+    torch.cuda.synchronize()
+    n_out = 0.0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    acc = torch.zeros((), dtype=torch.float32, device="cuda")
+    e0.record()
+    for i in range(reps):
+        tk, dl, tl = dev[i % n_dev]
+        g.verify(tk, dl if T > 0 else None, tl, T, 1, 1000 + i, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / reps * 1e3
+    for i in range(min(reps, 4 * len(host))):     # acceptance statistics (untimed)
+        tk, dl, tl = dev[i % n_dev]
+        g.verify(tk, dl if T > 0 else None, tl, T, 1, 5000 + i, out=out)
+        acc += out["n_out"].float().mean()
+        n_out += 1
+    torch.cuda.synchronize()
+    nbytes = (8 if T > 0 else 4) * B * R * V
+    return {"us": round(us, 2), "bytes": nbytes, "gbs": round(nbytes / (us * 1e-6) / 1e9, 1),
+            "frac_of_peak": round(nbytes / (us * 1e-6) / 1e9 / peak, 4),
+            "mean_tokens_per_round": round(float(acc.item()) / n_out, 3), "sigma": VERIFY_SIGMA,
+            "buffers": n_dev, "buffer_bytes_total": n_dev * per_set, "temperature": T,
+            "note": "ps_verify alone, n_draft = n_target = k+1, logits read from HBM (buffers rotate over more than L2)"}
 
 
 def main():
@@ -368,36 +583,17 @@ def main():
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peak, peak_kind = measured_peak()
 
     s = workload_shape(args)
-    B, R, V, T = s.batch, s.rows, s.vocab, args.temperature
-    lens = synth.ctx_lengths(s, B)
-    W = synth.weights(s)
-    kv_bytes_seq = 2 * s.n_kv_heads * s.head_dim * int(lens.mean()) * (4 if s.dtype == 0 else 2)
-    # rotate over enough distinct KV sets that consecutive steps never find their KV in L2
-    n_sets = 1 if kv_bytes_seq * B > 2 * L2_BYTES else max(2, min(16, -(-2 * L2_BYTES // max(1, kv_bytes_seq * B))))
-    n_sets = min(n_sets, 128 // B)
-    max_ctx_bench = int(lens.max()) + R + 64        # + room for the groups of the training-layout leg
-    g = ps.drafter_from_shape(s, W, max_batch=B * n_sets, max_ctx=max_ctx_bench)
-    del W
-    for i in range(n_sets):
-        for b in range(B):
-            K, Vv = synth.kv_rows(s, ("kv", b), int(lens[b]))
-            g.kv_import(i * B + b, ps.to_device(K), ps.to_device(Vv))
-    hl_np, tl_np = synth.hidden_states(s, "last", B), synth.token_ids(s, "last", B)
-    tgt_np = [(synth.zipf_logits(s.seed, f"tgt{i}", B, R, V) if s.logits_kind == "zipf"
-               else synth.gauss_logits(s.seed, f"tgt{i}", (B, R, V))) for i in range(min(n_sets, 4))]
-    hl, tl = ps.to_device(hl_np), ps.to_device(tl_np)
-    tgt = [ps.to_device(t) for t in tgt_np]
-    slots = [[i * B + b for b in range(B)] for i in range(n_sets)]
-    d_out, v_out = {}, {}
+    T = args.temperature
+    w = Workload(s, flags=args.flags, extra_ctx=64)   # + room for the groups of the training-layout leg
+    g, B, R, V = w.g, w.B, w.R, s.vocab
+    lens = w.lens
 
-    def step(i):
-        o = g.draft_step(slots[i % n_sets], hl, tl, top_n=1, want_logits=True, out=d_out)
-        g.verify(o["top_ids"].view(B, R), o["logits"], tgt[i % len(tgt)], T, 1, i, out=v_out)
-
+    # ---- headline: K timed steps after W warm-up steps, barrier + synchronize on both sides -----
     for i in range(max(3, args.warmup)):
-        step(i)
+        w.step(i, T)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
@@ -408,7 +604,7 @@ def main():
     torch.cuda.synchronize()
     e0.record()
     for i in range(args.steps):
-        step(i)
+        w.step(i, T)
     e1.record()
     torch.cuda.synchronize()
     launches = g.launch_count() - l0
@@ -417,108 +613,116 @@ def main():
         dist.barrier()
     ms = max_over_ranks(e0.elapsed_time(e1))
     assert g.poll() == 0, "device status word set during the timed region"
-    n_accept = float(v_out["n_out"].float().mean().item())
+    n_accept = float(w.v_out["n_out"].float().mean().item())
 
-    # ---- per-stage times (CUDA events recorded by the library between stages) -------------
-    g.profile(True)
-    n_prof = min(args.steps, 200)
-    for i in range(n_prof):
-        step(i)
-    torch.cuda.synchronize()
-    prof = g.profile_read()
-    g.profile(False)
-    sb = stage_bytes(s, B, lens)
-    peak, peak_kind = measured_peak()
-    stages = {}
-    for name, (tot, cnt) in prof.items():
-        if cnt and name in sb:
-            # per step, not per launch: a batch beyond 128 rows runs a stage several times a step
-            us = tot / n_prof * 1e3
-            stages[name] = {"us": round(us, 2), "gbs": round(sb[name] / (us * 1e-6) / 1e9, 1),
-                            "launches_per_step": round(cnt / n_prof, 2)}
+    # ---- steady state: the same step for at least a second, clocks sampled meanwhile ------------
+    per = ms / args.steps
+    n_steady = int(min(20000, max(args.steps, 1100.0 / max(per, 1e-3))))
+    sampler2 = ClockSampler(local)
+    sampler2.start()
+    ms_steady = w.timed(n_steady, T, warmup=3)
+    steady = {"ms_per_step": round(ms_steady / n_steady, 5), "steps": n_steady, "seconds": round(ms_steady * 1e-3, 3),
+              "clocks": sampler2.stop()}
+
+    # ---- per-stage times and the roofline of the slowest stage's kernel -------------------------
+    n_prof = min(max(args.steps, 20), 200)
+    stages, sb = w.stage_profile(n_prof, T, peak)
     dom = max(stages, key=lambda k: stages[k]["us"]) if stages else None
     step_bytes = sum(sb.values())
     roofline = None
     if dom:
+        per_launch_us = stages[dom]["us"] / max(stages[dom]["launches_per_step"], 1.0)
         roofline = {
             "bound": "hbm", "kernel": kernel_of_stage(dom, B * R), "stage": dom,
-            "achieved": stages[dom]["gbs"], "peak": peak,
-            "unit": "GB/s", "frac": round(stages[dom]["gbs"] / peak, 4),
-            "traffic": NCU_DRAM_BYTES.get((args.workload, B, s.k_masks, dom)),
-            "peak_kind": f"of {peak_kind}", "bytes_per_launch": sb[dom],
+            "achieved": stages[dom]["gbs"], "peak": peak, "unit": "GB/s",
+            "frac": round(stages[dom]["gbs"] / peak, 4),
+            "traffic": captured_dram_bytes(args.workload, B, s.k_masks, dom),
+            "peak_kind": f"of {peak_kind}", "bytes_per_launch": sb[dom], "us_per_launch": round(per_launch_us, 2),
+            "note": "dominant stage's kernel, events between stages; the step-level fractions are hbm_frac_of_*",
         }
 
-    # ---- the same step with the drafts sampled in the LM head (lossless at T > 0) -------------
-    sampled = None
+    # ---- the other temperature of the headline workload (Table 1 has T = 0 and T = 1) -----------
+    T_other = 0.0 if T > 0 else 1.0
+    n_o = min(args.steps, 300)
+    ms_o = w.timed(n_o, T_other) / n_o
+    other_T = {"temperature": T_other, "ms_per_step": round(ms_o, 5), "steps": n_o,
+               "step_gbs": round(step_bytes / (ms_o * 1e-3) / 1e9, 1),
+               "hbm_frac_of_measured": round(step_bytes / (ms_o * 1e-3) / 1e9 / peak, 4),
+               "note": "arg-max drafts + greedy verify" if T_other == 0 else "drafts drawn from q + stochastic verify"}
+    # arg-max drafts verified against the full q at T > 0: the faster but biased variant, for comparison
+    argmax_T = None
     if T > 0:
-        s_out = {}
+        a_out = {}
 
-        def step_sampled(i):
-            o = g.draft_step_sampled(slots[i % n_sets], hl, tl, T, 1, i, top_n=1, want_logits=True, out=s_out)
-            g.verify(o["sampled"], o["logits"], tgt[i % len(tgt)], T, 1, i, out=v_out)
+        def step_argmax(i):
+            o = g.draft_step(w.slots[i % w.n_sets], w.hl, w.tl, top_n=1, want_logits=True, out=a_out)
+            g.verify(o["top_ids"].view(B, R), o["logits"], w.tgt[i % len(w.tgt)], T, 1, i, out=w.v_out)
 
         for i in range(5):
-            step_sampled(i)
+            step_argmax(i)
         torch.cuda.synchronize()
-        n_s = min(args.steps, 300)
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record()
-        for i in range(n_s):
-            step_sampled(i)
+        for i in range(n_o):
+            step_argmax(i)
         f1.record()
         torch.cuda.synchronize()
-        sampled = {"ms_per_step": f0.elapsed_time(f1) / n_s, "steps": n_s,
-                   "note": "ps_draft_step_sampled (Gumbel-max in the LM-head epilogue) + ps_verify"}
+        argmax_T = {"ms_per_step": round(f0.elapsed_time(f1) / n_o, 5), "steps": n_o,
+                    "note": "ps_draft_step (arg-max drafts) + ps_verify with the full draft distribution: not lossless at T > 0"}
 
-    # ---- group-wise training layout, forward only (Sec. 4.1): groups on the last KV set ---------
+    # ---- verify alone in the paper's acceptance regime ------------------------------------------
+    verify_alone = verify_alone_leg(w, T, peak) if s.vocab >= 1000 else None
+
+    # ---- group-wise training layout, forward only (Sec. 4.1): groups on the first KV set --------
     group = None
-    if int(lens.max()) + 64 + s.k_masks <= max_ctx_bench:
+    if int(lens.max()) + 64 + s.k_masks <= w.max_ctx:
         n_g = 64
         gh = ps.to_device(synth.hidden_states(s, "grp", n_g))
         gt = ps.to_device(synth.token_ids(s, "grp", n_g))
         for i in range(2):
-            g.group_forward(int(slots[0][0]), gh, gt, top_n=1, want_logits=False)
+            g.group_forward(int(w.slots[0][0]), gh, gt, top_n=1, want_logits=False)
         torch.cuda.synchronize()
         h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         h0.record()
         for i in range(5):
-            g.group_forward(int(slots[0][0]), gh, gt, top_n=1, want_logits=False)
+            g.group_forward(int(w.slots[0][0]), gh, gt, top_n=1, want_logits=False)
         h1.record()
         torch.cuda.synchronize()
         group = {"ms_per_call": h0.elapsed_time(h1) / 5, "groups": n_g, "rows": n_g * R,
                  "note": "ps_group_forward; the groups run as draft steps of up to 128 rows per launch"}
 
-    # ---- token-tree verification (Algorithm 1 in full), timed on its own ---------------------
-    tree = None
-    if V % 4 == 0 and V <= 131072 and s.dtype == 1:
-        tree = tree_verify_leg(g, ps, s, B, T, peak)
+    # ---- token-tree verification (Algorithm 1 in full) and the whole tree round -----------------
+    tree, tree_round = (None, None)
+    if V % 4 == 0 and V <= 131072 and s.dtype == 1 and s.k_masks >= 1:
+        tree, tree_round = tree_legs(w, T, peak)
 
-    # ---- end to end through the host-buffer entry point -----------------------------------
-    hl_h = torch.from_numpy(hl_np.view(np.int16) if hl_np.dtype == np.uint16 else hl_np).pin_memory()
-    tl_h = torch.from_numpy(tl_np).pin_memory()
-    tgt_h = [torch.from_numpy(t).pin_memory() for t in tgt_np]
+    # ---- end to end through the host-buffer entry point -----------------------------------------
+    hl_h = torch.from_numpy(w.hl_np.view(np.int16) if w.hl_np.dtype == np.uint16 else w.hl_np).pin_memory()
+    tl_h = torch.from_numpy(w.tl_np).pin_memory()
+    tgt_h = [torch.from_numpy(t).pin_memory() for t in w.tgt_np]
     r_out = {}
     n_e2e = min(args.steps, 500)
     for i in range(3):
-        g.round_host(slots[i % n_sets], hl_h, tl_h, tgt_h[i % len(tgt_h)], T, 1, i, out=r_out)
+        g.round_host(w.slots[i % w.n_sets], hl_h, tl_h, tgt_h[i % len(tgt_h)], T, 1, i, out=r_out)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     t0 = time.perf_counter()
     for i in range(n_e2e):
-        g.round_host(slots[i % n_sets], hl_h, tl_h, tgt_h[i % len(tgt_h)], T, 1, i, out=r_out)
+        g.round_host(w.slots[i % w.n_sets], hl_h, tl_h, tgt_h[i % len(tgt_h)], T, 1, i, out=r_out)
     torch.cuda.synchronize()
     e2e_s = max_over_ranks(time.perf_counter() - t0)
     eb = 4 if s.dtype == 0 else 2
     e2e = {"value": aggregate_steps_per_s(world, n_e2e, e2e_s * 1e3), "unit": "steps/s",
            "h2d_bytes_per_step": B * s.hidden * eb + B * 4 + B * R * V * 4,
-           "d2h_bytes_per_step": B * (R + 3) * 4, "steps": n_e2e}
+           "d2h_bytes_per_step": B * (R + 3) * 4, "steps": n_e2e,
+           "note": "ps_round_host: pinned host inputs up, results down and a stream wait, every step"}
 
     # ---- ps_kv_append (once per round, off the draft step's path): 4 accepted pairs a sequence ----
     n_new = 4
     ka_h = ps.to_device(synth.hidden_states(s, "app", B * n_new))
     ka_t = ps.to_device(synth.token_ids(s, "app", B * n_new))
-    app_slots = slots[0]   # last leg on the device: these slots' contexts are not needed again
+    app_slots = w.slots[0]   # last leg on this context: these slots' contexts are not needed again
 
     def append_once():
         for x in app_slots:   # host bookkeeping only: the same cache rows are written every time
@@ -539,10 +743,32 @@ def main():
     kv_append = {"us": round(app_us, 2), "rows": B * n_new, "bytes": app_bytes,
                  "gbs": round(app_bytes / (app_us * 1e-6) / 1e9, 1),
                  "note": "fc + k|v weights read once, 4 new real positions per sequence"}
+    hl_np, tl_np, tgt0 = w.hl_np, w.tl_np, w.tgt_np[0]
+    w.close()
+
+    # ---- the other workloads: step time, roofline fractions and the stage table of each --------
+    configs = None
+    if rank == 0 and world == 1 and not args.no_configs and args.workload == "13b" and args.batch == 0 \
+            and args.k_masks < 0 and args.flags == 0:
+        configs = {}
+        n_c = min(max(args.steps, 20), 200)
+        for name in ("7b", "33b"):
+            wc = Workload(synth.CONFIGS[name])
+            configs[wc.s.name] = dict(wc.summary(n_c, T, peak), config=workload_config(wc.s, wc.B, wc.lens, T)["workload"])
+            wc.close()
+        W13 = synth.weights(synth.CONFIGS["13b_sweep"])
+        for Bc, kc in ((1, 2), (16, 4), (64, 8)):
+            sc = synth.CONFIGS["13b_sweep"].with_(batch=Bc, k_masks=kc)
+            Wc = dict(W13, mask_embed=W13["mask_embed"][:kc], mask_feat=W13["mask_feat"][:kc])
+            wc = Workload(sc, weights=Wc)
+            configs[f"13b_sweep_B{Bc}_k{kc}"] = dict(wc.summary(max(20, n_c // (1 + Bc // 8)), T, peak),
+                                                   config=workload_config(sc, Bc, wc.lens, T)["workload"])
+            wc.close()
+        del W13
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_baseline(s, B, lens, hl_np, tl_np, tgt_np[0], T, args.cpu_seconds)
+        cpu = cpu_baseline(s, B, lens, hl_np, tl_np, tgt0, T, args.cpu_seconds)
 
     if rank == 0:
         ms_per_step = ms / args.steps
@@ -553,17 +779,20 @@ def main():
             "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if s.dtype == 0 else "bf16", "data": "synthetic",
-            "config": dict(workload_config(s, B, lens),
+            "config": dict(workload_config(s, B, lens, T),
                            l2="weights exceed L2 and are streamed every step; KV caches rotate over "
-                              f"{n_sets} distinct sets, target logits over {len(tgt)} buffers",
-                           parallelism="replicas" if world > 1 else "single GPU"),
+                              f"{w.n_sets} distinct sets, target logits over {len(w.tgt_np)} buffers",
+                           parallelism="replicas" if world > 1 else "single GPU", flags=args.flags),
             "drafted_tokens_per_s": value * B * R,
             "step_bytes": step_bytes, "step_gbs": round(gbs, 1),
             "hbm_frac_of_measured": round(gbs / peak, 4),
             "hbm_frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
             "mean_tokens_per_round": n_accept,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "stages": stages, "sampled_drafts": sampled, "group_forward": group, "tree_verify": tree, "kv_append": kv_append, "cpu_baseline": cpu,
+            "roofline": roofline, "stages": stages, "steady": steady, "other_temperature": other_T,
+            "argmax_drafts": argmax_T, "verify_alone": verify_alone, "group_forward": group,
+            "tree_verify": tree, "tree_round": tree_round, "kv_append": kv_append, "configs": configs,
+            "cpu_baseline": cpu,
         }
         print(json.dumps(line))
     if world > 1:

@@ -292,6 +292,13 @@ ps_status ps_poll(ps_ctx* ctx, void* stream);
  * exist only on the fused bf16 path.  PS_ERR_INVALID_ARG for an unknown name. */
 ps_status ps_debug_buffer(ps_ctx* ctx, const char* name, void** ptr, size_t* bytes);
 
+/* Test helper for the error path of bounded device-side waits.  Every wait of the kernels on a
+ * copy or on tensor-core work gives up after about a second, raises the device status word
+ * and lets the kernel return, so that a lost completion is an error code, not a hung GPU.  This
+ * call enqueues a one-thread kernel that waits, with a limit of `limit_cycles` clock cycles
+ * (at most 4e9), on a barrier nothing completes; ps_poll then returns PS_ERR_TIMEOUT. */
+ps_status ps_debug_wait_expires(ps_ctx* ctx, long long limit_cycles, void* stream);
+
 /* Number of kernel launches the context has enqueued so far (host counter). */
 long long ps_launch_count(ps_ctx* ctx);
 

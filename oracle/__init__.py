@@ -12,6 +12,7 @@ from .ps_oracle import (  # noqa: F401
     num_threads,
     philox4x32,
     row_stats,
+    set_threads,
     uniforms,
     verify,
     verify_tree,

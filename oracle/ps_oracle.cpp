@@ -271,6 +271,15 @@ int pso_num_threads() {
 #endif
 }
 
+// Sets the number of threads the row loops use from now on (timing on one core and on all).
+void pso_set_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
 void* pso_create(const Config* cfg, const Weights* w) {
   Ctx* C = new Ctx();
   C->c = *cfg;

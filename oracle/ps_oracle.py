@@ -214,6 +214,11 @@ def num_threads() -> int:
     return _load().pso_num_threads()
 
 
+def set_threads(n: int) -> None:
+    """Number of OpenMP threads the oracle's row loops use from now on."""
+    _load().pso_set_threads(int(n))
+
+
 def row_stats(logits: np.ndarray, top_n: int):
     logits = np.ascontiguousarray(logits, dtype=np.float64)
     n, V = logits.shape

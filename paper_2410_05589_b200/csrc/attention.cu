@@ -373,7 +373,9 @@ static ps_status launch_attn_t(ps_ctx* c, const SeqMap& sm, int B, int max_len, 
   // the largest tile whose grid, one tile per block, is resident at once; else full tiles and
   // several of them per block
   auto kern = k_attn_mma<D, NB>;
-  static int blocks_per_sm[kTileMax / 16 + 1];   // per tile size, asked once (0 = not yet)
+  // resident blocks per SM by tile size, asked of this context's device once (0 = not yet)
+  int* blocks_per_sm = c->attn_blocks_per_sm[(D == 128 ? 0 : 2) + (NB == 1 ? 0 : 1)];
+  static_assert(kTileMax / 16 + 1 <= 16, "cache row covers every tile size");
   // the partial buffers hold 16 rows x kAttnMaxSplit splits: more rows, fewer splits
   const int M_rows = B * (g.k_masks + 1);
   const int max_split = std::max(1, std::min(kAttnMaxSplit, 16 * kAttnMaxSplit / std::max(M_rows, 1)));

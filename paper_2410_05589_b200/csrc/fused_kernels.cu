@@ -1180,6 +1180,20 @@ __global__ void __launch_bounds__(256) k_embed_x0(const __nv_bfloat16* __restric
   }
 }
 
+// The bounded wait of the GEMM kernels on a barrier that nothing ever completes: what a lost
+// copy would look like to them.  The wait gives up after `limit` cycles, the kernel raises the
+// status word as they do and returns normally.
+__global__ void k_wait_expires(long long limit, int* status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait(&bar, 0, &abort_flag, limit)) atomicOr(status, kStatTimeout);
+  }
+}
+
 // ---- host side: tensor maps ---------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1499,6 +1513,12 @@ ps_status fused_kv_append(ps_ctx* c, const SeqMap& sm, int rows, const void* hid
 }
 
 size_t fused_scratch_bytes(const ps_config& g) { return carve_fused(g, nullptr).bytes; }
+
+ps_status launch_wait_expires(ps_ctx* c, long long limit_cycles, cudaStream_t st) {
+  k_wait_expires<<<1, 32, 0, st>>>(limit_cycles, c->dev_status);
+  c->launches++;
+  return cuda_check(c, cudaGetLastError(), "k_wait_expires");
+}
 
 void fused_release(ps_ctx* c) {
   delete static_cast<UmmaMaps*>(c->umma_maps);

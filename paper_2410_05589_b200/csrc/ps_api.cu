@@ -242,6 +242,11 @@ ps_status ps_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* bytes
   return fused_debug_buffer(c, name, ptr, bytes);
 }
 
+ps_status ps_debug_wait_expires(ps_ctx* c, long long limit_cycles, void* stream) {
+  if (!c || limit_cycles < 0 || limit_cycles > 4000000000LL) return PS_ERR_INVALID_ARG;
+  return launch_wait_expires(c, limit_cycles, (cudaStream_t)stream);
+}
+
 ps_status ps_kv_len(ps_ctx* c, int slot, int* len) {
   if (!c || !len || slot < 0 || slot >= c->cfg.max_batch) return PS_ERR_INVALID_ARG;
   *len = c->len[slot];

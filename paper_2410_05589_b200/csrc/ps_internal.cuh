@@ -134,6 +134,9 @@ struct ps_ctx {
   double* rope_inv_freq;    // [head_dim/2] base^(-2i/d), filled once at ps_init
   int n_sm;                 // multiprocessors of the context's device
   int smem_optin;           // opt-in shared memory per block
+  // answers asked of this context's device once (0 = not asked yet)
+  int cluster_ok[2][17] = {};     // [chain verify, tree verify][cluster size]: 1 yes, -1 no
+  int attn_blocks_per_sm[4][16] = {};   // [kernel variant][tile size / 16]: resident blocks, -1 none
   cudaStream_t copy_stream = nullptr;   // ps_round_host: carries the target logits beside the draft step
   cudaEvent_t copy_done = nullptr;
   void* st_hidden; int* st_tok; float* st_tlogits; float* st_dlogits; int* st_top; int* st_res;
@@ -179,6 +182,8 @@ size_t fused_scratch_bytes(const ps_config& g);
 void fused_release(ps_ctx* c);   // frees what the fused path holds on the host
 ps_status fused_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* bytes);
 ps_status launch_rope_table(ps_ctx* c, cudaStream_t st);
+// Test kernel: a bounded barrier wait that runs out after `limit_cycles` and raises the status word.
+ps_status launch_wait_expires(ps_ctx* c, long long limit_cycles, cudaStream_t st);
 ps_status launch_attn_split(ps_ctx* c, const SeqMap& sm, int B, const float* qkv, float* att_ml,
                             float* att_o, unsigned* tickets, __nv_bfloat16* out_hi,
                             __nv_bfloat16* out_lo, cudaStream_t st);

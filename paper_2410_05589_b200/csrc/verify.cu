@@ -961,14 +961,14 @@ cudaError_t launch_cluster(void (*kern)(Args), dim3 grid, int nclu, cudaStream_t
   return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
-// Whether the device can co-schedule nclu blocks of this kernel as one cluster (sizes above 8
-// are an opt-in of the kernel).  Asked once per size.
+// Whether the context's device can co-schedule nclu blocks of this kernel as one cluster (sizes
+// above 8 are an opt-in of the kernel, a per-device function attribute).  Asked once per context
+// and size; `cache` is the context's row for this kernel.
 template <class Args>
-bool cluster_size_ok(void (*kern)(Args), int nclu) {
-  static int ok[17] = {0};   // 0 unknown, 1 yes, -1 no
+bool cluster_size_ok(int* cache, void (*kern)(Args), int nclu) {
   if (nclu <= 8) return true;
-  if (ok[nclu] == 0) {
-    ok[nclu] = -1;
+  if (cache[nclu] == 0) {
+    cache[nclu] = -1;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3(nclu);
@@ -979,11 +979,11 @@ bool cluster_size_ok(void (*kern)(Args), int nclu) {
       cfg.attrs = at;
       cfg.numAttrs = 1;
       int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0) ok[nclu] = 1;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0) cache[nclu] = 1;
     }
     (void)cudaGetLastError();
   }
-  return ok[nclu] > 0;
+  return cache[nclu] > 0;
 }
 
 ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* draft_tokens,
@@ -1000,7 +1000,7 @@ ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* 
   a.rec = c->vrec; a.tickets = c->tickets; a.status = c->dev_status;
   const bool aligned = (((uintptr_t)target_logits | (uintptr_t)draft_logits) & 15u) == 0;
   const int nclu = a.V <= kCluMaxVocab ? kClu : 16;
-  if (a.V % 4 == 0 && a.V <= kCluMaxVocab16 && aligned && (nclu == kClu || cluster_size_ok(k_verify_cluster16, 16))) {
+  if (a.V % 4 == 0 && a.V <= kCluMaxVocab16 && aligned && (nclu == kClu || cluster_size_ok(c->cluster_ok[0], k_verify_cluster16, 16))) {
     prof_mark(c, st, "begin");
     // (a plain launch: joining the dependent-launch chain here was measured to cost 7 us a step)
     cudaError_t e;
@@ -1066,7 +1066,7 @@ ps_status launch_verify_tree(ps_ctx* c, int B, int n_nodes, const int* parent, c
   // blocks per decision row: 8 (16 for vocabularies beyond 65536), fewer when the tree would
   // otherwise need a second wave of blocks and a thread can still hold its share of a row
   int nclu = a.V <= kCluMaxVocab ? kClu : 16;
-  if (!cluster_size_ok(k_verify_tree, nclu))
+  if (!cluster_size_ok(c->cluster_ok[1], k_verify_tree, nclu))
     return fail(c, PS_ERR_UNSUPPORTED, "this device cannot run the 16-block clusters a vocabulary beyond 65536 needs");
   while (nclu > 1 && (long)(n_nodes + 1) * B * nclu > c->n_sm && a.V <= (nclu / 2) * kCluThreads * 4 * kCluV4)
     nclu /= 2;

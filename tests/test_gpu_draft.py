@@ -270,3 +270,17 @@ def test_group_wise_training_forward(name, n, max_batch):
     ref = p.oracle_step(0)
     assert logits_close(step["logits"][0].cpu().numpy(), ref["logits"], s.dtype) <= 1.0
     assert p.g.poll() == 0
+
+
+def test_bounded_device_wait_reports_timeout():
+    """Every device-side wait is bounded; when one runs out the kernel raises the status word and
+    returns.  A test kernel waits (2 ms at most) on a barrier nothing completes: ps_poll reports
+    PS_ERR_TIMEOUT once, the context keeps working."""
+    s = synth.CONFIGS["mini"]
+    p = Pair(s, 1, lens=[12])
+    before = p.gpu_step(top_n=1)
+    p.g.debug_wait_expires(4_000_000)
+    assert p.g.poll() == -5          # PS_ERR_TIMEOUT
+    assert p.g.poll() == 0
+    after = p.gpu_step(top_n=1)
+    assert np.array_equal(before["logits"], after["logits"])
