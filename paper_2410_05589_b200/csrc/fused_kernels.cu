@@ -737,6 +737,70 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
   }
 }
 
+// Epilogue of 16 activation rows [m0, m0 + mc) of a tile for launches of more than 16 rows
+// (EPI_STORE and EPI_SWIGLU): the thread of accumulator row r holds the rows' sums in v[] (no
+// detour through shared memory) and their residual values in rv[] (loaded by the caller before the
+// sums were ready).  With that many rows the epilogue runs eight times per tile and is what a
+// launch costs beyond its weight stream, so the per-row work is kept free of cross-lane steps:
+// the rows' sums of squares go through a [16][128] tile in shared memory (ctl.acc) and are added
+// by 8 threads per row, instead of a shuffle reduction per row and warp.
+template <int EPI>
+__device__ __forceinline__ void big_chunk_epilogue(const UArgs& a, umma::Ctl& ctl, int n, bool valid, int pidx, int r,
+                                                   int m0, int mc, const float (&v)[16], float bias, float gain,
+                                                   const float (&rv)[16], bool dry) {
+  using namespace umma;
+  constexpr int kSqLd = 132;   // row pitch of the squares' tile: the 8 x 4 threads of a warp read different banks
+  static_assert(16 * kSqLd <= 2 * kN * 128, "the squares' tile fits ctl.acc + ctl.land");
+  if (EPI == EPI_STORE) {
+    float sq[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      sq[j] = 0.f;
+      if (j < mc && valid) {
+        const float x = v[j] * ctl.scale[m0 + j] + bias + rv[j];
+        sq[j] = x * x;
+        if (!dry) {
+          a.out[(size_t)(m0 + j) * a.ldo + n] = x;
+          if (a.out_hi)
+            split_store(a.out_hi + (size_t)(m0 + j) * a.ld_plane + n, a.out_lo + (size_t)(m0 + j) * a.ld_plane + n, x * gain);
+        }
+      }
+    }
+    if (a.ssq_out) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) ctl.acc[j * kSqLd + r] = sq[j];   // (runs on into ctl.land, unused here)
+      epi_sync();
+      const int row = r >> 3, part = r & 7;   // 8 threads per row, every 8th feature each
+      float sum = 0.f;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) sum += ctl.acc[row * kSqLd + i * 8 + part];
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+      if (part == 0 && row < mc && !dry) a.ssq_out[(size_t)pidx * a.M + m0 + row] = sum;
+      epi_sync();
+    }
+  } else {   // EPI_SWIGLU: rows 0..63 of the tile are gate features, rows 64..127 the same features of up
+    if (r >= 64) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) ctl.xch[j * 64 + (r - 64)] = v[j] * ctl.scale[min(m0 + j, kMaxRows - 1)];
+    }
+    epi_sync();
+    if (r < 64 && valid && !dry) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        if (j < mc) {
+          const float gv = v[j] * ctl.scale[m0 + j], uv = ctl.xch[j * 64 + r];
+          const float act = gv / (1.f + __expf(-gv)) * uv;
+          if (a.out) a.out[(size_t)(m0 + j) * a.ldo + n] = act;
+          split_store(a.out_hi + (size_t)(m0 + j) * a.ld_plane + n, a.out_lo + (size_t)(m0 + j) * a.ld_plane + n, act);
+        }
+      }
+    }
+    epi_sync();
+  }
+}
+
 static_assert(umma::kMaxCtas >= kMaxSm, "contributor table covers every CTA of a launch");
 
 template <int EPI, int MP>
@@ -912,13 +976,24 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
       float* P = a.partials + ((size_t)blockIdx.x * 2 + slot) * kMaxRows * 128;
       bool finish = whole || dry;   // this CTA runs the tile's epilogue
       int c_first = blockIdx.x, c_last = blockIdx.x;
+      // (launches of more than 16 rows keep a partial as [accumulator row][activation row]: a
+      // thread writes and reads its 16 rows of a chunk as four 16-byte vectors)
+      constexpr bool kBig = MP > 16 && EPI != EPI_LMHEAD;
       if (!whole && !dry) {
         for (int m0 = 0; m0 < a.M; m0 += 16) {
           float v[16];
           load_chunk(m0, v);
+          if (kBig) {
+            float4* d4 = reinterpret_cast<float4*>(P + (size_t)r * kMaxRows + m0);
+            d4[0] = make_float4(v[0], v[1], v[2], v[3]);
+            d4[1] = make_float4(v[4], v[5], v[6], v[7]);
+            d4[2] = make_float4(v[8], v[9], v[10], v[11]);
+            d4[3] = make_float4(v[12], v[13], v[14], v[15]);
+          } else {
 #pragma unroll
-          for (int m = 0; m < 16; ++m)
-            if (m0 + m < a.M) P[(m0 + m) * 128 + r] = v[m];
+            for (int m = 0; m < 16; ++m)
+              if (m0 + m < a.M) P[(m0 + m) * 128 + r] = v[m];
+          }
         }
         fence_before_sync();
         mbar_arrive(&ctl.acc_empty[buf]);
@@ -952,7 +1027,54 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
         }
         epi_sync();
       }
-      if (finish) {
+      if (finish && kBig) {
+        // many rows: the sums stay in registers from tensor memory (or from the partials, added in
+        // CTA order with all of a contributor's vectors in flight together) to the stores
+        bool valid;
+        const int n = tile_feature(a, t, r, valid);
+        const float bias = (EPI == EPI_STORE && a.bias && valid) ? __bfloat162float(a.bias[n]) : 0.f;
+        const float gain = (EPI == EPI_STORE && a.gain_next && valid) ? __bfloat162float(a.gain_next[n]) : 1.f;
+        const int nc = c_last - c_first + 1;
+        const int m_end = dry ? min(a.M, 16) : a.M;   // the rehearsal takes one chunk
+        for (int m0 = 0; m0 < m_end; m0 += 16) {
+          const int mc = min(16, a.M - m0);
+          float rv[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            rv[j] = (EPI == EPI_STORE && a.res && valid && j < mc && !dry) ? __ldcg(a.res + (size_t)(m0 + j) * a.ldr + n) : 0.f;
+          float v[16];
+          if (whole) {
+            load_chunk(m0, v);
+            if (m0 + 16 >= a.M) {   // the accumulator is read: the MMA warp may reuse it
+              fence_before_sync();
+              mbar_arrive(&ctl.acc_empty[buf]);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = 0.f;
+            const float* Pr = a.partials + (size_t)r * kMaxRows + m0;
+#pragma unroll 1
+            for (int j0 = 0; j0 < nc; j0 += 2) {   // two contributors' vectors in flight at a time
+              const int o0 = ctl.coff[j0], o1 = j0 + 1 < nc ? ctl.coff[j0 + 1] : -1;
+              float4 x0[4], x1[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                x0[i] = o0 >= 0 ? __ldcg(reinterpret_cast<const float4*>(Pr + o0) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                x1[i] = o1 >= 0 ? __ldcg(reinterpret_cast<const float4*>(Pr + o1) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                v[4 * i] += x0[i].x; v[4 * i + 1] += x0[i].y; v[4 * i + 2] += x0[i].z; v[4 * i + 3] += x0[i].w;
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                v[4 * i] += x1[i].x; v[4 * i + 1] += x1[i].y; v[4 * i + 2] += x1[i].z; v[4 * i + 3] += x1[i].w;
+              }
+            }
+          }
+          big_chunk_epilogue<EPI>(a, ctl, n, valid, t, r, m0, mc, v, bias, gain, rv, dry);
+        }
+      } else if (finish) {
         // 16 activation rows at a time: the tile's sums into ctl.acc (from tensor memory, or the
         // partials added in CTA order, which does not depend on who came last), then the epilogue
         const int m_end = dry ? min(a.M, 16) : a.M;   // the rehearsal takes one chunk
@@ -1269,12 +1391,14 @@ UmmaMaps* build_maps(const ps_ctx* c, const FusedScratch& f) {
 // Blocks per tile (UArgs::split) for a launch of M rows on G CTAs.  Up to 16 rows single units
 // are dealt (split = KB).  Beyond, a tile shared between CTAs costs more the more rows there
 // are (its partial sums come back 16 rows x one contributor at a time), so a model of the
-// slowest CTA picks the split.  Its constants are measured on a B200 with 30 to 125 rows: 0.3 us
-// per unit, 7 us of epilogue per 16 rows of a finished tile, 2 us per contributor and 16 rows
-// of a shared tile plus 1 us per 16 rows to publish a partial.
+// slowest CTA picks the split.  Its constants are fitted on a B200 with 80 to 144 rows: 0.3 us
+// per unit, 2 us of epilogue per 16 rows of a finished tile, 1 us per contributor and 16 rows
+// of a shared tile plus 0.5 us per 16 rows to publish a partial.  (At these row counts a unit
+// brings 32 KB of activation planes from L2 beside its 16 KB of weights, and the launches are
+// bound by that traffic rather than by HBM: the split moves their time by a tenth at most.)
 static int choose_split(int M, int Mp, int n_tiles, int KB, int G) {
   if (Mp <= 16) return KB;
-  const double t_unit = 0.3, t_epi = 7.0, t_trip = 2.0, t_part = 1.0;   // microseconds
+  const double t_unit = 0.3, t_epi = 2.0, t_trip = 1.0, t_part = 0.5;   // microseconds
   const int chunks = (M + 15) / 16, finished = (n_tiles + G - 1) / G;
   int best = 1;
   double best_cost = 1e30;

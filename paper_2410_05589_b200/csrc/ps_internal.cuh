@@ -89,8 +89,14 @@ struct SampleArgs {
 __device__ __forceinline__ float gumbel_noise(const SampleArgs& sa, uint32_t v, uint32_t row_id) {
   uint32_t c[4] = {v, row_id, sa.off_lo, sa.off_hi};
   philox4x32_10(sa.key0, sa.key1, c);
-  const double u = ((double)(c[0] >> 8) + 0.5) * (1.0 / 16777216.0);
-  return (float)(-log(-log(u)));   // in double: u may sit within 2^-25 of 1
+  // e = -ln u in single precision without losing u's distance from 1 (u can sit within 2^-25
+  // of it): below one half from u itself, above from 1 - u = (2^24 - w - 0.5) / 2^24, which like
+  // w + 0.5 is exact in fp32 on its half of the range.
+  const uint32_t w = c[0] >> 8;
+  float e;
+  if (w < (1u << 23)) e = -__logf(((float)w + 0.5f) * (1.0f / 16777216.0f));
+  else e = -log1pf(-((float)(16777216u - w) - 0.5f) * (1.0f / 16777216.0f));
+  return -__logf(e);
 }
 
 // Device status word values (bit flags).
