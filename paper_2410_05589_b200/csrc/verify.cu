@@ -338,7 +338,10 @@ struct CluScratch {
 };
 
 // (NCLU blocks per cluster: 8; 16 for vocabularies beyond 65536; 4 for batches of several waves.)
-template <int NCLU>
+// (V4: 16-byte vectors a thread holds per row: 4, or 2 when the row fits in half as many -- the
+// loops over a thread's tokens are unrolled, and this kernel runs its code once per launch, so
+// what it is not asked to execute it should not have to fetch.)
+template <int NCLU, int V4>
 __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
   namespace cg = cooperative_groups;
   cg::cluster_group cl = cg::this_cluster();
@@ -353,20 +356,28 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
   const bool greedy = a.temperature == 0.f;
   const float* drow = (!bonus && !greedy && a.draft_logits)
                           ? a.draft_logits + ((size_t)b * a.n_draft + i) * V : nullptr;
-  const int x = bonus ? -1 : a.draft_tokens[(size_t)b * a.n_draft + i];
   const int nv4 = ((V + nclu * kCluThreads - 1) / (nclu * kCluThreads) + 3) / 4;
   const int C = nv4 * 4, v0 = (rank * kCluThreads + tid) * C;
 
-  float t[kCluV4 * 4], d[kCluV4 * 4];
+  // The target rows are an input of the call; the draft rows and the draft tokens may be what the
+  // kernel before this one in the stream (the draft step) wrote last.  Were this kernel launched
+  // as its dependent, it would ask for the target row first and wait for that kernel only then.
+  pdl_launch_dependents();
+  float t[V4 * 4], d[V4 * 4];
 #pragma unroll
-  for (int k = 0; k < kCluV4; ++k) {
+  for (int k = 0; k < V4; ++k) {
     const int v = v0 + 4 * k;   // V % 4 == 0: a vector lies inside the row or outside it
-    float4 tv = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY), dv = tv;
-    if (k < nv4 && v < V) {
-      tv = *reinterpret_cast<const float4*>(trow + v);
-      if (drow) dv = *reinterpret_cast<const float4*>(drow + v);
-    }
+    float4 tv = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    if (k < nv4 && v < V) tv = __ldcs(reinterpret_cast<const float4*>(trow + v));
     t[4 * k] = tv.x; t[4 * k + 1] = tv.y; t[4 * k + 2] = tv.z; t[4 * k + 3] = tv.w;
+  }
+  pdl_wait();
+  const int x = bonus ? -1 : a.draft_tokens[(size_t)b * a.n_draft + i];
+#pragma unroll
+  for (int k = 0; k < V4; ++k) {
+    const int v = v0 + 4 * k;
+    float4 dv = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    if (drow && k < nv4 && v < V) dv = *reinterpret_cast<const float4*>(drow + v);
     d[4 * k] = dv.x; d[4 * k + 1] = dv.y; d[4 * k + 2] = dv.z; d[4 * k + 3] = dv.w;
   }
 
@@ -374,7 +385,7 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
   float tm = -INFINITY, dm = -INFINITY;
   int ti = 0x7fffffff, bad = 0;
 #pragma unroll
-  for (int e = 0; e < kCluV4 * 4; ++e) {
+  for (int e = 0; e < V4 * 4; ++e) {
     const int v = v0 + e;
     if (e < C && v < V) {
       float xt = t[e];
@@ -434,7 +445,7 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
     const double inv_t = 1.0 / (double)a.temperature;
     double st = 0.0, sd = 0.0;
 #pragma unroll
-    for (int e = 0; e < kCluV4 * 4; ++e) {
+    for (int e = 0; e < V4 * 4; ++e) {
       const bool in = e < C && v0 + e < V;
       t[e] = in ? expf((float)(((double)t[e] - (double)tmax) * inv_t)) : 0.f;
       st += (double)t[e];
@@ -476,11 +487,11 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
       const float inv_st = (float)(1.0 / st), inv_sd = (float)(1.0 / sd);
       // attempt 0: residual max(0, p - q); attempt 1: p itself (extra row, or an empty residual)
       for (int attempt = bonus ? 1 : 0; attempt < 2 && token < 0; ++attempt) {
-        float w[kCluV4 * 4];
+        float w[V4 * 4];
         double mine = 0.0;
         int lastp = -1;
 #pragma unroll
-        for (int e = 0; e < kCluV4 * 4; ++e) {
+        for (int e = 0; e < V4 * 4; ++e) {
           const float p = t[e] * inv_st;
           float wv = p;
           if (attempt == 0) {
@@ -541,7 +552,7 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
                   double run4 = 0.0;
                   int pick = -1, lp = -1;
 #pragma unroll
-                  for (int e = 0; e < kCluV4 * 4; ++e) {
+                  for (int e = 0; e < V4 * 4; ++e) {
                     if (w[e] > 0.f) lp = e;
                     run4 += (double)w[e];
                     if (pick < 0 && run4 > t4) pick = e;
@@ -572,17 +583,21 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
 
 // The 8-block cluster is fixed at compile time; the 16-block one (an opt-in size) is a launch attribute.
 __global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads) k_verify_cluster(VerifyArgs a) {
-  verify_cluster_body<kClu>(a);
+  verify_cluster_body<kClu, kCluV4>(a);
+}
+// (rows of up to 32768 tokens: 8 tokens per thread)
+__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kCluThreads) k_verify_cluster_v2(VerifyArgs a) {
+  verify_cluster_body<kClu, 2>(a);
 }
 __global__ void __launch_bounds__(kCluThreads) k_verify_cluster16(VerifyArgs a) {
-  verify_cluster_body<16>(a);
+  verify_cluster_body<16, kCluV4>(a);
 }
 // Four blocks per row pair: for batches whose 8-block clusters would not be resident at once
 // (one block fills an SM), while a thread can still hold its share of a row (16 tokens).
 constexpr int kCluSmall = 4;
 constexpr int kCluSmallMaxVocab = kCluSmall * kCluThreads * 4 * kCluV4;
 __global__ void __cluster_dims__(kCluSmall, 1, 1) __launch_bounds__(kCluThreads) k_verify_cluster4(VerifyArgs a) {
-  verify_cluster_body<kCluSmall>(a);
+  verify_cluster_body<kCluSmall, kCluV4>(a);
 }
 
 // ---- token-tree verification (Algorithm 1 in full) -------------------------------------------
@@ -1002,14 +1017,16 @@ ps_status launch_verify(ps_ctx* c, int B, int n_draft, int n_target, const int* 
   const int nclu = a.V <= kCluMaxVocab ? kClu : 16;
   if (a.V % 4 == 0 && a.V <= kCluMaxVocab16 && aligned && (nclu == kClu || cluster_size_ok(c->cluster_ok[0], k_verify_cluster16, 16))) {
     prof_mark(c, st, "begin");
-    // (a plain launch: joining the dependent-launch chain here was measured to cost 7 us a step)
     cudaError_t e;
-    if (nclu == kClu && a.V <= kCluSmallMaxVocab && n_target * B * kClu > c->n_sm) {
-      k_verify_cluster4<<<dim3(n_target * kCluSmall, B), kCluThreads, 0, st>>>(a);   // half the waves
-      e = cudaGetLastError();
+    // (plain launches: as dependents of the LM head these kernels start their loads earlier and
+    // run 3 us shorter alone, but the step gets 3 us longer -- measured twice: clusters of 8
+    // blocks that each fill an SM are slow to place while the LM head's CTAs drain)
+    const bool pdl = false;
+    if (nclu == kClu && a.V <= kCluSmallMaxVocab && n_target * B * kClu > c->n_sm) {   // half the waves
+      e = launch_after(k_verify_cluster4, dim3(n_target * kCluSmall, B), dim3(kCluThreads), 0, st, pdl, a);
     } else if (nclu == kClu) {
-      k_verify_cluster<<<dim3(n_target * kClu, B), kCluThreads, 0, st>>>(a);
-      e = cudaGetLastError();
+      e = launch_after(a.V <= kClu * kCluThreads * 4 * 2 ? k_verify_cluster_v2 : k_verify_cluster,
+                       dim3(n_target * kClu, B), dim3(kCluThreads), 0, st, pdl, a);
     } else {
       e = launch_cluster(k_verify_cluster16, dim3(n_target * 16, B), 16, st, a);
     }
