@@ -91,7 +91,7 @@ def check_top(ids, vals, want_logits, dtype):
             assert abs(want_logits[ids[t]] - w) <= 2 * tol(w), (t, ids[t], order[t])
 
 
-ACCEPT_BAND = 1e-6   # |r - min(1, p/q)| below which an acceptance decision may flip (spec exception)
+ACCEPT_BAND = 1e-6   # |r - min(1, p/q)| below which an acceptance decision may flip (the stated exception to bit-exactness)
 CDF_BAND = 1e-5      # distance of the sampling point to a CDF step (fraction of the total weight) below
                      # which the emitted token may be the neighbouring positive-weight token
 
