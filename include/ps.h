@@ -292,6 +292,12 @@ ps_status ps_poll(ps_ctx* ctx, void* stream);
  * exist only on the fused bf16 path.  PS_ERR_INVALID_ARG for an unknown name. */
 ps_status ps_debug_buffer(ps_ctx* ctx, const char* name, void** ptr, size_t* bytes);
 
+/* Test helper: every slice of the workspace (KV slabs, activation buffers, scratch) is followed by
+ * 256 bytes of guard words written at ps_init.  This call waits for `stream`, reads them back and
+ * counts the slices whose guard no longer holds its fill: a kernel that wrote past the end of one
+ * of its buffers.  n_bad: host int. */
+ps_status ps_debug_check_guards(ps_ctx* ctx, void* stream, int* n_bad);
+
 /* Test helper for the error path of bounded device-side waits.  Every wait of the kernels on a
  * copy or on tensor-core work gives up after about a second, raises the device status word
  * and lets the kernel return, so that a lost completion is an error code, not a hung GPU.  This

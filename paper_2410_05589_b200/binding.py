@@ -30,7 +30,7 @@ EXPORTS = (
     "ps_kv_len", "ps_kv_reset", "ps_kv_export", "ps_kv_import", "ps_poll", "ps_launch_count",
     "ps_last_error", "ps_destroy", "ps_philox_fill", "ps_profile", "ps_profile_read",
     "ps_verify_static", "ps_debug_buffer", "ps_verify_tree", "ps_draft_step_sampled", "ps_group_forward",
-    "ps_build_tree", "ps_debug_wait_expires",
+    "ps_build_tree", "ps_debug_wait_expires", "ps_debug_check_guards",
 )
 
 
@@ -82,6 +82,7 @@ def load_library(path: str | None = None) -> C.CDLL:
                                    vp, vp, vp, vp, vp]
     lib.ps_build_tree.argtypes = [vp, C.c_int, C.c_int, ip, ip, vp, C.c_int, vp, vp, vp]
     lib.ps_debug_wait_expires.argtypes = [vp, C.c_longlong, vp]
+    lib.ps_debug_check_guards.argtypes = [vp, vp, ip]
     lib.ps_kv_len.argtypes = [vp, C.c_int, ip]
     lib.ps_kv_reset.argtypes = [vp, C.c_int]
     lib.ps_kv_export.argtypes = [vp, C.c_int, vp, vp, vp]
@@ -369,6 +370,12 @@ class Drafter:
             float(temperature), seed, offset, hp(o["accept_len"]), hp(o["out_tokens"]),
             hp(o["n_out"]), _stream(stream)))
         return o
+
+    def check_guards(self, stream=None) -> int:
+        """ps_debug_check_guards: number of workspace slices whose guard words were overwritten."""
+        n = C.c_int(-1)
+        self._check(self.lib.ps_debug_check_guards(self.h, _stream(stream), C.byref(n)))
+        return n.value
 
     def debug_wait_expires(self, limit_cycles: int, stream=None) -> None:
         """ps_debug_wait_expires: a bounded device wait that runs out (sets the status word)."""

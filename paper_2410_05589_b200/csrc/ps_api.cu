@@ -54,9 +54,13 @@ ps_status check_config(const ps_config* g) {
 // Walks the workspace layout; with c == nullptr only the size is computed.
 size_t carve(const ps_config& g, ps_ctx* c, char* base) {
   size_t off = 0;
+  // every slice is followed by kGuardBytes of guard words (filled at ps_init, compared by
+  // ps_debug_check_guards): a kernel that writes past the end of its buffer shows up there
   auto take = [&](size_t bytes) {
     size_t at = off;
     off = align_up(off + bytes);
+    if (c) c->guards.push_back(off);
+    off += kGuardBytes;
     return base ? base + at : nullptr;
   };
   const size_t H = g.hidden, Hq = (size_t)g.n_heads * g.head_dim,
@@ -169,7 +173,10 @@ ps_status ps_init(ps_ctx** out, const ps_config* cfg, const ps_weights* w, void*
   }
   c->n_sm = std::min(prop.multiProcessorCount, kMaxSm);
   c->smem_optin = (int)prop.sharedMemPerBlockOptin;
-  cudaError_t e = cudaMemsetAsync(c->dev_status, 0, 256, st);
+  cudaError_t e = cudaSuccess;
+  for (size_t go : c->guards)
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + go, kGuardFill, kGuardBytes, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->dev_status, 0, 256, st);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(c->fused_scratch, 0, fused_scratch_bytes(*cfg), st);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->tickets, 0, sizeof(unsigned) * PS_MAX_BATCH, st);
@@ -240,6 +247,25 @@ ps_status ps_debug_buffer(ps_ctx* c, const char* name, void** ptr, size_t* bytes
   if (!std::strcmp(name, "x0")) { *ptr = c->x0; *bytes = Md * g.hidden * 4; return PS_OK; }
   if (!std::strcmp(name, "a")) { *ptr = c->a; *bytes = Md * g.hidden * 4; return PS_OK; }
   return fused_debug_buffer(c, name, ptr, bytes);
+}
+
+ps_status ps_debug_check_guards(ps_ctx* c, void* stream, int* n_bad) {
+  if (!c || !n_bad) return PS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  std::vector<unsigned char> host(c->guards.size() * kGuardBytes);
+  cudaError_t e = cudaSuccess;
+  for (size_t i = 0; i < c->guards.size() && e == cudaSuccess; ++i)
+    e = cudaMemcpyAsync(host.data() + i * kGuardBytes, c->ws + c->guards[i], kGuardBytes, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_check(c, e, "ps_debug_check_guards");
+  int bad = 0;
+  for (size_t i = 0; i < c->guards.size(); ++i) {
+    bool ok = true;
+    for (size_t j = 0; j < kGuardBytes; ++j) ok = ok && host[i * kGuardBytes + j] == (unsigned char)kGuardFill;
+    bad += !ok;
+  }
+  *n_bad = bad;
+  return PS_OK;
 }
 
 ps_status ps_debug_wait_expires(ps_ctx* c, long long limit_cycles, void* stream) {

@@ -17,6 +17,8 @@ constexpr int kMaxRowsPerSeq = PS_MAX_MASKS + 1;  // rows of one sequence in a d
 constexpr int kAppendChunk = 256;                 // rows handled per pass of ps_kv_append
 constexpr int kAttnMaxSplit = 32;                 // key-range splits of the fused attention
 constexpr int kMaxSm = 192;                       // bound used to size per-CTA scratch
+constexpr size_t kGuardBytes = 256;               // guard words behind every slice of the workspace
+constexpr int kGuardFill = 0x5A;
 
 // Which sequence each row of a launch belongs to.  Passed by value as a kernel parameter.
 // Row m (0-based within the launch) belongs to the sequence b with
@@ -147,6 +149,7 @@ struct ps_ctx {
   cudaEvent_t copy_done = nullptr;
   void* st_hidden; int* st_tok; float* st_tlogits; float* st_dlogits; int* st_top; int* st_res;
   std::vector<int> len;     // committed positions per slot (host is the source of truth)
+  std::vector<size_t> guards;   // offsets of the guard words in the workspace
   long long launches;
   std::string err;
   // optional stage timing (ps_profile): events recorded between stages

@@ -284,3 +284,30 @@ def test_bounded_device_wait_reports_timeout():
     assert p.g.poll() == 0
     after = p.gpu_step(top_n=1)
     assert np.array_equal(before["logits"], after["logits"])
+
+
+def test_workspace_guard_words_stay_intact():
+    """Every slice of the workspace is followed by guard words; after appends, draft steps on both
+    kernel sets' shapes, sampling, verify and the tree calls none of them has been touched.  The
+    detector itself is checked by overwriting one guard byte from the host side."""
+    import ctypes as C
+    import paper_2410_05589_b200 as ps
+    s = synth.CONFIGS["mini"]
+    p = Pair(s, 3, extra_ctx=8)
+    g = p.g
+    out = p.g.draft_step_sampled([0, 1, 2], p.to_device(p.hidden_last), p.to_device(p.token_last), 1.0, 3, 1, top_n=4)
+    tgt = ps.to_device(synth.gauss_logits(1, "gw", (3, s.rows, s.vocab)))
+    g.verify(out["sampled"], out["logits"], tgt, 1.0, 1, 0)
+    parent, rank = [-1, -1, 0, 0, 1], [0, 1, 0, 1, 0]
+    toks = g.build_tree(parent, rank, out["top_ids"])
+    g.verify_tree(parent, toks, out["logits"][:, :2].contiguous(), ps.to_device(synth.gauss_logits(1, "gt", (3, 6, s.vocab))), 1.0, 1, 0)
+    g.group_forward(0, p.to_device(synth.hidden_states(s, "grp", 3)), p.to_device(synth.token_ids(s, "grp", 3)), top_n=1)
+    assert g.check_guards() == 0
+    ptr, nbytes = C.c_void_p(), C.c_size_t()
+    assert g.lib.ps_debug_buffer(g.h, b"a", C.byref(ptr), C.byref(nbytes)) == 0
+    off = ptr.value - g.workspace.data_ptr() + ((nbytes.value + 255) // 256) * 256   # first guard byte behind "a"
+    g.workspace[off + 7] = 0
+    assert g.check_guards() == 1
+    g.workspace[off + 7] = 0x5A
+    assert g.check_guards() == 0
+    assert g.poll() == 0
