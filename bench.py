@@ -77,15 +77,18 @@ def kernel_of_stage(stage, rows):
     return KERNEL_OF_STAGE.get(stage, stage)
 
 
+GEMM_SOURCES = ("fused_kernels.cu", "umma_gemm.cuh", "ws_gemm.cuh", "ps_internal.cuh")
+
+
 def kernel_sources_digest():
-    """sha256 over the kernel sources: a counter capture is valid for the sources it was taken on."""
+    """sha256 over the sources of the GEMM kernels' translation unit: a counter capture is valid
+    for the sources it was taken on."""
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2410_05589_b200", "csrc")
-    for name in sorted(os.listdir(d)):
-        if name.endswith((".cu", ".cuh")):
-            with open(os.path.join(d, name), "rb") as f:
-                h.update(name.encode())
-                h.update(f.read())
+    for name in GEMM_SOURCES:
+        with open(os.path.join(d, name), "rb") as f:
+            h.update(name.encode())
+            h.update(f.read())
     return h.hexdigest()
 
 

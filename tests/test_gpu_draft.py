@@ -207,7 +207,7 @@ def _weights_13b_sweep():
     return _W13["w"]
 
 
-@pytest.mark.parametrize("B,k", [(4, 8), (16, 2), (64, 4), (64, 8)])
+@pytest.mark.parametrize("B,k", [(1, 2), (4, 8), (16, 2), (16, 4), (64, 4), (64, 8)])
 def test_13b_batch_sweep_sampled_sequences(B, k):
     """Points of the 13B-shaped batch / mask-count sweep at full size (ragged contexts of 256 to
     2048 positions, imported): every sequence runs on the GPU, the oracle recomputes three of
