@@ -264,7 +264,8 @@ ps_status ps_build_tree(ps_ctx* ctx, int B, int n_nodes, const int* parent, cons
  * the round then emits tokens that follow the target distribution (Eq. 1 holds for drafts drawn
  * from q, not for arg-max drafts with a full q).  All pointers except ctx are host memory; pinned
  * memory makes the copies asynchronous.  The target logits travel on a stream of the context's
- * own (created by the first call) while the draft step runs.
+ * own while the draft step runs, and the three results come back in one copy through a small
+ * pinned host buffer of the context (stream and buffer are created by the first call).
  *   hidden_last [B][H] config dtype, token_last [B], target_logits [B][k+1][V] float,
  *   accept_len [B], out_tokens [B][k+2], n_out [B]. */
 ps_status ps_round_host(ps_ctx* ctx, int B, const int* seq_slot, const void* hidden_last,

@@ -197,6 +197,7 @@ void ps_destroy(ps_ctx* c) {
     cudaEventDestroy(c->copy_done);
     cudaStreamDestroy(c->copy_stream);
   }
+  if (c->host_res) cudaFreeHost(c->host_res);
   delete c;
 }
 
@@ -558,6 +559,8 @@ ps_status ps_round_host(ps_ctx* c, int B, const int* seq_slot, const void* hidde
   if (!c->copy_stream) {
     e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->copy_done, cudaEventDisableTiming);
+    if (e == cudaSuccess)   // (pinned HOST memory for the results; no device memory is allocated)
+      e = cudaMallocHost((void**)&c->host_res, (size_t)g.max_batch * (g.k_masks + 4) * sizeof(int));
     if (e != cudaSuccess) return cuda_check(c, e, "ps_round_host copy stream");
   }
   e = cudaMemcpyAsync(c->st_tlogits, target_logits, (size_t)B * R * g.vocab * 4, cudaMemcpyHostToDevice,
@@ -588,11 +591,16 @@ ps_status ps_round_host(ps_ctx* c, int B, const int* seq_slot, const void* hidde
   s = ps_verify(c, B, R, R, c->st_top, c->st_dlogits, c->st_tlogits, temperature, seed, offset,
                 r_acc, r_out, r_n, st);
   if (s != PS_OK) return s;
-  e = cudaMemcpyAsync(accept_len, r_acc, (size_t)B * 4, cudaMemcpyDeviceToHost, st);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(n_out, r_n, (size_t)B * 4, cudaMemcpyDeviceToHost, st);
-  if (e == cudaSuccess)
-    e = cudaMemcpyAsync(out_tokens, r_out, (size_t)B * (R + 1) * 4, cudaMemcpyDeviceToHost, st);
+  // one copy back for the three results (they are adjacent in the staging slice), into pinned
+  // host memory of the context, then plain host copies into the caller's arrays
+  const size_t res_words = (size_t)B * (R + 3);
+  e = cudaMemcpyAsync(c->host_res, c->st_res, res_words * 4, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e == cudaSuccess) {
+    std::memcpy(accept_len, c->host_res, (size_t)B * 4);
+    std::memcpy(n_out, c->host_res + B, (size_t)B * 4);
+    std::memcpy(out_tokens, c->host_res + 2 * B, (size_t)B * (R + 1) * 4);
+  }
   return cuda_check(c, e, "ps_round_host d2h");
 }
 

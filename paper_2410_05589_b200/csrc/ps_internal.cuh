@@ -147,6 +147,7 @@ struct ps_ctx {
   int attn_blocks_per_sm[4][16] = {};   // [kernel variant][tile size / 16]: resident blocks, -1 none
   cudaStream_t copy_stream = nullptr;   // ps_round_host: carries the target logits beside the draft step
   cudaEvent_t copy_done = nullptr;
+  int* host_res = nullptr;              // ps_round_host: pinned host copy of the round's results
   void* st_hidden; int* st_tok; float* st_tlogits; float* st_dlogits; int* st_top; int* st_res;
   std::vector<int> len;     // committed positions per slot (host is the source of truth)
   std::vector<size_t> guards;   // offsets of the guard words in the workspace
