@@ -311,3 +311,13 @@ def test_workspace_guard_words_stay_intact():
     g.workspace[off + 7] = 0x5A
     assert g.check_guards() == 0
     assert g.poll() == 0
+
+
+@pytest.mark.parametrize("k,B", [(0, 1), (0, 5), (15, 1), (15, 3)])
+def test_mask_count_extremes(k, B):
+    """No [MASK] position at all (the step is an ordinary one-token drafter step) and the most the
+    library takes (15: 16 rows per sequence), one sequence and a ragged batch."""
+    s = synth.CONFIGS["mini"].with_(k_masks=k, batch=B, ctx_lo=0, ctx_hi=120)
+    p = Pair(s, B)
+    _compare_step(p, top_n=2)
+    assert p.g.poll() == 0

@@ -52,7 +52,7 @@ def test_device_philox_equals_oracle_words():
     assert [hex(x) for x in zero[0]] == ["0x6627e8d5", "0xe169c58d", "0xbc57ac4c", "0x9b00dbd8"]
 
 
-@pytest.mark.parametrize("V,n_draft,bonus", [(1000, 5, 0), (1000, 4, 1), (5003, 3, 1), (130, 1, 0),
+@pytest.mark.parametrize("V,n_draft,bonus", [(1000, 16, 0), (32000, 15, 1), (1000, 5, 0), (1000, 4, 1), (5003, 3, 1), (130, 1, 0),
                                             (32000, 4, 1), (65536, 2, 1), (8, 1, 1), (65540, 1, 1), (128256, 2, 1),
                                             (131070, 1, 1)])
 @pytest.mark.parametrize("T", [1.0, 0.6])
