@@ -465,7 +465,7 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
 // =============================================================================================
 struct UArgs {
   int N, K, M;
-  int Mp;                  // M padded to 16, 32, 64 or 128: rows of a plane box, half the MMA's N
+  int Mp;                  // M padded to 16, 32, 48, 64, 96 or 128: rows of a plane box, half the MMA's N
   int n_tiles, KB;         // tiles of 128 weight rows (64 features when zipped), k-blocks of 64
   int split;               // blocks a tile's k range is dealt in, 1..KB (see cta_begin)
   int zip;                 // 1: a tile is 64 rows of matrix 0 (gate) over 64 rows of matrix 1 (up)
@@ -1347,8 +1347,8 @@ bool make_map(CUtensorMap* m, const void* base, size_t rows, size_t cols, int bo
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct PlaneMaps {   // one activation plane with boxes of 16, 32, 64 and 128 rows
-  CUtensorMap m[4];
+struct PlaneMaps {   // one activation plane with boxes of every padded row count (umma::kRowPads)
+  CUtensorMap m[umma::kNumRowPads];
 };
 struct UmmaMaps {
   CUtensorMap w_fc, w_q, w_k, w_v, w_o, w_gate, w_up, w_down, w_lm;
@@ -1356,8 +1356,8 @@ struct UmmaMaps {
 };
 
 bool make_plane_maps(PlaneMaps* pm, const void* base, size_t cols) {
-  for (int i = 0; i < 4; ++i)
-    if (!make_map(&pm->m[i], base, umma::kMaxRows, cols, 16 << i)) return false;
+  for (int i = 0; i < umma::kNumRowPads; ++i)
+    if (!make_map(&pm->m[i], base, umma::kMaxRows, cols, umma::kRowPads[i])) return false;
   return true;
 }
 
@@ -1418,8 +1418,9 @@ template <int EPI>
 ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
                       const PlaneMaps& ph, const PlaneMaps& pl, UArgs& a, const FusedScratch& f,
                       cudaStream_t st) {
-  const int mi = a.M <= 16 ? 0 : a.M <= 32 ? 1 : a.M <= 64 ? 2 : 3;
-  a.Mp = 16 << mi;
+  int mi = 0;
+  while (umma::kRowPads[mi] < a.M) ++mi;
+  a.Mp = umma::kRowPads[mi];
   const CUtensorMap &bh = ph.m[mi], &bl = pl.m[mi];
   a.KB = (a.K + umma::kBK - 1) / umma::kBK;
   if (a.zip) {
@@ -1437,8 +1438,12 @@ ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, c
   if ((long long)a.n_tiles * a.KB * (c->n_sm + 1) >= (1ll << 31)) return fail(c, PS_ERR_UNSUPPORTED, "too many GEMM units");
   a.split = choose_split(a.M, a.Mp, a.n_tiles, a.KB, c->n_sm);
   a.partials = f.partials; a.tile_tickets = f.tile_tickets; a.status = c->dev_status;
-  auto kern = mi == 0 ? k_umma_gemm<EPI, 16> : mi == 1 ? k_umma_gemm<EPI, 32> : mi == 2 ? k_umma_gemm<EPI, 64>
-                                                                                     : k_umma_gemm<EPI, 128>;
+  auto kern = mi == 0   ? k_umma_gemm<EPI, 16>
+              : mi == 1 ? k_umma_gemm<EPI, 32>
+              : mi == 2 ? k_umma_gemm<EPI, 48>
+              : mi == 3 ? k_umma_gemm<EPI, 64>
+              : mi == 4 ? k_umma_gemm<EPI, 96>
+                        : k_umma_gemm<EPI, 128>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, umma::kSmemBytes);
   if (e != cudaSuccess) return cuda_check(c, e, "umma smem attribute");
   e = launch_after(kern, dim3(c->n_sm), dim3(umma::kThreads), umma::kSmemBytes, st, !c->prof, a0, a1, a2, bh, bl, a);

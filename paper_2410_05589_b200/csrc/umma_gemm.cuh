@@ -1,6 +1,6 @@
 // Weight-streaming small-M GEMM on the 5th-generation tensor cores:
 //   Y[m][n] = sum_k A[m][k] * W[n][k],  M = B*(k+1) <= 128 rows, W row-major bf16, fp32 sums.
-// (The description below is for up to 16 rows; with Mp = 32, 64 or 128 padded rows the planes
+// (The description below is for up to 16 rows; with Mp = 32, 48, 64, 96 or 128 padded rows the planes
 // form an N = 2 Mp operand, stages grow and get fewer, and fewer accumulators fit: see
 // stage_bytes(), n_stages(), k_split() below.)
 //
@@ -48,7 +48,7 @@ using ws::smem_u32;
 constexpr int kTile = 128;                        // weight rows per tile (MMA M)
 constexpr int kBK = 64;                           // k columns per unit: one 128-byte swizzle span
 constexpr int kN = 16;                            // activation rows per epilogue chunk
-constexpr int kMaxRows = 128;                     // activation rows of a launch (padded to 16, 32, 64 or 128)
+constexpr int kMaxRows = 128;                     // activation rows of a launch (padded to one of kRowPads)
 constexpr int kABytes = kTile * kBK * 2;          // 16 KB
 constexpr int kBBytes = kN * kBK * 2;             // 2 KB per plane at 16 rows
 constexpr int kStageBytes = kABytes + 2 * kBBytes;
@@ -56,7 +56,7 @@ constexpr int kStages = 10;                       // at 16 rows; fewer, larger s
 constexpr int kRingBytes = kStages * kStageBytes;
 constexpr int kThreads = 192;
 constexpr int kEpiThreads = 128;
-// Geometry of a launch with Mp padded activation rows (16, 32, 64 or 128): the hi and lo planes
+// Geometry of a launch with Mp padded activation rows (one of kRowPads): the hi and lo planes
 // form one MMA operand of N = 2 Mp columns; ksplit independent accumulators per tile (one per k
 // step of a unit while tensor memory allows: MMAs into one accumulator serialise); two tiles'
 // accumulators in tensor memory.
@@ -64,9 +64,14 @@ __host__ __device__ constexpr int stage_bytes(int Mp) { return kABytes + 2 * Mp 
 __host__ __device__ constexpr int n_stages(int Mp) {
   return kRingBytes / stage_bytes(Mp) < kStages ? kRingBytes / stage_bytes(Mp) : kStages;
 }
-__host__ __device__ constexpr int k_split(int Mp) { return 256 / (2 * Mp) < kBK / 16 ? 256 / (2 * Mp) : kBK / 16; }
+// (a power of two: 4 up to 32 rows, 2 up to 64, else 1)
+__host__ __device__ constexpr int k_split(int Mp) { return Mp <= 32 ? kBK / 16 : (Mp <= 64 ? 2 : 1); }
 __host__ __device__ constexpr int acc_cols(int Mp) { return k_split(Mp) * 2 * Mp; }
-__host__ __device__ constexpr int tmem_cols(int Mp) { return 2 * acc_cols(Mp); }   // 256 or 512
+// columns to allocate: two tiles' accumulators, rounded up to a power of two (256 or 512)
+__host__ __device__ constexpr int tmem_cols(int Mp) { return 2 * acc_cols(Mp) <= 256 ? 256 : 512; }
+// padded row counts the kernel is compiled for
+constexpr int kRowPads[] = {16, 32, 48, 64, 96, 128};
+constexpr int kNumRowPads = 6;
 // Instruction descriptor of kind::f16: fp32 accumulator, bf16 x bf16, both operands K-major,
 // N / 8 in bits [17,23), M / 16 in bits [24,29).
 constexpr uint32_t idesc(int n) {
