@@ -420,15 +420,24 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
     part.pick = -1; part.lastp = -1; part.wsum = 0.0; part.st = 0.0; part.sd = 0.0;
   }
   cl.sync();
+  // lane r of every warp fetches block r's partial (one round trip through distributed shared
+  // memory for the whole cluster instead of one per block), a shuffle tree combines them; every
+  // warp of every block runs the same tree on the same values
   tm = -INFINITY; dm = -INFINITY; ti = 0x7fffffff; bad = 0;
-  for (int r = 0; r < nclu; ++r) {
-    const CluPart* pr = cl.map_shared_rank(&part, r);
-    const float ov = pr->tmax;
-    const int oi = pr->targ;
-    if (ov > tm || (ov == tm && oi < ti)) { tm = ov; ti = oi; }
-    dm = fmaxf(dm, pr->dmax);
-    bad |= pr->bad;
+  if (lane < nclu) {
+    const CluPart* pr = cl.map_shared_rank(&part, lane);
+    tm = pr->tmax; ti = pr->targ; dm = pr->dmax; bad = pr->bad;
   }
+#pragma unroll
+  for (int o = nclu / 2; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, tm, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, ti, o);
+    if (ov > tm || (ov == tm && oi < ti)) { tm = ov; ti = oi; }
+    dm = fmaxf(dm, __shfl_xor_sync(0xffffffffu, dm, o));
+    bad |= __shfl_xor_sync(0xffffffffu, bad, o);
+  }
+  tm = __shfl_sync(0xffffffffu, tm, 0); ti = __shfl_sync(0xffffffffu, ti, 0);
+  dm = __shfl_sync(0xffffffffu, dm, 0); bad = __shfl_sync(0xffffffffu, bad, 0);
   if (tm == -INFINITY || (drow && dm == -INFINITY)) bad = 1;  // a row without a distribution
   const float tmax = tm, dmax = dm;
   const int targ = ti;
@@ -465,10 +474,16 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
     }
     cl.sync();
     st = 0.0; sd = 0.0;
-    for (int r = 0; r < nclu; ++r) {
-      const CluPart* pr = cl.map_shared_rank(&part, r);
-      st += pr->st; sd += pr->sd;
+    if (lane < nclu) {
+      const CluPart* pr = cl.map_shared_rank(&part, lane);
+      st = pr->st; sd = pr->sd;
     }
+#pragma unroll
+    for (int o = nclu / 2; o > 0; o >>= 1) {
+      st += __shfl_xor_sync(0xffffffffu, st, o);
+      sd += __shfl_xor_sync(0xffffffffu, sd, o);
+    }
+    st = __shfl_sync(0xffffffffu, st, 0); sd = __shfl_sync(0xffffffffu, sd, 0);
     if (!drow) sd = 1.0;
     uint32_t c[4] = {(uint32_t)i, (uint32_t)b, a.off_lo, a.off_hi};
     philox4x32_10(a.key0, a.key1, c);
@@ -519,17 +534,24 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
           part.wsum = x1; part.lastp = lp; part.pick = -1;
         }
         cl.sync();
-        // level 1: the block whose running sum first exceeds the target
-        double total = 0.0;
-        for (int rr = 0; rr < nclu; ++rr) total += cl.map_shared_rank(&part, rr)->wsum;
+        // level 1: the block whose running sum first exceeds the target (lane r holds block r's
+        // weight; a shuffle scan gives every block's running sum)
+        double bw = lane < nclu ? cl.map_shared_rank(&part, lane)->wsum : 0.0;
+        double binc = bw;
+#pragma unroll
+        for (int o = 1; o < nclu; o <<= 1) {
+          const double up = __shfl_up_sync(0xffffffffu, binc, o);
+          if (lane >= o) binc += up;
+        }
+        const double total = __shfl_sync(0xffffffffu, binc, nclu - 1);
         int sel = -1;
         if (total > 0.0) {
           const double target = u2 * total;
-          double run = 0.0, base = 0.0;
-          for (int rr = 0; rr < nclu; ++rr) {
-            const double nx = run + cl.map_shared_rank(&part, rr)->wsum;
-            if (sel < 0 && nx > target) { sel = rr; base = run; }
-            run = nx;
+          const unsigned over_b = __ballot_sync(0xffffffffu, lane < nclu && binc > target);
+          double base = 0.0;
+          if (over_b) {
+            sel = __ffs(over_b) - 1;
+            base = __shfl_sync(0xffffffffu, binc - bw, sel);
           }
           if (sel == rank) {
             // level 2: the warp, level 3: the lane, level 4: the token
