@@ -410,14 +410,22 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
   }
   if (lane == 0) { s.f[warp] = tm; s.i[warp] = ti; s.flag[warp] = bad; s.f2[warp] = dm; }
   __syncthreads();
-  if (tid == 0) {
-    for (int w = 1; w < kCluWarps; ++w) {
-      if (s.f[w] > tm || (s.f[w] == tm && s.i[w] < ti)) { tm = s.f[w]; ti = s.i[w]; }
-      dm = fmaxf(dm, s.f2[w]);
-      bad |= s.flag[w];
+  if (warp == 0) {   // the warps' values, one per lane, through a shuffle tree
+    static_assert(kCluWarps == 16, "one lane per warp in the low half of warp 0");
+    tm = -INFINITY; dm = -INFINITY; ti = 0x7fffffff; bad = 0;
+    if (lane < kCluWarps) { tm = s.f[lane]; ti = s.i[lane]; bad = s.flag[lane]; dm = s.f2[lane]; }
+#pragma unroll
+    for (int o = kCluWarps / 2; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, tm, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, ti, o);
+      if (ov > tm || (ov == tm && oi < ti)) { tm = ov; ti = oi; }
+      dm = fmaxf(dm, __shfl_xor_sync(0xffffffffu, dm, o));
+      bad |= __shfl_xor_sync(0xffffffffu, bad, o);
     }
-    part.tmax = tm; part.targ = ti; part.dmax = dm; part.bad = bad;
-    part.pick = -1; part.lastp = -1; part.wsum = 0.0; part.st = 0.0; part.sd = 0.0;
+    if (lane == 0) {
+      part.tmax = tm; part.targ = ti; part.dmax = dm; part.bad = bad;
+      part.pick = -1; part.lastp = -1; part.wsum = 0.0; part.st = 0.0; part.sd = 0.0;
+    }
   }
   cl.sync();
   // lane r of every warp fetches block r's partial (one round trip through distributed shared
@@ -467,10 +475,14 @@ __device__ __forceinline__ void verify_cluster_body(const VerifyArgs& a) {
     sd = warp_sum_d(sd);
     if (lane == 0) { s.d[warp] = st; s.d2[warp] = sd; }
     __syncthreads();
-    if (tid == 0) {
-      double x1 = 0.0, x2 = 0.0;
-      for (int w = 0; w < kCluWarps; ++w) { x1 += s.d[w]; x2 += s.d2[w]; }
-      part.st = x1; part.sd = x2;
+    if (warp == 0) {
+      double x1 = lane < kCluWarps ? s.d[lane] : 0.0, x2 = lane < kCluWarps ? s.d2[lane] : 0.0;
+#pragma unroll
+      for (int o = kCluWarps / 2; o > 0; o >>= 1) {
+        x1 += __shfl_xor_sync(0xffffffffu, x1, o);
+        x2 += __shfl_xor_sync(0xffffffffu, x2, o);
+      }
+      if (lane == 0) { part.st = x1; part.sd = x2; }
     }
     cl.sync();
     st = 0.0; sd = 0.0;
