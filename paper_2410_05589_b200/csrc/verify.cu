@@ -677,8 +677,11 @@ __device__ double cluster_sum(cooperative_groups::cluster_group& cl, CluPart& pa
     part.wsum = x1;
   }
   cl.sync();
-  double tot = 0.0;
-  for (int rr = 0; rr < (int)cl.num_blocks(); ++rr) tot += cl.map_shared_rank(&part, rr)->wsum;
+  // lane r fetches block r's sum (one remote round trip), a shuffle tree adds them
+  double tot = lane < (int)cl.num_blocks() ? cl.map_shared_rank(&part, lane)->wsum : 0.0;
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+  tot = __shfl_sync(0xffffffffu, tot, 0);
   cl.sync();   // every block has read the partials before they are rewritten
   return tot;
 }
@@ -713,16 +716,24 @@ __device__ int cluster_draw(cooperative_groups::cluster_group& cl, CluPart& part
     part.wsum = x1; part.lastp = lp; part.pick = -1;
   }
   cl.sync();
-  double total = 0.0;
-  for (int rr = 0; rr < (int)cl.num_blocks(); ++rr) total += cl.map_shared_rank(&part, rr)->wsum;
+  // lane r holds block r's weight; a shuffle scan gives every block's running sum
+  const int nb = (int)cl.num_blocks();
+  const double bw = lane < nb ? cl.map_shared_rank(&part, lane)->wsum : 0.0;
+  double binc = bw;
+#pragma unroll
+  for (int o = 1; o < 16; o <<= 1) {
+    const double up = __shfl_up_sync(0xffffffffu, binc, o);
+    if (lane >= o) binc += up;
+  }
+  const double total = __shfl_sync(0xffffffffu, binc, nb - 1);
   int sel = -1, token = -1;
   if (total > 0.0) {
     const double target = u * total;
-    double run = 0.0, base = 0.0;
-    for (int rr = 0; rr < (int)cl.num_blocks(); ++rr) {
-      const double nx = run + cl.map_shared_rank(&part, rr)->wsum;
-      if (sel < 0 && nx > target) { sel = rr; base = run; }
-      run = nx;
+    const unsigned over_b = __ballot_sync(0xffffffffu, lane < nb && binc > target);
+    double base = 0.0;
+    if (over_b) {
+      sel = __ffs(over_b) - 1;
+      base = __shfl_sync(0xffffffffu, binc - bw, sel);
     }
     if (sel == rank) {
       double t2 = target - base, wrun = 0.0, wbase = 0.0;
