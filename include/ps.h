@@ -49,6 +49,8 @@ enum {
   PS_FLAG_FC_BIAS = 1,          /* ps_weights.b_fc is used */
   PS_FLAG_UNFUSED_KERNELS = 2,  /* force the unfused fp32-activation kernels (debugging aid) */
   PS_FLAG_MMA_SYNC_GEMM = 4,    /* fused path: mma.sync GEMM kernels instead of the tcgen05 ones */
+  PS_FLAG_STAGE_LAUNCHES = 16,  /* tensor-core path: one launch per GEMM stage also with up to 16 rows, where
+                                   the stages on either side of the attention otherwise share a launch */
   PS_FLAG_NO_FC = 8             /* embedding-only input (the Medusa integration, Sec. 4.3): x0 is the token /
                                    [MASK] embedding, there is no fc layer and no target feature; w_fc,
                                    mask_feat and every `hidden` argument are ignored and may be NULL */

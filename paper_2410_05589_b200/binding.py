@@ -18,6 +18,7 @@ STATUS_NAMES = {0: "PS_OK", -1: "PS_ERR_INVALID_ARG", -2: "PS_ERR_UNSUPPORTED", 
                 -4: "PS_ERR_CUDA", -5: "PS_ERR_TIMEOUT", -6: "PS_ERR_NONFINITE"}
 PS_DTYPE_F32, PS_DTYPE_BF16 = 0, 1
 PS_FLAG_FC_BIAS, PS_FLAG_UNFUSED_KERNELS, PS_FLAG_MMA_SYNC_GEMM, PS_FLAG_NO_FC = 1, 2, 4, 8
+PS_FLAG_STAGE_LAUNCHES = 16
 PS_MAX_BATCH, PS_MAX_MASKS, PS_MAX_TOP_N = 128, 15, 8
 
 WEIGHT_NAMES = (

@@ -415,6 +415,7 @@ struct FusedScratch {
   __nv_bfloat16* xin;       // [kMaxM][2H] gathered fc input (exact bf16: one plane)
   float* partials;          // [kMaxSm][2][16][128] partial tiles of CTAs that share a tile
   unsigned* tile_tickets;   // one per tile of the widest stage, zero between launches
+  unsigned* chain_ctr;      // chained stages: finished-tile and passed-CTA counts, zero between launches
   int n_part_rows;          // rows of `parts` and of each ssq array
   size_t bytes;
 };
@@ -453,6 +454,7 @@ FusedScratch carve_fused(const ps_config& g, char* base) {
   const size_t max_tiles = std::max<size_t>({(size_t)tiles_v, (size_t)(g.ffn + 63) / 64,
                                              (Hq + 127) / 128 + 2 * ((Hkv + 127) / 128), (size_t)tiles_h});
   s.tile_tickets = (unsigned*)take(max_tiles * 4);
+  s.chain_ctr = (unsigned*)take(256);
   s.x0p = planes(g.hidden); s.ap = planes(g.hidden); s.hdnp = planes(g.hidden);
   s.attnp = planes(Hq); s.actp = planes(g.ffn);
   s.bytes = off;
@@ -578,14 +580,15 @@ __device__ __forceinline__ int tile_feature(const UArgs& a, int t, int r, bool& 
 // Epilogue of one finished tile for the activation rows [m0, m0 + mc), mc <= 16; called by the
 // 128 epilogue threads after each has put its accumulator row r (= 32 * q + lane) of those
 // rows into ctl.acc[(m - m0) * 128 + r].  A dry call executes the same instructions and writes
-// nothing to global memory.  With UNR = 1
+// nothing to global memory.  res_pre: the caller has put the rows' residual values into
+// ctl.land[m * 128 + r] already (m0 = 0).  With UNR = 1
 // the loops over m are rolled on purpose: for up to 16 rows this code runs once or twice per
 // CTA, so what it costs is the fetch of its instructions, not their execution.  With more rows
 // it runs once per 16 rows of every tile and its single warp per scheduler is bound by the
 // latency of dependent instructions: UNR = 4 interleaves four rows.
 template <int EPI, int UNR>
 __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, int t, int r, int q, int lane,
-                                              int m0, int mc, bool dry) {
+                                              int m0, int mc, bool dry, bool res_pre = false) {
   using namespace umma;
   const int et = r;
   bool valid;
@@ -600,7 +603,9 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
       float rv[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        rv[j] = (a.res && valid && mg + j < mc) ? __ldcg(a.res + (size_t)(m0 + mg + j) * a.ldr + n) : 0.f;
+        rv[j] = (a.res && valid && mg + j < mc)
+                    ? (res_pre ? ctl.land[(mg + j) * 128 + r] : __ldcg(a.res + (size_t)(m0 + mg + j) * a.ldr + n))
+                    : 0.f;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int m = mg + j;
@@ -799,6 +804,113 @@ __device__ __forceinline__ void big_chunk_epilogue(const UArgs& a, umma::Ctl& ct
     }
     epi_sync();
   }
+}
+
+// Last step of an LM-head launch, called by all threads of every CTA after its tiles are done:
+// the last CTA to finish merges the per-tile summaries (no CTA waits for another).
+__device__ __forceinline__ void lm_merge(const UArgs& a, umma::Ctl& ctl, int tid, int warp, int lane) {
+  if (tid == 0) {
+    __threadfence();
+    const unsigned tk = atomicAdd(a.ticket, 1u);
+    ctl.is_last = (tk == gridDim.x - 1);
+    if (ctl.is_last) __threadfence();
+  }
+  __syncthreads();
+  if (ctl.is_last && !ctl.abort_flag) {
+    // all six warps, one activation row each; the loops are unrolled so that the loads of
+    // eight tiles are in flight together (they come from L2, written by other SMs)
+    const int Gt = a.n_tiles;
+    for (int m = warp; m < a.M; m += umma::kThreads / 32) {
+      const LmPart* P = a.parts + m;
+      // 256 tiles per round, 8 per lane, their loads issued together.  The first round also
+      // fetches every tile's best token: the row's arg-max needs nothing else.
+      float mx = -FLT_MAX, se = 0.f;
+      float bv0 = -FLT_MAX; int bi0 = 0x7fffffff;
+      for (int c0 = 0; c0 < Gt; c0 += 256) {
+        float vm[8], sx[8], tv[8]; int ti[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int c = c0 + lane + 32 * j;
+          float4 hd = make_float4(-FLT_MAX, 0.f, -FLT_MAX, __int_as_float(0x7fffffff));
+          if (c < Gt) hd = __ldcg(reinterpret_cast<const float4*>(&P[(size_t)c * a.M]));
+          vm[j] = hd.x; sx[j] = hd.y; tv[j] = hd.z;
+          ti[j] = a.top_n > 0 ? __float_as_int(hd.w) : 0x7fffffff;
+        }
+        float nm = mx;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          nm = fmaxf(nm, vm[j]);
+          if (ti[j] != 0x7fffffff && (tv[j] > bv0 || (tv[j] == bv0 && ti[j] < bi0))) { bv0 = tv[j]; bi0 = ti[j]; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) nm = fmaxf(nm, __shfl_xor_sync(0xffffffffu, nm, o));
+        float add = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) add += sx[j] * __expf(vm[j] - nm);
+        se = se * __expf(mx - nm) + warp_sum(add);
+        mx = nm;
+      }
+      if (lane == 0) {
+        if (a.row_max) a.row_max[m] = mx;
+        if (a.row_lse) a.row_lse[m] = mx + logf(se);
+      }
+      float pv = FLT_MAX; int pi = -1;
+      for (int tn = 0; tn < a.top_n; ++tn) {
+        float bv = bv0; int bi = bi0;
+        if (tn > 0) {   // deeper picks: a tile's list is sorted, any of its entries may be next
+          bv = -FLT_MAX; bi = 0x7fffffff;
+          for (int k = 0; k < a.top_n; ++k) {
+            for (int c0 = 0; c0 < Gt; c0 += 256) {
+              float xv[8]; int id[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const int c = c0 + lane + 32 * j;
+                xv[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_v[k]) : 0.f;
+                id[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_i[k]) : 0x7fffffff;
+              }
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const bool after = id[j] != 0x7fffffff && ((xv[j] < pv) || (xv[j] == pv && id[j] > pi));
+                if (after && (xv[j] > bv || (xv[j] == bv && id[j] < bi))) { bv = xv[j]; bi = id[j]; }
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+          if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == 0) { a.top_ids[(size_t)m * a.top_n + tn] = bi; a.top_logit[(size_t)m * a.top_n + tn] = bv; }
+        pv = bv; pi = bi;
+      }
+      if (a.sample) {   // the row's sampled token: arg-max of the ranges' perturbed maxima
+        float bv = -FLT_MAX; int bi = 0x7fffffff;
+        for (int c0 = 0; c0 < Gt; c0 += 256) {
+          float xv[8]; int id[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int c = c0 + lane + 32 * j;
+            xv[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].sv) : -FLT_MAX;
+            id[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].si) : 0x7fffffff;
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (xv[j] > bv || (xv[j] == bv && id[j] < bi)) { bv = xv[j]; bi = id[j]; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+          if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == 0) a.sa.sampled[m] = bi;
+      }
+    }
+  }
+  if (ctl.is_last && tid == 0) *a.ticket = 0u;
+  __syncthreads();
 }
 
 static_assert(umma::kMaxCtas >= kMaxSm, "contributor table covers every CTA of a launch");
@@ -1129,115 +1241,410 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   }
 
   __syncthreads();
-  if (EPI == EPI_LMHEAD) {
-    // the last CTA to finish merges the per-tile summaries (no CTA waits for another)
-    if (tid == 0) {
-      __threadfence();
-      const unsigned tk = atomicAdd(a.ticket, 1u);
-      ctl.is_last = (tk == gridDim.x - 1);
-      if (ctl.is_last) __threadfence();
-    }
-    __syncthreads();
-    if (ctl.is_last && !ctl.abort_flag) {
-      // all six warps, one activation row each; the loops are unrolled so that the loads of
-      // eight tiles are in flight together (they come from L2, written by other SMs)
-      const int Gt = a.n_tiles;
-      for (int m = warp; m < a.M; m += umma::kThreads / 32) {
-        const LmPart* P = a.parts + m;
-        // 256 tiles per round, 8 per lane, their loads issued together.  The first round also
-        // fetches every tile's best token: the row's arg-max needs nothing else.
-        float mx = -FLT_MAX, se = 0.f;
-        float bv0 = -FLT_MAX; int bi0 = 0x7fffffff;
-        for (int c0 = 0; c0 < Gt; c0 += 256) {
-          float vm[8], sx[8], tv[8]; int ti[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int c = c0 + lane + 32 * j;
-            float4 hd = make_float4(-FLT_MAX, 0.f, -FLT_MAX, __int_as_float(0x7fffffff));
-            if (c < Gt) hd = __ldcg(reinterpret_cast<const float4*>(&P[(size_t)c * a.M]));
-            vm[j] = hd.x; sx[j] = hd.y; tv[j] = hd.z;
-            ti[j] = a.top_n > 0 ? __float_as_int(hd.w) : 0x7fffffff;
-          }
-          float nm = mx;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            nm = fmaxf(nm, vm[j]);
-            if (ti[j] != 0x7fffffff && (tv[j] > bv0 || (tv[j] == bv0 && ti[j] < bi0))) { bv0 = tv[j]; bi0 = ti[j]; }
-          }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) nm = fmaxf(nm, __shfl_xor_sync(0xffffffffu, nm, o));
-          float add = 0.f;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) add += sx[j] * __expf(vm[j] - nm);
-          se = se * __expf(mx - nm) + warp_sum(add);
-          mx = nm;
-        }
-        if (lane == 0) {
-          if (a.row_max) a.row_max[m] = mx;
-          if (a.row_lse) a.row_lse[m] = mx + logf(se);
-        }
-        float pv = FLT_MAX; int pi = -1;
-        for (int tn = 0; tn < a.top_n; ++tn) {
-          float bv = bv0; int bi = bi0;
-          if (tn > 0) {   // deeper picks: a tile's list is sorted, any of its entries may be next
-            bv = -FLT_MAX; bi = 0x7fffffff;
-            for (int k = 0; k < a.top_n; ++k) {
-              for (int c0 = 0; c0 < Gt; c0 += 256) {
-                float xv[8]; int id[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const int c = c0 + lane + 32 * j;
-                  xv[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_v[k]) : 0.f;
-                  id[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_i[k]) : 0x7fffffff;
-                }
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const bool after = id[j] != 0x7fffffff && ((xv[j] < pv) || (xv[j] == pv && id[j] > pi));
-                  if (after && (xv[j] > bv || (xv[j] == bv && id[j] < bi))) { bv = xv[j]; bi = id[j]; }
-                }
-              }
-            }
-          }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-          }
-          if (lane == 0) { a.top_ids[(size_t)m * a.top_n + tn] = bi; a.top_logit[(size_t)m * a.top_n + tn] = bv; }
-          pv = bv; pi = bi;
-        }
-        if (a.sample) {   // the row's sampled token: arg-max of the ranges' perturbed maxima
-          float bv = -FLT_MAX; int bi = 0x7fffffff;
-          for (int c0 = 0; c0 < Gt; c0 += 256) {
-            float xv[8]; int id[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const int c = c0 + lane + 32 * j;
-              xv[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].sv) : -FLT_MAX;
-              id[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].si) : 0x7fffffff;
-            }
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-              if (xv[j] > bv || (xv[j] == bv && id[j] < bi)) { bv = xv[j]; bi = id[j]; }
-          }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-          }
-          if (lane == 0) a.sa.sampled[m] = bi;
-        }
-      }
-    }
-    if (ctl.is_last && tid == 0) *a.ticket = 0u;
-    __syncthreads();
-  }
+  if (EPI == EPI_LMHEAD) lm_merge(a, ctl, tid, warp, lane);
   if (ctl.abort_flag) {
     // let copies and MMAs that are still in flight finish before shared and tensor memory go
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     if (tid == 0) atomicOr(a.status, kStatTimeout);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    fence_after_sync();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols(MP)) : "memory");
+  }
+}
+
+// ---- several GEMM stages in one launch (up to 16 activation rows) ---------------------------------
+// Consecutive stages of the draft step (fc -> q|k|v, and o -> gate|up -> down -> LM head) run
+// as one launch of one CTA per SM.  Between two launches the stream of weights stops: the ring
+// drains, the blocks leave, the next launch's blocks arrive and start asking again.  Inside one
+// launch the producer thread goes straight on to the next stage's weight boxes as ring slots
+// come free, so the stream only stops when the ring is full of them and the stage's
+// activations are not there yet.  A stage's activations are complete when all tiles of the
+// stage before it have run their epilogue: every finisher adds one to a counter in global
+// memory (release); the producer thread and one epilogue thread of every CTA wait for the count
+// (acquire, bounded), and the last of them to see it complete zeroes it for the next launch.
+// The CTAs wait for one another, so all must be resident at once: one CTA per SM, see the
+// launch in run_stages; every wait is bounded.  The tail of a tile (partials, ticket, sum of
+// the partials, epilogue, count) is a chain of round trips to L2 and is what a stage costs
+// beyond its stream: partials are kept as 16-byte vectors per accumulator row so that the last
+// arriver has all contributors' values in flight at once, and what does not depend on the sums
+// (who shares the tile, the residual rows) is fetched while the MMAs still run.
+constexpr int kChainMax = 4, kChainMaps = 13;
+struct ChainParams {
+  int n;                                  // stages
+  int epi[kChainMax];
+  int map_a[kChainMax][3], map_bh[kChainMax], map_bl[kChainMax];   // indices into maps
+  unsigned* done;                         // [kChainMax] tiles finished per stage, zero between launches
+  unsigned* passed;                       // [kChainMax] CTAs that have seen the stage complete
+  UArgs a[kChainMax];
+  CUtensorMap maps[kChainMaps];
+};
+static_assert(sizeof(ChainParams) <= 4000, "kernel parameters");
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+template <int MP>
+__global__ void __launch_bounds__(umma::kThreads, 1) k_umma_chain(const __grid_constant__ ChainParams p) {
+  using namespace umma;
+  static_assert(MP == 16, "chained stages take up to 16 rows");
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* stages = smem_raw + (base - raw);
+  Ctl& ctl = *reinterpret_cast<Ctl*>(stages + kStages * kStageBytes);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    for (int i = 0; i < kStages; ++i) { mbar_init(&ctl.full[i], 1); mbar_init(&ctl.empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], kEpiThreads); }
+    ctl.abort_flag = 0; ctl.is_last = 0; ctl.tile_last = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    pdl_launch_dependents();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
+                 "r"(tmem_cols(MP))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem = *(volatile uint32_t*)&ctl.tmem_base;
+
+  const int G = gridDim.x;
+  volatile int* abort_flag = &ctl.abort_flag;
+  constexpr int sbytes = stage_bytes(MP), nst = n_stages(MP), ksplit = k_split(MP), acols = acc_cols(MP);
+  constexpr int plane_bytes = MP * kBK * 2;
+  auto stage_segs = [&](const UArgs& a) {
+    const int U = a.n_tiles * a.KB;
+    return Segs(unit_begin(blockIdx.x, U, G), unit_begin(blockIdx.x + 1, U, G), a.KB);
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {   // ---- TMA producer
+      // Ring position g counts this CTA's units over all stages: unit g goes to slot g % nst and
+      // is the slot's use number g / nst.  Two cursors per stage: weight boxes are requested as
+      // soon as a slot is free, activation boxes follow once the stage before is complete.
+      int sa = 0;                    // ring position of the next weight request: slot and use number
+      uint32_t ua = 0;
+      bool alive = true;
+      for (int s = 0; s < p.n && alive; ++s) {
+        const UArgs& a = p.a[s];
+        const Segs segs = stage_segs(a);
+        const int n_units = segs.u1 - segs.u0;
+        bool seen_done = false;   // this thread has seen the count of the stage before complete
+        if (s == 0 && n_units <= 0) pdl_wait();
+        const uint32_t bytes = kABytes + plane_bytes * (a.lo ? 2 : 1);
+        const CUtensorMap *tA0 = &p.maps[p.map_a[s][0]], *tA1 = &p.maps[p.map_a[s][1]], *tA2 = &p.maps[p.map_a[s][2]];
+        const CUtensorMap *tBh = &p.maps[p.map_bh[s]], *tBl = &p.maps[p.map_bl[s]];
+        UnitWalk wa, wb;
+        wa.start(segs, a);
+        wb.start(segs, a);
+        int ia = 0, ib = 0, sb = sa;   // (sb: slot of the next activation request)
+        bool dep_ok = false;
+        long long t0 = 0;
+        while (ib < n_units) {
+          bool moved = false;
+          if (ia < n_units && (ua == 0 || mbar_peek(&ctl.empty[sa], (ua & 1) ^ 1))) {
+            const uint32_t dst = base + sa * sbytes;
+            const int x = wa.kb * kBK;
+            mbar_arrive_expect_tx(&ctl.full[sa], bytes);
+            if (a.zip) {
+              tma_load_2d(dst, tA0, x, wa.row0, &ctl.full[sa]);
+              tma_load_2d(dst + kABytes / 2, tA1, x, wa.row0, &ctl.full[sa]);
+            } else {
+              tma_load_2d(dst, wa.mat == 0 ? tA0 : (wa.mat == 1 ? tA1 : tA2), x, wa.row0, &ctl.full[sa]);
+            }
+            wa.next(segs, a);
+            ++ia;
+            if (++sa == nst) { sa = 0; ++ua; }
+            moved = true;
+          }
+          if (dep_ok) {
+            if (ib < ia) {
+              const uint32_t dst = base + sb * sbytes + kABytes;
+              const int x = wb.kb * kBK;
+              tma_load_2d(dst, tBh, x, 0, &ctl.full[sb]);
+              if (a.lo) tma_load_2d(dst + plane_bytes, tBl, x, 0, &ctl.full[sb]);
+              wb.next(segs, a);
+              ++ib;
+              if (++sb == nst) sb = 0;
+              moved = true;
+            }
+          } else if (s == 0) {
+            if (!moved) {   // the first stage's weight requests fill the ring, then the kernel before this one
+              pdl_wait();
+              dep_ok = true;
+              moved = true;
+            }
+          } else if (ld_acquire_u32(p.done + (s - 1)) >= (unsigned)p.a[s - 1].n_tiles) {
+            fence_proxy_async();   // what other SMs wrote is read by the copy engine from here on
+            dep_ok = true;
+            seen_done = true;
+            moved = true;
+          }
+          if (!moved) {
+            if (dep_ok) {   // every request made, the ring is full: wait for the slot
+              if (!mbar_wait(&ctl.empty[sa], (ua & 1) ^ 1, abort_flag)) { alive = false; break; }
+            } else {
+              if (t0 == 0) t0 = clock64();
+              if (*abort_flag || clock64() - t0 > ws::kWaitCycles) { *abort_flag = 1; alive = false; break; }
+            }
+          }
+        }
+        // both this thread and the epilogue warps' poller check in on every count, also a CTA
+        // without units: the last of the 2 G to do so zeroes it
+        if (s > 0 && alive) {
+          if (!seen_done) {
+            const long long t1 = clock64();
+            while (ld_acquire_u32(p.done + (s - 1)) < (unsigned)p.a[s - 1].n_tiles) {
+              if (*abort_flag || clock64() - t1 > ws::kWaitCycles) { *abort_flag = 1; alive = false; break; }
+            }
+          }
+          if (alive && atomicAdd(p.passed + (s - 1), 1u) == (unsigned)(2 * G - 1)) {
+            p.done[s - 1] = 0u;
+            p.passed[s - 1] = 0u;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {   // ---- MMA issuer
+      int stage = 0, segc = 0;
+      uint32_t parity = 0;
+      bool alive = true;
+      for (int s = 0; s < p.n && alive; ++s) {
+        const UArgs& a = p.a[s];
+        const Segs segs = stage_segs(a);
+        const uint32_t id = a.lo ? idesc(2 * MP) : idesc(MP);
+        for (int si = 0; si < segs.n && alive; ++si, ++segc) {
+          int t, b, e;
+          segs.get(si, t, b, e);
+          const int buf = segc & 1;
+          if (!mbar_wait(&ctl.acc_empty[buf], ((segc >> 1) & 1) ^ 1, abort_flag)) { alive = false; break; }
+          fence_after_sync();
+          const uint32_t d = tmem + buf * acols;
+          uint32_t acc = 0;
+          for (int j = b; j < e; ++j) {
+            if (!mbar_wait(&ctl.full[stage], parity, abort_flag)) { alive = false; break; }
+            fence_after_sync();
+            const uint32_t sa = base + stage * sbytes;
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k) {
+              const int ai = k & (ksplit - 1);
+              mma_f16(d + ai * 2 * MP, smem_desc(sa + k * 32), smem_desc(sa + kABytes + k * 32), id,
+                      (acc || k >= ksplit) ? 1u : 0u);
+            }
+            acc = 1;
+            mma_commit(&ctl.empty[stage]);
+            if (++stage == nst) { stage = 0; parity ^= 1; }
+          }
+          if (alive) mma_commit(&ctl.acc_full[buf]);
+        }
+      }
+    }
+  } else {
+    // ---- epilogue warps: accumulator row r = 32 q + lane
+    const int q = warp & 3, r = 32 * q + lane, et = r;
+    int segc = 0;
+    bool alive = true;
+    for (int s = 0; s < p.n && alive; ++s) {
+      const UArgs& a = p.a[s];
+      const Segs segs = stage_segs(a);
+      const int epi = p.epi[s];
+      // (pass -1 of the first stage: a rehearsal of the reduction and epilogue code, see k_umma_gemm;
+      // rehearsing the later stages' kinds of epilogue as well was measured and changes nothing)
+      for (int seg = (s == 0 && segs.n > 0) ? -1 : 0; seg <= segs.n && alive; ++seg) {
+        const bool dry = seg < 0;
+        if (seg == 0) {
+          // the stage before this one is complete: its outputs, sums of squares and residuals may be read
+          if (s == 0) {
+            pdl_wait();
+          } else {
+            if (et == 0) {
+              const unsigned want = (unsigned)p.a[s - 1].n_tiles;
+              const long long t0 = clock64();
+              bool ok = true;
+              while (ld_acquire_u32(p.done + (s - 1)) < want) {
+                if (*abort_flag || clock64() - t0 > ws::kWaitCycles) { *abort_flag = 1; ok = false; break; }
+              }
+              if (ok && atomicAdd(p.passed + (s - 1), 1u) == (unsigned)(2 * G - 1)) {
+                p.done[s - 1] = 0u;
+                p.passed[s - 1] = 0u;
+              }
+            }
+            if (epi_any(*abort_flag != 0)) { alive = false; break; }
+          }
+          for (int m = warp - 2; m < a.M; m += 4) {   // RMSNorm row scales of the input
+            float sc = 1.f;
+            if (a.ssq_in) {
+              float ss = 0.f;
+              for (int c = lane; c < a.ssq_n; c += 32) ss += __ldcg(a.ssq_in + (size_t)c * a.M + m);
+              ss = warp_sum(ss);
+              sc = rsqrtf(ss / (float)a.K + a.eps);
+            }
+            if (lane == 0) ctl.scale[m] = sc;
+          }
+          epi_sync();
+        }
+        if (seg == segs.n) break;
+        int t, sb, se;
+        segs.get(dry ? 0 : seg, t, sb, se);
+        const int t_begin = t * a.KB, t_end = t_begin + a.KB;
+        const bool whole = !dry && se - sb == a.KB;
+        const int buf = segc & 1, mc = a.M, nvec = (mc + 3) >> 2;
+        const int slot = (t == segs.t0) ? 0 : 1;
+        // (a partial is kept as [accumulator row][16 activation rows]: a thread writes and reads its
+        // rows as 16-byte vectors)
+        float* P = a.partials + ((size_t)blockIdx.x * 2 + slot) * kMaxRows * 128;
+        const int U = a.n_tiles * a.KB;
+        // ---- while the MMAs still run: who shares the tile and where their partials lie, and the
+        // residual rows of a storing epilogue (into ctl.land, each thread its own feature)
+        int c_first = blockIdx.x, c_last = blockIdx.x;
+        if (!whole) {
+          if (!dry) {
+            c_first = unit_owner(t_begin, U, G);
+            c_last = unit_owner(t_end - 1, U, G);
+          }
+          for (int j = et; j <= c_last - c_first; j += kEpiThreads) {
+            const int c = c_first + j, cb = unit_begin(c, U, G);
+            int off = -1;
+            if (cb < unit_begin(c + 1, U, G)) {
+              const int sl = (c == c_first && cb / a.KB != t) ? 1 : 0;
+              off = (c * 2 + sl) * kMaxRows * 128;
+            }
+            ctl.coff[j] = off;
+          }
+        }
+        const bool res_pre = epi == EPI_STORE && a.res != nullptr;
+        if (res_pre) {
+          bool valid;
+          const int n = tile_feature(a, t, r, valid);
+          float rvp[16];
+#pragma unroll
+          for (int m = 0; m < 16; ++m) rvp[m] = (valid && m < mc) ? __ldcg(a.res + (size_t)m * a.ldr + n) : 0.f;
+#pragma unroll
+          for (int m = 0; m < 16; ++m) ctl.land[m * 128 + r] = rvp[m];
+        }
+        if (!whole) epi_sync();   // the contributor table is complete
+        if (!dry && epi_any(!mbar_wait(&ctl.acc_full[buf], (segc >> 1) & 1, abort_flag))) { alive = false; break; }
+        fence_after_sync();
+        const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + buf * acols;
+        float v[16];
+        if (!dry) {   // the tile's sums over this CTA's k-blocks: the accumulators and their hi / lo halves
+          tmem_ld16(ta, v);
+#pragma unroll
+          for (int c = 1; c < 2 * ksplit; ++c) {
+            if (!a.lo && (c & 1)) continue;
+            float vp[16];
+            tmem_ld16(ta + (c >> 1) * 2 * MP + (c & 1) * MP, vp);
+#pragma unroll
+            for (int m = 0; m < 16; ++m) v[m] += vp[m];
+          }
+          fence_before_sync();
+          mbar_arrive(&ctl.acc_empty[buf]);   // the accumulator is read: the MMA warp may reuse it
+        }
+        bool finish = whole || dry;
+        if (!whole && !dry) {
+          float4* d4 = reinterpret_cast<float4*>(P + r * 16);
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            if (i < nvec) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          epi_sync();
+          if (et == 0) {
+            // one thread publishes the block's partial (the barrier above ordered the other
+            // threads' stores before this release) and, if it came last, acquires the others'
+            int n_contrib = 0;
+            for (int j = 0; j <= c_last - c_first; ++j) n_contrib += ctl.coff[j] >= 0;
+            unsigned old;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(&a.tile_tickets[t]) : "memory");
+            const int last = old == (unsigned)(n_contrib - 1);
+            if (last) a.tile_tickets[t] = 0u;
+            ctl.tile_last = last;
+          }
+          epi_sync();
+          finish = ctl.tile_last != 0;
+          epi_sync();   // everyone has read the flag before a later segment rewrites it
+        }
+        if (finish) {
+          if (!whole) {
+            // the partials added in CTA order (the sum does not depend on who came last), all of
+            // up to four contributors' vectors in flight together
+            const int nc = c_last - c_first + 1;
+            const float* Pr = a.partials + r * 16;
+#pragma unroll
+            for (int m = 0; m < 16; ++m) v[m] = 0.f;
+            const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (mc <= 8) {
+#pragma unroll 1
+              for (int j0 = 0; j0 < nc; j0 += 4) {
+                float4 x[4][2];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int o = j0 + j < nc ? ctl.coff[j0 + j] : -1;
+#pragma unroll
+                  for (int i = 0; i < 2; ++i)
+                    x[j][i] = o >= 0 ? __ldcg(reinterpret_cast<const float4*>(Pr + o) + i) : zero4;
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                  for (int i = 0; i < 2; ++i) {
+                    v[4 * i] += x[j][i].x; v[4 * i + 1] += x[j][i].y; v[4 * i + 2] += x[j][i].z; v[4 * i + 3] += x[j][i].w;
+                  }
+              }
+            } else {
+#pragma unroll 1
+              for (int j0 = 0; j0 < nc; j0 += 2) {
+                float4 x[2][4];
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                  const int o = j0 + j < nc ? ctl.coff[j0 + j] : -1;
+#pragma unroll
+                  for (int i = 0; i < 4; ++i)
+                    x[j][i] = o >= 0 ? __ldcg(reinterpret_cast<const float4*>(Pr + o) + i) : zero4;
+                }
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    v[4 * i] += x[j][i].x; v[4 * i + 1] += x[j][i].y; v[4 * i + 2] += x[j][i].z; v[4 * i + 3] += x[j][i].w;
+                  }
+              }
+            }
+          }
+#pragma unroll
+          for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
+          if (epi == EPI_STORE) tile_epilogue<EPI_STORE, 1>(a, ctl, t, r, q, lane, 0, mc, dry, res_pre);
+          else if (epi == EPI_SWIGLU) tile_epilogue<EPI_SWIGLU, 1>(a, ctl, t, r, q, lane, 0, mc, dry);
+          else tile_epilogue<EPI_LMHEAD, 1>(a, ctl, t, r, q, lane, 0, mc, dry);
+          if (!dry && s + 1 < p.n) {   // one more tile of this stage is complete
+            fence_proxy_async();
+            epi_sync();
+            if (et == 0) {
+              __threadfence();
+              atomicAdd(p.done + s, 1u);
+            }
+          }
+        }
+        if (!dry) ++segc;
+      }
+    }
+    fence_before_sync();
+  }
+
+  __syncthreads();
+  if (p.epi[p.n - 1] == EPI_LMHEAD) lm_merge(p.a[p.n - 1], ctl, tid, warp, lane);
+  if (ctl.abort_flag) {
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    if (tid == 0) atomicOr(p.a[0].status, kStatTimeout);
     __syncthreads();
   }
   if (warp == 1) {
@@ -1414,14 +1821,12 @@ static int choose_split(int M, int Mp, int n_tiles, int KB, int G) {
   return best;
 }
 
-template <int EPI>
-ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
-                      const PlaneMaps& ph, const PlaneMaps& pl, UArgs& a, const FusedScratch& f,
-                      cudaStream_t st) {
-  int mi = 0;
-  while (umma::kRowPads[mi] < a.M) ++mi;
-  a.Mp = umma::kRowPads[mi];
-  const CUtensorMap &bh = ph.m[mi], &bl = pl.m[mi];
+// Geometry of one GEMM stage: padded rows, tiles, k-blocks, the split, the shared scratch.
+// *mi = index of the padded row count in umma::kRowPads.
+ps_status prep_uargs(ps_ctx* c, UArgs& a, const FusedScratch& f, int* mi) {
+  *mi = 0;
+  while (umma::kRowPads[*mi] < a.M) ++*mi;
+  a.Mp = umma::kRowPads[*mi];
   a.KB = (a.K + umma::kBK - 1) / umma::kBK;
   if (a.zip) {
     a.n_tiles = (a.N + 63) / 64;
@@ -1438,6 +1843,17 @@ ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, c
   if ((long long)a.n_tiles * a.KB * (c->n_sm + 1) >= (1ll << 31)) return fail(c, PS_ERR_UNSUPPORTED, "too many GEMM units");
   a.split = choose_split(a.M, a.Mp, a.n_tiles, a.KB, c->n_sm);
   a.partials = f.partials; a.tile_tickets = f.tile_tickets; a.status = c->dev_status;
+  return PS_OK;
+}
+
+template <int EPI>
+ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& a2,
+                      const PlaneMaps& ph, const PlaneMaps& pl, UArgs& a, const FusedScratch& f,
+                      cudaStream_t st) {
+  int mi;
+  ps_status s = prep_uargs(c, a, f, &mi);
+  if (s) return s;
+  const CUtensorMap &bh = ph.m[mi], &bl = pl.m[mi];
   auto kern = mi == 0   ? k_umma_gemm<EPI, 16>
               : mi == 1 ? k_umma_gemm<EPI, 32>
               : mi == 2 ? k_umma_gemm<EPI, 48>
@@ -1449,6 +1865,72 @@ ps_status launch_umma(ps_ctx* c, const CUtensorMap& a0, const CUtensorMap& a1, c
   e = launch_after(kern, dim3(c->n_sm), dim3(umma::kThreads), umma::kSmemBytes, st, !c->prof, a0, a1, a2, bh, bl, a);
   c->launches++;
   return cuda_check(c, e, "k_umma_gemm");
+}
+
+// One stage of the draft step as the launchers take it.
+struct StageDesc {
+  int epi;
+  const CUtensorMap *a0, *a1, *a2;
+  const PlaneMaps *ph, *pl;
+  UArgs a;
+  const char* name;   // of the stage, for the stage timers
+};
+
+// Runs stages d[0..n): as one chained launch (up to 16 rows, `chain`; chain_id 0 or 1: which of a
+// step's chains), else one launch each.
+ps_status run_stages(ps_ctx* c, StageDesc* d, int n, bool chain, int chain_id, const FusedScratch& f,
+                     cudaStream_t st) {
+  ps_status s;
+  if (!chain || n < 2) {
+    for (int i = 0; i < n; ++i) {
+      StageDesc& x = d[i];
+      if (x.epi == EPI_STORE) s = launch_umma<EPI_STORE>(c, *x.a0, *x.a1, *x.a2, *x.ph, *x.pl, x.a, f, st);
+      else if (x.epi == EPI_SWIGLU) s = launch_umma<EPI_SWIGLU>(c, *x.a0, *x.a1, *x.a2, *x.ph, *x.pl, x.a, f, st);
+      else s = launch_umma<EPI_LMHEAD>(c, *x.a0, *x.a1, *x.a2, *x.ph, *x.pl, x.a, f, st);
+      if (s) return s;
+      if (x.name) prof_mark(c, st, x.name);
+    }
+    return PS_OK;
+  }
+  if (n > kChainMax) return fail(c, PS_ERR_INVALID_ARG, "too many chained stages");
+  ChainParams p{};
+  p.n = n;
+  // (every chain of a step has counters of its own: a launch may start before the one two ahead of it has ended)
+  p.done = f.chain_ctr + chain_id * 2 * kChainMax;
+  p.passed = p.done + kChainMax;
+  int nm = 0;
+  for (int i = 0; i < n; ++i) {
+    StageDesc& x = d[i];
+    int mi;
+    if ((s = prep_uargs(c, x.a, f, &mi))) return s;
+    if (mi != 0) return fail(c, PS_ERR_INVALID_ARG, "chained stages take up to 16 rows");
+    p.a[i] = x.a;
+    p.epi[i] = x.epi;
+    const CUtensorMap* am[3] = {x.a0, x.a1, x.a2};
+    for (int j = 0; j < 3; ++j) {
+      if (j > 0 && am[j] == am[j - 1]) { p.map_a[i][j] = p.map_a[i][j - 1]; continue; }
+      if (nm >= kChainMaps) return fail(c, PS_ERR_INVALID_ARG, "too many tensor maps in a chain");
+      p.map_a[i][j] = nm;
+      p.maps[nm++] = *am[j];
+    }
+    if (nm + 2 > kChainMaps + (x.a.lo ? 0 : 1)) return fail(c, PS_ERR_INVALID_ARG, "too many tensor maps in a chain");
+    p.map_bh[i] = nm;
+    p.maps[nm++] = x.ph->m[0];
+    p.map_bl[i] = p.map_bh[i];
+    if (x.a.lo) { p.map_bl[i] = nm; p.maps[nm++] = x.pl->m[0]; }
+  }
+  auto kern = k_umma_chain<16>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, umma::kSmemBytes);
+  if (e != cudaSuccess) return cuda_check(c, e, "chain smem attribute");
+  // A dependent launch like the others.  Its CTAs wait for one another: the grid is one CTA per
+  // SM, each filling its SM's shared memory, and a launch's dependents start only once all of
+  // its CTAs have, so on a device that runs nothing else beside this stream all are resident; if
+  // they are not (kernels of other streams holding SMs), the bounded waits expire into
+  // PS_ERR_TIMEOUT.  (A cooperative launch guarantees residency but does not overlap with the
+  // launch before it: measured 15 us slower per step.)
+  e = launch_after(kern, dim3(c->n_sm), dim3(umma::kThreads), umma::kSmemBytes, st, true, p);
+  c->launches++;
+  return cuda_check(c, e, "k_umma_chain");
 }
 
 // ps_kv_append on the tensor-core GEMM: rows [sm.row_base, sm.row_base + rows) of the call's real
@@ -1502,91 +1984,102 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
   typedef const __nv_bfloat16* BP;
   const FusedScratch f = carve_fused(g, (char*)c->fused_scratch);
   const int tiles_h = (H + umma::kTile - 1) / umma::kTile;
+  // up to 16 rows the stages on either side of the attention run as one launch each (the stage
+  // timers need a launch per stage)
+  const bool chain = M <= 16 && !c->prof && !(g.flags & PS_FLAG_STAGE_LAUNCHES);
   ps_status s;
   prof_mark(c, st, "begin");
   const bool no_fc = (g.flags & PS_FLAG_NO_FC) != 0;
+  StageDesc d[kChainMax];
+  int n = 0;
   if (no_fc) {   // embedding-only input: x0 and its planes come straight from the embedding rows
     cudaError_t ee = launch_after(k_embed_x0, dim3(M), dim3(256), 0, st, !c->prof, (BP)w.embed, (BP)w.mask_embed,
                                   token_last, (BP)w.g_in, H, V, R, c->x0, f.x0p.hi, f.x0p.lo, f.ssq[0]);
     c->launches++;
     if (ee != cudaSuccess) return cuda_check(c, ee, "k_embed_x0");
+    prof_mark(c, st, "fc_norm");
   } else {
     cudaError_t ge = launch_after(k_gather_x, dim3(M), dim3(256), 0, st, !c->prof, (BP)w.embed, (BP)w.mask_embed,
                                   (BP)w.mask_feat, (BP)hidden_last, token_last, H, V, R, f.xin);
     c->launches++;
     if (ge != cudaSuccess) return cuda_check(c, ge, "k_gather_x");
-    {  // S1 fc: x0 = W_fc [e ; f] (+ b)
-      UArgs a{};
-      a.N = H; a.K = 2 * H; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 0;
-      a.out = c->x0; a.ldo = H; a.bias = (g.flags & PS_FLAG_FC_BIAS) ? (BP)w.b_fc : nullptr;
-      a.ssq_out = f.ssq[0];
-      a.out_hi = f.x0p.hi; a.out_lo = f.x0p.lo; a.ld_plane = H; a.gain_next = (BP)w.g_in;
-      if ((s = launch_umma<EPI_STORE>(c, u.w_fc, u.w_fc, u.w_fc, u.xin, u.xin, a, f, st))) return s;
-    }
+    // S1 fc: x0 = W_fc [e ; f] (+ b)
+    StageDesc& x = d[n++];
+    x = StageDesc{EPI_STORE, &u.w_fc, &u.w_fc, &u.w_fc, &u.xin, &u.xin, UArgs{}, "fc_norm"};
+    UArgs& a = x.a;
+    a.N = H; a.K = 2 * H; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 0;
+    a.out = c->x0; a.ldo = H; a.bias = (g.flags & PS_FLAG_FC_BIAS) ? (BP)w.b_fc : nullptr;
+    a.ssq_out = f.ssq[0];
+    a.out_hi = f.x0p.hi; a.out_lo = f.x0p.lo; a.ld_plane = H; a.gain_next = (BP)w.g_in;
   }
-  prof_mark(c, st, "fc_norm");
   {  // S2 q|k|v = W rms(x0)
-    UArgs a{};
+    StageDesc& x = d[n++];
+    x = StageDesc{EPI_STORE, &u.w_q, &u.w_k, &u.w_v, &u.x0_hi, &u.x0_lo, UArgs{}, "qkv_rope"};
+    UArgs& a = x.a;
     a.N = Hq + 2 * Hkv; a.K = H; a.M = M; a.n_mats = 3;
     a.mat_rows[0] = Hq; a.mat_rows[1] = Hkv; a.mat_rows[2] = Hkv; a.lo = 1;
     a.ssq_in = f.ssq[0]; a.ssq_n = no_fc ? 1 : tiles_h; a.eps = g.rms_eps;
     a.out = f.qkv; a.ldo = Hq + 2 * Hkv;
-    if ((s = launch_umma<EPI_STORE>(c, u.w_q, u.w_k, u.w_v, u.x0_hi, u.x0_lo, a, f, st))) return s;
   }
-  prof_mark(c, st, "qkv_rope");
+  if ((s = run_stages(c, d, n, chain, 0, f, st))) return s;
   if ((s = launch_attn_split(c, sm, B, f.qkv, f.att_ml, f.att_o, f.attn_tickets, f.attnp.hi, f.attnp.lo, st)))
     return s;
   prof_mark(c, st, "attention");
+  n = 0;
   {  // S4 a = x0 + W_o attn
-    UArgs a{};
+    StageDesc& x = d[n++];
+    x = StageDesc{EPI_STORE, &u.w_o, &u.w_o, &u.w_o, &u.attn_hi, &u.attn_lo, UArgs{}, "o_proj"};
+    UArgs& a = x.a;
     a.N = H; a.K = Hq; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 1;
     a.out = c->a; a.ldo = H; a.res = c->x0; a.ldr = H;
     a.ssq_out = f.ssq[1];
     a.out_hi = f.ap.hi; a.out_lo = f.ap.lo; a.ld_plane = H; a.gain_next = (BP)w.g_post;
-    if ((s = launch_umma<EPI_STORE>(c, u.w_o, u.w_o, u.w_o, u.attn_hi, u.attn_lo, a, f, st))) return s;
   }
-  prof_mark(c, st, "o_proj");
   {  // S5a act = silu(W_g rms(a)) * (W_u rms(a))
-    UArgs a{};
+    StageDesc& x = d[n++];
+    x = StageDesc{EPI_SWIGLU, &u.w_gate, &u.w_up, &u.w_up, &u.a_hi, &u.a_lo, UArgs{}, "ffn_gate_up"};
+    UArgs& a = x.a;
     a.N = F; a.K = H; a.M = M; a.zip = 1; a.n_mats = 2; a.lo = 1;
     a.ssq_in = f.ssq[1]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
     a.out = f.act; a.ldo = F;
     a.out_hi = f.actp.hi; a.out_lo = f.actp.lo; a.ld_plane = F;
-    if ((s = launch_umma<EPI_SWIGLU>(c, u.w_gate, u.w_up, u.w_up, u.a_hi, u.a_lo, a, f, st))) return s;
   }
-  prof_mark(c, st, "ffn_gate_up");
   float* hdn = feat_out ? feat_out : c->hdn;
   {  // S5b hdn = a + W_d act
-    UArgs a{};
+    StageDesc& x = d[n++];
+    x = StageDesc{EPI_STORE, &u.w_down, &u.w_down, &u.w_down, &u.act_hi, &u.act_lo, UArgs{}, "ffn_down"};
+    UArgs& a = x.a;
     a.N = H; a.K = F; a.M = M; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 1;
     a.out = hdn; a.ldo = H; a.res = c->a; a.ldr = H;
     a.ssq_out = f.ssq[2];
     a.out_hi = f.hdnp.hi; a.out_lo = f.hdnp.lo; a.ld_plane = H; a.gain_next = (BP)w.g_final;
-    if ((s = launch_umma<EPI_STORE>(c, u.w_down, u.w_down, u.w_down, u.act_hi, u.act_lo, a, f, st))) return s;
   }
-  prof_mark(c, st, "ffn_down");
-  if (M > 32 && logits_out) {
-    // S6 with many rows and the logits kept: the row statistics in the tile epilogue cost more
-    // than the weights' streaming then (they are serial in the rows), so the GEMM only stores
-    // the logits and one block per row reads them back from L2
-    UArgs a{};
+  const bool stats_pass = M > 32 && logits_out;
+  {
+    StageDesc& x = d[n++];
+    x = StageDesc{stats_pass ? EPI_STORE : EPI_LMHEAD, &u.w_lm, &u.w_lm, &u.w_lm, &u.hdn_hi, &u.hdn_lo, UArgs{}, "lm_head"};
+    UArgs& a = x.a;
     a.N = V; a.K = H; a.M = M; a.n_mats = 1; a.mat_rows[0] = V; a.lo = 1;
     a.ssq_in = f.ssq[2]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
-    a.out = logits_out; a.ldo = V;
-    if ((s = launch_umma<EPI_STORE>(c, u.w_lm, u.w_lm, u.w_lm, u.hdn_hi, u.hdn_lo, a, f, st))) return s;
+    if (stats_pass) {
+      // S6 with many rows and the logits kept: the row statistics in the tile epilogue cost more
+      // than the weights' streaming then (they are serial in the rows), so the GEMM only stores
+      // the logits and one block per row reads them back from L2
+      a.out = logits_out; a.ldo = V;
+      x.name = nullptr;   // (timed together with the statistics pass below)
+    } else {  // S6 logits = W_lm rms(hdn), softmax statistics and top-n without a second pass over logits
+      a.logits_out = logits_out; a.parts = f.parts; a.ticket = f.ticket;
+      a.top_n = top_n; a.top_ids = top_ids; a.top_logit = top_logit; a.row_max = row_max; a.row_lse = row_lse;
+      a.R = R;
+      if (sa) { a.sample = 1; a.sa = *sa; }
+    }
+  }
+  if ((s = run_stages(c, d, n, chain, 1, f, st))) return s;
+  if (stats_pass) {
     if ((s = launch_row_stats(c, logits_out, M, V, top_n, top_ids, top_logit, row_max, row_lse, st))) return s;
     if (sa && (s = launch_gumbel_argmax(c, logits_out, M, V, R, *sa, st))) return s;
-  } else {  // S6 logits = W_lm rms(hdn), softmax statistics and top-n without a second pass over logits
-    UArgs a{};
-    a.N = V; a.K = H; a.M = M; a.n_mats = 1; a.mat_rows[0] = V; a.lo = 1;
-    a.ssq_in = f.ssq[2]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
-    a.logits_out = logits_out; a.parts = f.parts; a.ticket = f.ticket;
-    a.top_n = top_n; a.top_ids = top_ids; a.top_logit = top_logit; a.row_max = row_max; a.row_lse = row_lse;
-    a.R = R;
-    if (sa) { a.sample = 1; a.sa = *sa; }
-    if ((s = launch_umma<EPI_LMHEAD>(c, u.w_lm, u.w_lm, u.w_lm, u.hdn_hi, u.hdn_lo, a, f, st))) return s;
+    prof_mark(c, st, "lm_head");
   }
-  prof_mark(c, st, "lm_head");
   return PS_OK;
 }
 

@@ -42,6 +42,7 @@ namespace umma {
 using ws::mbar_arrive;
 using ws::mbar_arrive_expect_tx;
 using ws::mbar_init;
+using ws::mbar_peek;
 using ws::mbar_wait;
 using ws::smem_u32;
 

@@ -54,10 +54,12 @@ def test_mini32_ragged_batch():
     _compare_step(p, top_n=8)
 
 
-@pytest.mark.parametrize("flags", [0, 2, 4], ids=["tcgen05", "unfused", "mma_sync"])
+@pytest.mark.parametrize("flags", [0, 16, 2, 4], ids=["tcgen05", "stage_launches", "unfused", "mma_sync"])
 def test_mini_bf16_ragged_batch(flags):
-    """The bf16 shape on each of the three kernel sets the library holds: the tcgen05 GEMMs, the
-    plain one-kernel-per-stage path (PS_FLAG_UNFUSED_KERNELS) and the mma.sync weight-streaming
+    """The bf16 shape on each of the kernel sets the library holds: the tcgen05 GEMMs with the
+    stages on either side of the attention chained into one launch each (15 rows: some CTAs of a
+    chain have no unit in a stage) or launched one by one (PS_FLAG_STAGE_LAUNCHES), the plain
+    one-kernel-per-stage path (PS_FLAG_UNFUSED_KERNELS) and the mma.sync weight-streaming
     GEMMs (PS_FLAG_MMA_SYNC_GEMM); contexts built by ps_kv_append on the same path."""
     s = synth.CONFIGS["mini"]
     p = Pair(s, s.batch, flags=flags)
@@ -196,6 +198,38 @@ def test_full_size_batch1(name):
     Kg, Vg = Kg.float().cpu().numpy(), Vg.float().cpu().numpy()
     assert (np.abs(Kg[L:] - Ko[L:]) <= 2.0 ** -7 * np.abs(Ko[L:]) + 1e-2).all()
     assert (np.abs(Vg[L:] - Vo[L:]) <= 2.0 ** -7 * np.abs(Vo[L:]) + 1e-2).all()
+
+
+@pytest.mark.parametrize("name,B", [("mini", 3), ("7b", 1)])
+def test_chained_stages_equal_stage_launches(name, B):
+    """Up to 16 rows the GEMM stages before and after the attention share a launch.  The sums are
+    the same sums in the same order as with one launch per stage (PS_FLAG_STAGE_LAUNCHES), so
+    every output is equal bit for bit; forty chained steps in a row leave the stage counters
+    as they found them (equal outputs every time, no expired wait)."""
+    import paper_2410_05589_b200 as ps
+    s = synth.CONFIGS[name]
+    W = synth.weights(s)
+    lens = synth.ctx_lengths(s, B)
+    outs = []
+    for flags in (0, 16):
+        g = ps.drafter_from_shape(s, W, max_batch=B, max_ctx=int(lens.max()) + s.rows + 1, flags=flags)
+        for b in range(B):
+            K, V = synth.kv_rows(s, ("kv", b), int(lens[b]))
+            g.kv_import(b, ps.to_device(K), ps.to_device(V))
+        hl, tl = ps.to_device(synth.hidden_states(s, "last", B)), ps.to_device(synth.token_ids(s, "last", B))
+        first = None
+        for it in range(40 if flags == 0 else 1):
+            o = g.draft_step(list(range(B)), hl, tl, top_n=4, want_logits=True, want_feat=True)
+            cur = {k: o[k].cpu().numpy().copy() for k in ("logits", "feat", "top_ids", "top_logit", "row_max", "row_lse")}
+            if first is None:
+                first = cur
+            else:
+                for k in cur:
+                    assert np.array_equal(cur[k], first[k]), (it, k)
+        assert g.poll() == 0
+        outs.append(first)
+    for k in outs[0]:
+        assert np.array_equal(outs[0][k], outs[1][k]), k
 
 
 _W13 = {}

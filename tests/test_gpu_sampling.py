@@ -50,10 +50,11 @@ def _check_rows(s, got, want_logits_of, T, seed, offset, B):
                 assert margin[0] <= 2 * tol, (b, j, tok, int(t_o[0]), margin[0])
 
 
-@pytest.mark.parametrize("name,B,flags", [("mini", 3, 0), ("tiny", 1, 0), ("mini", 1, 0), ("mini", 3, 4), ("mini", 2, 2)])
+@pytest.mark.parametrize("name,B,flags", [("mini", 3, 0), ("tiny", 1, 0), ("mini", 1, 0), ("mini", 3, 4), ("mini", 2, 2), ("mini", 3, 16)])
 def test_sampled_tokens_match_oracle(name, B, flags):
-    """flags 4 / 2: the mma.sync GEMMs and the plain kernels, where one block per row draws the
-    token from the stored logits."""
+    """flags 16: one launch per GEMM stage instead of the chained stages; flags 4 / 2: the
+    mma.sync GEMMs and the plain kernels, where one block per row draws the token from the
+    stored logits."""
     s = synth.CONFIGS[name]
     p = Pair(s, B, flags=flags)
     T, seed, offset = 0.8, 5, 12
