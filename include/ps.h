@@ -312,7 +312,10 @@ ps_status ps_debug_wait_expires(ps_ctx* ctx, long long limit_cycles, void* strea
 long long ps_launch_count(ps_ctx* ctx);
 
 /* Stage timing.  ps_profile(ctx, 1) makes every later call record a CUDA event after each
- * stage it enqueues (a few microseconds of overhead per stage); ps_profile(ctx, 0) stops.
+ * stage it enqueues (a few microseconds of overhead per stage; every GEMM stage gets a launch
+ * of its own, as with PS_FLAG_STAGE_LAUNCHES); ps_profile(ctx, 2) records an event after each
+ * launch instead and leaves chained stages chained: their intervals are named "chain_fc_qkv"
+ * and "chain_o_ffn_lm"; ps_profile(ctx, 0) stops.
  * ps_profile_read waits for the recorded events and returns, per stage name, the summed time
  * and the number of intervals since profiling was switched on or last read.
  *   names     host [max_stages][32] chars;  total_ms, count: host [max_stages];  n_stages: host */

@@ -386,8 +386,9 @@ class Drafter:
         """Waits for the stream and returns the device status (PS_OK, PS_ERR_NONFINITE, ...)."""
         return self.lib.ps_poll(self.h, _stream())
 
-    def profile(self, enable: bool) -> None:
-        self._check(self.lib.ps_profile(self.h, 1 if enable else 0))
+    def profile(self, enable) -> None:
+        """ps_profile: False / 0 off, True / 1 an event per stage, 2 an event per launch."""
+        self._check(self.lib.ps_profile(self.h, int(enable)))
 
     def profile_read(self) -> dict:
         """{stage: (total_ms, intervals)} since profiling was enabled or last read."""

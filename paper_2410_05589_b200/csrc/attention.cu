@@ -113,9 +113,7 @@ __global__ void __launch_bounds__(kAttnThreads, NB == 1 ? 3 : 2) k_attn_mma(
   };
   pdl_launch_dependents();
   if (t_begin < t_end) stage(t_begin, min(tile, t_end - t_begin));   // the cache is older than the launch before
-  pdl_wait();   // q, k and v of the new rows come from the kernel before this one
-
-  // rotation table of the R new positions, then q: rotated, scaled, split into hi/lo planes
+  // rotation table of the R new positions (needs nothing of the kernel before this one)
   for (int idx = tid; idx < R * HALF; idx += kAttnThreads) {
     const int j = idx / HALF, i = idx - j * HALF;
     double ang = (double)(L + j) * inv_freq[i];
@@ -125,6 +123,9 @@ __global__ void __launch_bounds__(kAttnThreads, NB == 1 ? 3 : 2) k_attn_mma(
     s_cs[idx] = cs;
     s_sn[idx] = sn;
   }
+  pdl_wait();   // q, k and v of the new rows come from the kernel before this one
+
+  // q: rotated, scaled, split into hi/lo planes
   __syncthreads();
   const float scale = rsqrtf((float)D);
   for (int idx = tid; idx < RB * HALF; idx += kAttnThreads) {
@@ -328,21 +329,44 @@ __global__ void __launch_bounds__(kAttnThreads, NB == 1 ? 3 : 2) k_attn_mma(
   }
   __syncthreads();
   if (s_last) {
-    for (int idx = tid; idx < R * D; idx += kAttnThreads) {
-      const int j = idx / D, d = idx - j * D;
-      const size_t rec0 = ((size_t)(m0 + j) * n_heads + h) * n_split;
-      const volatile float* ml = att_ml + rec0 * 2;
-      float mxs = -FLT_MAX;
-      for (int s = 0; s < n_split; ++s) mxs = fmaxf(mxs, ml[2 * s]);
-      float den = 0.f, num = 0.f;
-      for (int s = 0; s < n_split; ++s) {
-        const float w = __expf(ml[2 * s] - mxs);
-        den += w * ml[2 * s + 1];
-        num += w * ((const volatile float*)att_o)[(rec0 + s) * D + d];
+    // This code runs once per (sequence, head), after everything else: what it costs is round
+    // trips to L2 and the fetch of its own instructions, so it is a few small rolled loops.
+    // All splits' partial outputs of a row are one contiguous block: asynchronous 16-byte
+    // copies bring the rows into the shared memory of the (finished) K / V tiles, as many rows
+    // per pass as fit, in one round trip; the (max, sum) pairs go to the q planes' place.
+    float* s_o = reinterpret_cast<float*>(att_smem);     // [rows of a pass][n_split][D]
+    float2* s_ml = reinterpret_cast<float2*>(s_qh);      // [R][n_split]
+    const int row_f = n_split * D;                        // floats per row
+    const int rows_pass = max(1, (2 * tile * P * 2) / (row_f * 4));
+    const float2* ml2 = reinterpret_cast<const float2*>(att_ml);
+    for (int idx = tid; idx < R * n_split; idx += kAttnThreads) {
+      const int j = idx / n_split, sp = idx - j * n_split;
+      s_ml[idx] = __ldcg(ml2 + ((size_t)(m0 + j) * n_heads + h) * n_split + sp);
+    }
+    for (int j0 = 0; j0 < R; j0 += rows_pass) {
+      const int nr = min(rows_pass, R - j0), vec_row = row_f / 4;
+      for (int idx = tid; idx < nr * vec_row; idx += kAttnThreads) {
+        const int jr = idx / vec_row, off = (idx - jr * vec_row) * 4;
+        cp_async16(s_o + jr * row_f + off, att_o + ((size_t)(m0 + j0 + jr) * n_heads + h) * row_f + off);
       }
-      const float x = num / den;
-      const size_t at = (size_t)(m0 + j) * n_heads * D + h * D + d;
-      split_bf16(x, out_hi[at], out_lo[at]);
+      asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+      __syncthreads();
+      for (int idx = tid; idx < nr * D; idx += kAttnThreads) {
+        const int jr = idx / D, d = idx - jr * D, j = j0 + jr;
+        const float2* ml = s_ml + j * n_split;
+        float mxs = -FLT_MAX;
+        for (int sp = 0; sp < n_split; ++sp) mxs = fmaxf(mxs, ml[sp].x);
+        float den = 0.f, num = 0.f;
+        for (int sp = 0; sp < n_split; ++sp) {
+          const float w = __expf(ml[sp].x - mxs);
+          den += w * ml[sp].y;
+          num += w * s_o[jr * row_f + sp * D + d];
+        }
+        const float x = num / den;
+        const size_t at = (size_t)(m0 + j) * n_heads * D + h * D + d;
+        split_bf16(x, out_hi[at], out_lo[at]);
+      }
+      __syncthreads();
     }
   }
 }

@@ -1928,7 +1928,7 @@ ps_status run_stages(ps_ctx* c, StageDesc* d, int n, bool chain, int chain_id, c
   // they are not (kernels of other streams holding SMs), the bounded waits expire into
   // PS_ERR_TIMEOUT.  (A cooperative launch guarantees residency but does not overlap with the
   // launch before it: measured 15 us slower per step.)
-  e = launch_after(kern, dim3(c->n_sm), dim3(umma::kThreads), umma::kSmemBytes, st, true, p);
+  e = launch_after(kern, dim3(c->n_sm), dim3(umma::kThreads), umma::kSmemBytes, st, !c->prof, p);
   c->launches++;
   return cuda_check(c, e, "k_umma_chain");
 }
@@ -1986,7 +1986,7 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
   const int tiles_h = (H + umma::kTile - 1) / umma::kTile;
   // up to 16 rows the stages on either side of the attention run as one launch each (the stage
   // timers need a launch per stage)
-  const bool chain = M <= 16 && !c->prof && !(g.flags & PS_FLAG_STAGE_LAUNCHES);
+  const bool chain = M <= 16 && (!c->prof || c->prof_launches) && !(g.flags & PS_FLAG_STAGE_LAUNCHES);
   ps_status s;
   prof_mark(c, st, "begin");
   const bool no_fc = (g.flags & PS_FLAG_NO_FC) != 0;
@@ -2022,6 +2022,7 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
     a.out = f.qkv; a.ldo = Hq + 2 * Hkv;
   }
   if ((s = run_stages(c, d, n, chain, 0, f, st))) return s;
+  if (chain && n > 1) prof_mark(c, st, "chain_fc_qkv");
   if ((s = launch_attn_split(c, sm, B, f.qkv, f.att_ml, f.att_o, f.attn_tickets, f.attnp.hi, f.attnp.lo, st)))
     return s;
   prof_mark(c, st, "attention");
@@ -2075,6 +2076,7 @@ ps_status umma_draft_step(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int B,
     }
   }
   if ((s = run_stages(c, d, n, chain, 1, f, st))) return s;
+  if (chain) prof_mark(c, st, "chain_o_ffn_lm");
   if (stats_pass) {
     if ((s = launch_row_stats(c, logits_out, M, V, top_n, top_ids, top_logit, row_max, row_lse, st))) return s;
     if (sa && (s = launch_gumbel_argmax(c, logits_out, M, V, R, *sa, st))) return s;

@@ -204,6 +204,7 @@ void ps_destroy(ps_ctx* c) {
 ps_status ps_profile(ps_ctx* c, int enable) {
   if (!c) return PS_ERR_INVALID_ARG;
   c->prof = enable != 0;
+  c->prof_launches = enable == 2;
   c->prof_used = 0;
   return PS_OK;
 }

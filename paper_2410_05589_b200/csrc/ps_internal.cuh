@@ -155,6 +155,7 @@ struct ps_ctx {
   std::string err;
   // optional stage timing (ps_profile): events recorded between stages
   bool prof = false;
+  bool prof_launches = false;   // events per launch: chained stages stay chained (ps_profile(ctx, 2))
   std::vector<cudaEvent_t> prof_ev;
   std::vector<const char*> prof_name;   // name of the stage that ENDS at the event
   size_t prof_used = 0;
