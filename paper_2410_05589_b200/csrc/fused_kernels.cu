@@ -807,8 +807,12 @@ __device__ __forceinline__ void big_chunk_epilogue(const UArgs& a, umma::Ctl& ct
 }
 
 // Last step of an LM-head launch, called by all threads of every CTA after its tiles are done:
-// the last CTA to finish merges the per-tile summaries (no CTA waits for another).
-__device__ __forceinline__ void lm_merge(const UArgs& a, umma::Ctl& ctl, int tid, int warp, int lane) {
+// the last CTA to finish merges the per-tile summaries (no CTA waits for another).  It runs
+// once, after everything else, so what it costs is round trips to L2 and the fetch of its own
+// instructions: the summaries of as many rows as fit come into the (idle) ring by asynchronous
+// 16-byte copies in one round trip, then a warp per row reduces them in small rolled loops.
+__device__ __forceinline__ void lm_merge(const UArgs& a, umma::Ctl& ctl, unsigned char* ring, int tid, int warp,
+                                         int lane) {
   if (tid == 0) {
     __threadfence();
     const unsigned tk = atomicAdd(a.ticket, 1u);
@@ -817,96 +821,92 @@ __device__ __forceinline__ void lm_merge(const UArgs& a, umma::Ctl& ctl, int tid
   }
   __syncthreads();
   if (ctl.is_last && !ctl.abort_flag) {
-    // all six warps, one activation row each; the loops are unrolled so that the loads of
-    // eight tiles are in flight together (they come from L2, written by other SMs)
     const int Gt = a.n_tiles;
-    for (int m = warp; m < a.M; m += umma::kThreads / 32) {
-      const LmPart* P = a.parts + m;
-      // 256 tiles per round, 8 per lane, their loads issued together.  The first round also
-      // fetches every tile's best token: the row's arg-max needs nothing else.
-      float mx = -FLT_MAX, se = 0.f;
-      float bv0 = -FLT_MAX; int bi0 = 0x7fffffff;
-      for (int c0 = 0; c0 < Gt; c0 += 256) {
-        float vm[8], sx[8], tv[8]; int ti[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int c = c0 + lane + 32 * j;
-          float4 hd = make_float4(-FLT_MAX, 0.f, -FLT_MAX, __int_as_float(0x7fffffff));
-          if (c < Gt) hd = __ldcg(reinterpret_cast<const float4*>(&P[(size_t)c * a.M]));
-          vm[j] = hd.x; sx[j] = hd.y; tv[j] = hd.z;
-          ti[j] = a.top_n > 0 ? __float_as_int(hd.w) : 0x7fffffff;
+    static_assert(offsetof(LmPart, sv) % 16 == 0, "the sample pair starts a 16-byte group");
+    const int rows_pass = max(1, min(a.M, umma::kRingBytes / (Gt * 32)));
+    float4* s_h = reinterpret_cast<float4*>(ring);   // [rows of a pass][Gt]: vmax, sumexp, v0, i0
+    float4* s_s = s_h + rows_pass * Gt;              // [rows of a pass][Gt]: sv, si
+    for (int m0 = 0; m0 < a.M; m0 += rows_pass) {
+      const int nr = min(rows_pass, a.M - m0);
+      for (int mr = 0; mr < nr; ++mr) {
+        for (int c = tid; c < Gt; c += umma::kThreads) {
+          const LmPart* e = a.parts + (size_t)c * a.M + m0 + mr;
+          umma::cp_async_16(s_h + mr * Gt + c, e);
+          if (a.sample) umma::cp_async_16(s_s + mr * Gt + c, &e->sv);
         }
-        float nm = mx;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          nm = fmaxf(nm, vm[j]);
-          if (ti[j] != 0x7fffffff && (tv[j] > bv0 || (tv[j] == bv0 && ti[j] < bi0))) { bv0 = tv[j]; bi0 = ti[j]; }
+      }
+      umma::cp_async_wait_all();
+      __syncthreads();
+      for (int mr = warp; mr < nr; mr += umma::kThreads / 32) {
+        const int m = m0 + mr;
+        const float4* H = s_h + mr * Gt;
+        float mx = -FLT_MAX;
+        float bv0 = -FLT_MAX; int bi0 = 0x7fffffff;   // the row's arg-max: the tiles' best tokens decide it
+        for (int c = lane; c < Gt; c += 32) {
+          const float4 hd = H[c];
+          mx = fmaxf(mx, hd.x);
+          const int ti = __float_as_int(hd.w);
+          if (a.top_n > 0 && (hd.z > bv0 || (hd.z == bv0 && ti < bi0))) { bv0 = hd.z; bi0 = ti; }
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) nm = fmaxf(nm, __shfl_xor_sync(0xffffffffu, nm, o));
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         float add = 0.f;
+        for (int c = lane; c < Gt; c += 32) add += H[c].y * __expf(H[c].x - mx);
+        const float se = warp_sum(add);
+        if (lane == 0) {
+          if (a.row_max) a.row_max[m] = mx;
+          if (a.row_lse) a.row_lse[m] = mx + logf(se);
+        }
+        const LmPart* P = a.parts + m;
+        float pv = FLT_MAX; int pi = -1;
+        for (int tn = 0; tn < a.top_n; ++tn) {
+          float bv = bv0; int bi = bi0;
+          if (tn > 0) {   // deeper picks: a tile's list is sorted, any of its entries may be next
+            bv = -FLT_MAX; bi = 0x7fffffff;
+            for (int k = 0; k < a.top_n; ++k) {
+              for (int c0 = 0; c0 < Gt; c0 += 256) {
+                float xv[8]; int id[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) add += sx[j] * __expf(vm[j] - nm);
-        se = se * __expf(mx - nm) + warp_sum(add);
-        mx = nm;
-      }
-      if (lane == 0) {
-        if (a.row_max) a.row_max[m] = mx;
-        if (a.row_lse) a.row_lse[m] = mx + logf(se);
-      }
-      float pv = FLT_MAX; int pi = -1;
-      for (int tn = 0; tn < a.top_n; ++tn) {
-        float bv = bv0; int bi = bi0;
-        if (tn > 0) {   // deeper picks: a tile's list is sorted, any of its entries may be next
-          bv = -FLT_MAX; bi = 0x7fffffff;
-          for (int k = 0; k < a.top_n; ++k) {
-            for (int c0 = 0; c0 < Gt; c0 += 256) {
-              float xv[8]; int id[8];
+                for (int j = 0; j < 8; ++j) {
+                  const int c = c0 + lane + 32 * j;
+                  xv[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_v[k]) : 0.f;
+                  id[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_i[k]) : 0x7fffffff;
+                }
 #pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                const int c = c0 + lane + 32 * j;
-                xv[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_v[k]) : 0.f;
-                id[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].top_i[k]) : 0x7fffffff;
-              }
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                const bool after = id[j] != 0x7fffffff && ((xv[j] < pv) || (xv[j] == pv && id[j] > pi));
-                if (after && (xv[j] > bv || (xv[j] == bv && id[j] < bi))) { bv = xv[j]; bi = id[j]; }
+                for (int j = 0; j < 8; ++j) {
+                  const bool after = id[j] != 0x7fffffff && ((xv[j] < pv) || (xv[j] == pv && id[j] > pi));
+                  if (after && (xv[j] > bv || (xv[j] == bv && id[j] < bi))) { bv = xv[j]; bi = id[j]; }
+                }
               }
             }
           }
-        }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-          if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+          }
+          if (lane == 0) { a.top_ids[(size_t)m * a.top_n + tn] = bi; a.top_logit[(size_t)m * a.top_n + tn] = bv; }
+          pv = bv; pi = bi;
         }
-        if (lane == 0) { a.top_ids[(size_t)m * a.top_n + tn] = bi; a.top_logit[(size_t)m * a.top_n + tn] = bv; }
-        pv = bv; pi = bi;
-      }
-      if (a.sample) {   // the row's sampled token: arg-max of the ranges' perturbed maxima
-        float bv = -FLT_MAX; int bi = 0x7fffffff;
-        for (int c0 = 0; c0 < Gt; c0 += 256) {
-          float xv[8]; int id[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int c = c0 + lane + 32 * j;
-            xv[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].sv) : -FLT_MAX;
-            id[j] = c < Gt ? __ldcg(&P[(size_t)c * a.M].si) : 0x7fffffff;
+        if (a.sample) {   // the row's sampled token: arg-max of the ranges' perturbed maxima
+          const float4* S = s_s + mr * Gt;
+          float bv = -FLT_MAX; int bi = 0x7fffffff;
+          for (int c = lane; c < Gt; c += 32) {
+            const float xv = S[c].x;
+            const int id = __float_as_int(S[c].y);
+            if (xv > bv || (xv == bv && id < bi)) { bv = xv; bi = id; }
           }
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (xv[j] > bv || (xv[j] == bv && id[j] < bi)) { bv = xv[j]; bi = id[j]; }
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+          }
+          if (lane == 0) a.sa.sampled[m] = bi;
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-          if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
-        if (lane == 0) a.sa.sampled[m] = bi;
       }
+      __syncthreads();   // the next pass overwrites the ring
     }
   }
   if (ctl.is_last && tid == 0) *a.ticket = 0u;
@@ -1241,7 +1241,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
   }
 
   __syncthreads();
-  if (EPI == EPI_LMHEAD) lm_merge(a, ctl, tid, warp, lane);
+  if (EPI == EPI_LMHEAD) lm_merge(a, ctl, stages, tid, warp, lane);
   if (ctl.abort_flag) {
     // let copies and MMAs that are still in flight finish before shared and tensor memory go
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);
@@ -1641,7 +1641,7 @@ __global__ void __launch_bounds__(umma::kThreads, 1) k_umma_chain(const __grid_c
   }
 
   __syncthreads();
-  if (p.epi[p.n - 1] == EPI_LMHEAD) lm_merge(p.a[p.n - 1], ctl, tid, warp, lane);
+  if (p.epi[p.n - 1] == EPI_LMHEAD) lm_merge(p.a[p.n - 1], ctl, stages, tid, warp, lane);
   if (ctl.abort_flag) {
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     if (tid == 0) atomicOr(p.a[0].status, kStatTimeout);
@@ -2108,6 +2108,7 @@ bool fused_supported(ps_ctx* c, int M) {
   if (M > umma::kMaxRows || (g.head_dim != 64 && g.head_dim != 128)) return false;
   const int Hq = g.n_heads * g.head_dim;
   if (g.hidden % 8 || Hq % 8 || g.ffn % 8) return false;   // 16-byte operand rows
+  if ((g.vocab + 127) / 128 > umma::kRingBytes / 32) return false;   // a row's tile summaries fit the ring (LM-head merge)
   ensure_maps(c);
   if (c->umma_maps) return true;
   if (M > kMaxM) return false;   // the mma.sync kernels take 16 rows
