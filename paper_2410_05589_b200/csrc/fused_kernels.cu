@@ -1539,14 +1539,26 @@ __global__ void __launch_bounds__(umma::kThreads, 1) k_umma_chain(const __grid_c
         const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + buf * acols;
         float v[16];
         if (!dry) {   // the tile's sums over this CTA's k-blocks: the accumulators and their hi / lo halves
-          tmem_ld16(ta, v);
+          // (the ksplit accumulators, hi half then lo half each, are 2 ksplit MP consecutive columns:
+          // two loads bring them all, one wait)
+          static_assert(2 * ksplit * MP == 128, "accumulators of a tile span 128 columns");
+          float w0[64], w1[64];
+          tmem_ld64(ta, w0);
+          tmem_ld64(ta + 64, w1);
+          tmem_ld_wait();
+          const bool lo = a.lo != 0;
 #pragma unroll
-          for (int c = 1; c < 2 * ksplit; ++c) {
-            if (!a.lo && (c & 1)) continue;
-            float vp[16];
-            tmem_ld16(ta + (c >> 1) * 2 * MP + (c & 1) * MP, vp);
-#pragma unroll
-            for (int m = 0; m < 16; ++m) v[m] += vp[m];
+          for (int m = 0; m < 16; ++m) {
+            // same order of additions as one load per group: acc0.hi, acc0.lo, acc1.hi, ...
+            float x = w0[m];
+            if (lo) x += w0[16 + m];
+            x += w0[32 + m];
+            if (lo) x += w0[48 + m];
+            x += w1[m];
+            if (lo) x += w1[16 + m];
+            x += w1[32 + m];
+            if (lo) x += w1[48 + m];
+            v[m] = x;
           }
           fence_before_sync();
           mbar_arrive(&ctl.acc_empty[buf]);   // the accumulator is read: the MMA warp may reuse it
