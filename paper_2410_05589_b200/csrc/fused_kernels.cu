@@ -1538,6 +1538,8 @@ __global__ void __launch_bounds__(umma::kThreads, 1) k_umma_chain(const __grid_c
         fence_after_sync();
         const uint32_t ta = tmem + ((uint32_t)(32 * q) << 16) + buf * acols;
         float v[16];
+#pragma unroll
+        for (int m = 0; m < 16; ++m) v[m] = 0.f;
         if (!dry) {   // the tile's sums over this CTA's k-blocks: the accumulators and their hi / lo halves
           // (the ksplit accumulators, hi half then lo half each, are 2 ksplit MP consecutive columns:
           // two loads bring them all, one wait)
@@ -1564,35 +1566,43 @@ __global__ void __launch_bounds__(umma::kThreads, 1) k_umma_chain(const __grid_c
           mbar_arrive(&ctl.acc_empty[buf]);   // the accumulator is read: the MMA warp may reuse it
         }
         bool finish = whole || dry;
+        // The CTA that owns the tile's last k-block finishes the tile.  The others store their
+        // partial and count themselves in (release); one thread of the finisher waits for the
+        // count (acquire, bounded) while its own sums stay in registers.
         if (!whole && !dry) {
-          float4* d4 = reinterpret_cast<float4*>(P + r * 16);
+          if (blockIdx.x != c_last) {
+            float4* d4 = reinterpret_cast<float4*>(P + r * 16);
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            if (i < nvec) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-          epi_sync();
-          if (et == 0) {
-            // one thread publishes the block's partial (the barrier above ordered the other
-            // threads' stores before this release) and, if it came last, acquires the others'
-            int n_contrib = 0;
-            for (int j = 0; j <= c_last - c_first; ++j) n_contrib += ctl.coff[j] >= 0;
-            unsigned old;
-            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(&a.tile_tickets[t]) : "memory");
-            const int last = old == (unsigned)(n_contrib - 1);
-            if (last) a.tile_tickets[t] = 0u;
-            ctl.tile_last = last;
+            for (int i = 0; i < 4; ++i)
+              if (i < nvec) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            epi_sync();   // (orders the other threads' stores before the release below)
+            if (et == 0) {
+              __threadfence();
+              atomicAdd(&a.tile_tickets[t], 1u);
+            }
+          } else {
+            if (et == 0) {
+              unsigned n_other = 0;
+              for (int j = 0; j < c_last - c_first; ++j) n_other += ctl.coff[j] >= 0;
+              const long long t0 = clock64();
+              while (ld_acquire_u32(&a.tile_tickets[t]) < n_other) {
+                if (*abort_flag || clock64() - t0 > ws::kWaitCycles) { *abort_flag = 1; break; }
+              }
+              a.tile_tickets[t] = 0u;   // everyone has counted itself in
+            }
+            epi_sync();
+            finish = true;
           }
-          epi_sync();
-          finish = ctl.tile_last != 0;
-          epi_sync();   // everyone has read the flag before a later segment rewrites it
         }
         if (finish) {
           if (!whole) {
             // the partials added in CTA order (the sum does not depend on who came last), all of
             // up to four contributors' vectors in flight together
-            const int nc = c_last - c_first + 1;
+            const int nc = dry ? 1 : c_last - c_first;   // (the rehearsal reads this CTA's own slot)
             const float* Pr = a.partials + r * 16;
+            float own[16];
 #pragma unroll
-            for (int m = 0; m < 16; ++m) v[m] = 0.f;
+            for (int m = 0; m < 16; ++m) { own[m] = v[m]; v[m] = 0.f; }
             const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
             if (mc <= 8) {
 #pragma unroll 1
@@ -1631,6 +1641,8 @@ __global__ void __launch_bounds__(umma::kThreads, 1) k_umma_chain(const __grid_c
                   }
               }
             }
+#pragma unroll
+            for (int m = 0; m < 16; ++m) v[m] += own[m];   // the finisher is the last in CTA order
           }
 #pragma unroll
           for (int m = 0; m < 16; ++m) ctl.acc[m * 128 + r] = v[m];
