@@ -606,23 +606,29 @@ __device__ __forceinline__ void tile_epilogue(const UArgs& a, umma::Ctl& ctl, in
         rv[j] = (a.res && valid && mg + j < mc)
                     ? (res_pre ? ctl.land[(mg + j) * 128 + r] : __ldcg(a.res + (size_t)(m0 + mg + j) * a.ldr + n))
                     : 0.f;
+      float sq[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int m = mg + j;
+        sq[j] = 0.f;
         if (m < mc) {   // uniform across the threads
-          float sq = 0.f;
           if (valid && !dry) {
             const float x = acc[m * 128] * ctl.scale[m0 + m] + bias + rv[j];
             a.out[(size_t)(m0 + m) * a.ldo + n] = x;
-            sq = x * x;
+            sq[j] = x * x;
             if (a.out_hi)
               split_store(a.out_hi + (size_t)(m0 + m) * a.ld_plane + n, a.out_lo + (size_t)(m0 + m) * a.ld_plane + n, x * gain);
           }
-          if (a.ssq_out) {
-            sq = warp_sum(sq);
-            if (lane == 0) ctl.red[q][m] = sq;
-          }
         }
+      }
+      if (a.ssq_out) {   // the eight rows' warp sums side by side (same tree as warp_sum)
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+          for (int j = 0; j < 8; ++j) sq[j] += __shfl_xor_sync(0xffffffffu, sq[j], o);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (lane == 0 && mg + j < mc) ctl.red[q][mg + j] = sq[j];
       }
     }
     if (a.ssq_out) {
