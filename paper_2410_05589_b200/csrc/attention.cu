@@ -339,17 +339,20 @@ __global__ void __launch_bounds__(kAttnThreads, NB == 1 ? 3 : 2) k_attn_mma(
     const int row_f = n_split * D;                        // floats per row
     const int rows_pass = max(1, (2 * tile * P * 2) / (row_f * 4));
     const float2* ml2 = reinterpret_cast<const float2*>(att_ml);
-    for (int idx = tid; idx < R * n_split; idx += kAttnThreads) {
-      const int j = idx / n_split, sp = idx - j * n_split;
-      s_ml[idx] = __ldcg(ml2 + ((size_t)(m0 + j) * n_heads + h) * n_split + sp);
-    }
     for (int j0 = 0; j0 < R; j0 += rows_pass) {
       const int nr = min(rows_pass, R - j0), vec_row = row_f / 4;
       for (int idx = tid; idx < nr * vec_row; idx += kAttnThreads) {
         const int jr = idx / vec_row, off = (idx - jr * vec_row) * 4;
         cp_async16(s_o + jr * row_f + off, att_o + ((size_t)(m0 + j0 + jr) * n_heads + h) * row_f + off);
       }
-      asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      if (j0 == 0) {   // (while the copies are on their way)
+        for (int idx = tid; idx < R * n_split; idx += kAttnThreads) {
+          const int j = idx / n_split, sp = idx - j * n_split;
+          s_ml[idx] = __ldcg(ml2 + ((size_t)(m0 + j) * n_heads + h) * n_split + sp);
+        }
+      }
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
       __syncthreads();
       for (int idx = tid; idx < nr * D; idx += kAttnThreads) {
         const int jr = idx / D, d = idx - jr * D, j = j0 + jr;
