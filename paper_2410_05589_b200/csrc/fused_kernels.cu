@@ -1982,22 +1982,25 @@ ps_status umma_kv_append(ps_ctx* c, const UmmaMaps& u, const SeqMap& sm, int row
                                 f.xin);
   c->launches++;
   if (ge != cudaSuccess) return cuda_check(c, ge, "k_gather_x");
+  // (up to 16 rows the two stages share a launch, like fc and q|k|v of a draft step)
+  const bool chain = rows <= 16 && (!c->prof || c->prof_launches) && !(g.flags & PS_FLAG_STAGE_LAUNCHES);
+  StageDesc d[2];
   {
-    UArgs a{};
+    d[0] = StageDesc{EPI_STORE, &u.w_fc, &u.w_fc, &u.w_fc, &u.xin, &u.xin, UArgs{}, "fc_norm"};
+    UArgs& a = d[0].a;
     a.N = H; a.K = 2 * H; a.M = rows; a.n_mats = 1; a.mat_rows[0] = H; a.lo = 0;
     a.out = c->x0; a.ldo = H; a.bias = (g.flags & PS_FLAG_FC_BIAS) ? (BP)w.b_fc : nullptr;
     a.ssq_out = f.ssq[0];
     a.out_hi = f.x0p.hi; a.out_lo = f.x0p.lo; a.ld_plane = H; a.gain_next = (BP)w.g_in;
-    if ((s = launch_umma<EPI_STORE>(c, u.w_fc, u.w_fc, u.w_fc, u.xin, u.xin, a, f, st))) return s;
   }
-  prof_mark(c, st, "fc_norm");
   {
-    UArgs a{};
+    d[1] = StageDesc{EPI_STORE, &u.w_k, &u.w_v, &u.w_v, &u.x0_hi, &u.x0_lo, UArgs{}, nullptr};
+    UArgs& a = d[1].a;
     a.N = 2 * Hkv; a.K = H; a.M = rows; a.n_mats = 2; a.mat_rows[0] = Hkv; a.mat_rows[1] = Hkv; a.lo = 1;
     a.ssq_in = f.ssq[0]; a.ssq_n = tiles_h; a.eps = g.rms_eps;
     a.out = c->kv_tmp; a.ldo = 2 * Hkv;
-    if ((s = launch_umma<EPI_STORE>(c, u.w_k, u.w_v, u.w_v, u.x0_hi, u.x0_lo, a, f, st))) return s;
   }
+  if ((s = run_stages(c, d, 2, chain, 0, f, st))) return s;
   if ((s = launch_rope_store_kv(c, sm, rows, st))) return s;
   prof_mark(c, st, "qkv_rope");
   return PS_OK;

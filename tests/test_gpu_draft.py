@@ -232,6 +232,27 @@ def test_chained_stages_equal_stage_launches(name, B):
         assert np.array_equal(outs[0][k], outs[1][k]), k
 
 
+def test_stage_timers_and_launch_timers():
+    """ps_profile(ctx, 1) times every stage (a launch per GEMM stage), ps_profile(ctx, 2) every launch
+    (the chained stages stay chained); the outputs do not depend on the mode."""
+    s = synth.CONFIGS["mini"]
+    p = Pair(s, s.batch)
+    ref = p.gpu_step(top_n=2)
+    seen = {}
+    for mode in (1, 2):
+        p.g.profile(mode)
+        got = p.gpu_step(top_n=2)
+        torch.cuda.synchronize()
+        seen[mode] = p.g.profile_read()
+        p.g.profile(0)
+        assert np.array_equal(got["logits"], ref["logits"]) and np.array_equal(got["top_ids"], ref["top_ids"])
+    for name in ("fc_norm", "qkv_rope", "attention", "o_proj", "ffn_gate_up", "ffn_down", "lm_head"):
+        assert name in seen[1] and seen[1][name][1] >= 1, (name, seen[1])
+    assert "chain_fc_qkv" in seen[2] and "chain_o_ffn_lm" in seen[2] and "attention" in seen[2], seen[2]
+    assert "ffn_down" not in seen[2] and "o_proj" not in seen[2], seen[2]
+    assert p.g.poll() == 0
+
+
 _W13 = {}
 
 
