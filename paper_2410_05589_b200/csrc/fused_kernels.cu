@@ -1271,11 +1271,14 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tA0, const __grid_constant__ CUt
 // memory (release); the producer thread and one epilogue thread of every CTA wait for the count
 // (acquire, bounded), and the last of them to see it complete zeroes it for the next launch.
 // The CTAs wait for one another, so all must be resident at once: one CTA per SM, see the
-// launch in run_stages; every wait is bounded.  The tail of a tile (partials, ticket, sum of
-// the partials, epilogue, count) is a chain of round trips to L2 and is what a stage costs
-// beyond its stream: partials are kept as 16-byte vectors per accumulator row so that the last
-// arriver has all contributors' values in flight at once, and what does not depend on the sums
-// (who shares the tile, the residual rows) is fetched while the MMAs still run.
+// launch in run_stages; every wait is bounded.  The tail of a tile (partials out, count, sum of
+// the partials, epilogue, release) is a chain of round trips to L2 and is what a stage costs
+// beyond its stream.  The owner of a tile's last k-block is its finisher: the other
+// contributors store their partial and count themselves in, one thread of the finisher waits
+// for the count while its own sums stay in registers; partials are kept as 16-byte vectors per
+// accumulator row so that the finisher has all contributors' values in flight at once, and
+// what does not depend on the sums (who shares the tile, the residual rows) is fetched while
+// the MMAs still run.
 constexpr int kChainMax = 4, kChainMaps = 13;
 struct ChainParams {
   int n;                                  // stages
